@@ -1,0 +1,152 @@
+/*
+ * moe.h - C ABI of the B200 (sm_100a) mixture-of-experts FFN layer, forward and backward.
+ *
+ * The layer is the MoE block of a Qwen3-30B-A3B-style reranker (paper, Section "Expert-Parallel MoE
+ * Training": 128 experts, top-8 routing; the LoRA target-group listing names its parts: router.weight,
+ * experts.*.linear_fc1, experts.*.linear_fc2).  Every expert is local to the GPU (expert-parallel degree 1).
+ *
+ *   forward :  l = x W_r (+ b_r)                     fp32 logits
+ *              p = softmax(l)                         over all E experts
+ *              idx = top-k of l                       lowest index wins ties, stored in pick order
+ *              g = p[idx] / sum p[idx]                renormalised gates
+ *              rows sorted by (expert, token)         counts, perm
+ *              a = silu(x W_gate[e]) * (x W_up[e])    per routed row, SwiGLU
+ *              o = a W_down[e]
+ *              y[t] = sum_j g[t,j] o[t,j]
+ *              aux = E * sum_e (c_e / (T k)) * mean_t p[t,e]
+ *   backward:  gradients of  <y, dy> + d_aux * aux  with respect to x, W_r, b_r, W_gate, W_up, W_down,
+ *              routing decisions held fixed.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  Tensors are dense row-major.
+ *   - bf16 tensors are passed as uint16_t bit patterns.  Pointers must be 16-byte aligned.
+ *   - The caller owns every buffer, the workspace included.  No entry point allocates or frees device
+ *     memory.
+ *   - All work is enqueued on the caller's CUDA stream (passed as void* = cudaStream_t).  Neither
+ *     moe_forward nor moe_backward synchronises with the host or copies anything to the host: expert
+ *     counts stay on the device and drive the tile schedulers there.
+ *   - Errors are return codes.  Argument errors are found before anything is launched.  A device-side
+ *     problem (a bounded wait that ran out) sets a status word inside the workspace; the kernels leave
+ *     cleanly and moe_poll_status reports it.
+ *   - Inputs must be finite.  One moe_ctx serves one stream at a time.
+ */
+#ifndef MOE_B200_H
+#define MOE_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define MOE_API __attribute__((visibility("default")))
+#else
+#define MOE_API
+#endif
+
+typedef struct {
+  int32_t d;      /* model width,  multiple of 64                                  */
+  int32_t E;      /* experts,      1 <= E <= 256                                   */
+  int32_t f;      /* expert width, multiple of 64                                  */
+  int32_t top_k;  /* experts per token, 1 <= top_k <= E and top_k <= 32            */
+  int32_t flags;  /* reserved, pass 0                                              */
+} moe_config;
+
+typedef struct moe_ctx moe_ctx; /* opaque, lives in host memory */
+
+typedef enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = -1,
+  MOE_ERR_UNSUPPORTED = -2,
+  MOE_ERR_WORKSPACE = -3,   /* workspace_bytes smaller than moe_workspace_bytes(ctx, T) */
+  MOE_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                       */
+  MOE_ERR_DEVICE_TIMEOUT = -5 /* a bounded device-side wait ran out                      */
+} moe_status;
+
+/* Number of per-stage timers filled by moe_stage_times (see below). */
+#define MOE_NUM_STAGES 16
+
+/* Creates a context for one layer shape on the current device.  Allocates host memory only. */
+MOE_API moe_status moe_create(const moe_config* cfg /* host */, moe_ctx** out /* host */);
+MOE_API void moe_destroy(moe_ctx* ctx);
+
+/* Bytes of workspace needed for a call with T tokens (0 if ctx is NULL or T < 0).  The workspace holds
+ * the routing tables and the activations that moe_forward saves for moe_backward. */
+MOE_API size_t moe_workspace_bytes(const moe_ctx* ctx, int64_t T);
+
+/* Byte offset and size of a named internal buffer inside the workspace, for stage-by-stage tests.
+ * Names: "counts" "offsets" "pad_offsets" "logits" "idx" "gates" "inv" "row_token" "xp" "hg" "hu" "act"
+ * "o" "dhg" "dhu" "dxp" "dg" "dl".  Internal row buffers (xp, hg, hu, act, o, dhg, dhu, dxp) are laid out
+ * expert-major with every expert's segment padded to a multiple of 128 rows ("pad_offsets"); pad rows
+ * are zero.  Returns MOE_ERR_INVALID_ARG for an unknown name. */
+MOE_API moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char* name /* host */,
+                              size_t* offset /* host */, size_t* bytes /* host */);
+
+MOE_API const char* moe_status_string(moe_status s);
+
+/* Synchronises the stream and returns the device-side status word of the workspace. */
+MOE_API moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_stream);
+
+/* Per-stage timing.  With enable != 0, moe_forward / moe_backward record CUDA events between their
+ * kernels on the caller's stream.  moe_stage_times synchronises on those events and adds, for each stage,
+ * the milliseconds of the last forward+backward pair to ms[0..MOE_NUM_STAGES) (host array).
+ * Stage order: 0 router, 1 permute (histogram, scan, scatter, gather), 2 gate/up GEMM + SwiGLU,
+ * 3 down GEMM, 4 combine, 5 combine-bwd, 6 dgrad-down + SwiGLU-bwd, 7 wgrad-down, 8 dgrad gate/up,
+ * 9 wgrad gate/up, 10 router-bwd (dl), 11 dW_r, 12 unpermute-bwd (dx), 13..15 unused. */
+MOE_API moe_status moe_set_profiling(moe_ctx* ctx, int enable);
+MOE_API moe_status moe_stage_times(moe_ctx* ctx, float* ms /* host, MOE_NUM_STAGES floats */);
+
+/* Forward pass over T tokens (T >= 0).
+ *   x          [T,d]   bf16
+ *   W_r        [d,E]   bf16 router weight; the contraction accumulates in fp32
+ *   b_r        [E]     fp32 additive logit bias, or NULL
+ *   logits_in  [T,E]   fp32, or NULL.  When given, routing starts from these logits and the router
+ *                      contraction is skipped (test hook: lets a caller construct exact ties).
+ *   W_gate,W_up [E,d,f] bf16        W_down [E,f,d] bf16
+ * Outputs
+ *   y          [T,d]   bf16
+ *   topk_idx   [T,k]   int32, pick order (descending logit, ties ascending index)
+ *   topk_w     [T,k]   fp32 gates, each row sums to 1
+ *   expert_counts [E]  int32
+ *   perm       [T*k]   int32 or NULL: perm[r] = t*k + j of the pair in row r of the expert-major order
+ *                      (rows sorted by expert, then token)
+ *   aux_loss   [1]     fp32, coefficient-free
+ *   logits_out [T,E]   fp32 or NULL
+ * The workspace must be at least moe_workspace_bytes(ctx, T) bytes and must stay untouched until the
+ * matching moe_backward has run. */
+MOE_API moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                       const float* logits_in, const uint16_t* W_gate, const uint16_t* W_up,
+                       const uint16_t* W_down, uint16_t* y, int32_t* topk_idx, float* topk_w,
+                       int32_t* expert_counts, int32_t* perm, float* aux_loss, float* logits_out,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward pass of the forward call that filled `workspace`.
+ *   dy    [T,d] bf16 upstream gradient of y;  d_aux: host scalar, dLoss/d(aux_loss)
+ *   x, W_r, W_gate, W_up, W_down: the forward inputs
+ * Outputs (all OVERWRITTEN, not accumulated)
+ *   dx [T,d] bf16;  dW_r [d,E] fp32;  db_r [E] fp32 or NULL;
+ *   dW_gate, dW_up [E,d,f] bf16;  dW_down [E,f,d] bf16 (zero slabs for experts without tokens). */
+MOE_API moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
+                        const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                        const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
+                        uint16_t* dW_up, uint16_t* dW_down, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+
+/* Host-buffer convenience used for end-to-end timing: every tensor argument is a HOST pointer (pinned
+ * memory recommended); the call copies inputs to the device buffers of `dev` (a device scratch of
+ * moe_e2e_device_bytes(ctx, T) bytes owned by the caller), runs forward and backward, copies y, dx, aux and
+ * the weight gradients back and synchronises the stream.  copy_weights != 0 also uploads the weights and
+ * downloads their gradients; with 0 the weights must already be resident from an earlier call. */
+MOE_API size_t moe_e2e_device_bytes(const moe_ctx* ctx, int64_t T);
+MOE_API moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16_t* x, const uint16_t* W_r,
+                         const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
+                         const uint16_t* dy, float d_aux, uint16_t* y, float* aux_loss, uint16_t* dx,
+                         float* dW_r, uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down,
+                         void* dev /* device */, size_t dev_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H */

@@ -1,0 +1,209 @@
+"""ctypes binding of the C ABI in include/moe.h.  Argument marshalling only: every step of the layer runs in
+the CUDA library.  torch supplies device memory and the current stream; there is no fallback path - if the
+shared library is missing or the device is not an sm_100a GPU, calls raise."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
+NUM_STAGES = 16
+STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine", "combine_bwd",
+               "dgrad_down_swiglu_bwd", "wgrad_down", "dgrad_gateup", "wgrad_gateup", "router_bwd", "dW_r",
+               "unpermute_bwd"]
+EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
+           "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
+           "moe_e2e_device_bytes", "moe_step_host"]
+
+
+class MoEConfig(C.Structure):
+    _fields_ = [("d", C.c_int32), ("E", C.c_int32), ("f", C.c_int32), ("top_k", C.c_int32), ("flags", C.c_int32)]
+
+
+class MoEError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads libmoe_b200.so built in-tree (python -m paper_2608_00916_b200.build).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise MoEError(f"{LIB_PATH} not found: build it with `python -m paper_2608_00916_b200.build`")
+    lib = C.CDLL(LIB_PATH)
+    vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+    lib.moe_create.argtypes = [C.POINTER(MoEConfig), C.POINTER(vp)]
+    lib.moe_create.restype = C.c_int
+    lib.moe_destroy.argtypes = [vp]
+    lib.moe_destroy.restype = None
+    lib.moe_workspace_bytes.argtypes = [vp, i64]
+    lib.moe_workspace_bytes.restype = sz
+    lib.moe_workspace_find.argtypes = [vp, i64, C.c_char_p, C.POINTER(sz), C.POINTER(sz)]
+    lib.moe_workspace_find.restype = C.c_int
+    lib.moe_status_string.argtypes = [C.c_int]
+    lib.moe_status_string.restype = C.c_char_p
+    lib.moe_poll_status.argtypes = [vp, vp, vp]
+    lib.moe_poll_status.restype = C.c_int
+    lib.moe_set_profiling.argtypes = [vp, C.c_int]
+    lib.moe_set_profiling.restype = C.c_int
+    lib.moe_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.moe_stage_times.restype = C.c_int
+    lib.moe_forward.argtypes = [vp, i64] + [vp] * 14 + [vp, sz, vp]
+    lib.moe_forward.restype = C.c_int
+    lib.moe_backward.argtypes = [vp, i64, vp, C.c_float] + [vp] * 11 + [vp, sz, vp]
+    lib.moe_backward.restype = C.c_int
+    lib.moe_e2e_device_bytes.argtypes = [vp, i64]
+    lib.moe_e2e_device_bytes.restype = sz
+    lib.moe_step_host.argtypes = [vp, i64, C.c_int] + [vp] * 6 + [C.c_float] + [vp] * 7 + [vp, sz, vp]
+    lib.moe_step_host.restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _check(lib, rc: int, what: str) -> None:
+    if rc != 0:
+        raise MoEError(f"{what}: {lib.moe_status_string(rc).decode()} ({rc})")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class MoELayer:
+    """One MoE FFN layer shape (d, E, f, top_k) bound to the CUDA library.
+
+    forward() / backward() take and return torch CUDA tensors (bf16 for activations and weights); the
+    tensors are only carriers of device pointers."""
+
+    def __init__(self, d: int, E: int, f: int, top_k: int):
+        self.lib = load_library()
+        self.d, self.E, self.f, self.k = d, E, f, top_k
+        cfg = MoEConfig(d, E, f, top_k, 0)
+        h = C.c_void_p()
+        _check(self.lib, self.lib.moe_create(C.byref(cfg), C.byref(h)), "moe_create")
+        self.h = h
+        self.ws = None
+        self.T = None
+        self._saved = None
+
+    def __del__(self):
+        try:
+            if getattr(self, "h", None):
+                self.lib.moe_destroy(self.h)
+                self.h = None
+        except Exception:
+            pass
+
+    # ---- workspace
+    def workspace_bytes(self, T: int) -> int:
+        return int(self.lib.moe_workspace_bytes(self.h, T))
+
+    def find(self, T: int, name: str):
+        off, n = C.c_size_t(), C.c_size_t()
+        _check(self.lib, self.lib.moe_workspace_find(self.h, T, name.encode(), C.byref(off), C.byref(n)),
+               f"moe_workspace_find({name})")
+        return off.value, n.value
+
+    def buffer(self, name: str, dtype):
+        """View of an internal workspace buffer of the last forward call (for stage-by-stage tests)."""
+        off, n = self.find(self.T, name)
+        return self.ws[off:off + n].view(dtype)
+
+    def _ensure_ws(self, T: int):
+        import torch
+        need = self.workspace_bytes(T)
+        if self.ws is None or self.ws.numel() < need:
+            self.ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+        self.T = T
+
+    def _stream(self):
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    # ---- calls
+    def forward(self, x, W_r, W_gate, W_up, W_down, b_r=None, logits_in=None, want_logits=False, want_perm=True):
+        import torch
+        T = x.shape[0]
+        d, E, f, k = self.d, self.E, self.f, self.k
+        assert x.dtype == torch.bfloat16 and tuple(x.shape) == (T, d) and x.is_contiguous()
+        assert tuple(W_r.shape) == (d, E) and W_r.dtype == torch.bfloat16 and W_r.is_contiguous()
+        for w, shp in ((W_gate, (E, d, f)), (W_up, (E, d, f)), (W_down, (E, f, d))):
+            assert tuple(w.shape) == shp and w.dtype == torch.bfloat16 and w.is_contiguous()
+        self._ensure_ws(T)
+        dev = x.device
+        out = {
+            "y": torch.empty(T, d, dtype=torch.bfloat16, device=dev),
+            "idx": torch.empty(T, k, dtype=torch.int32, device=dev),
+            "gates": torch.empty(T, k, dtype=torch.float32, device=dev),
+            "counts": torch.empty(E, dtype=torch.int32, device=dev),
+            "perm": torch.empty(T * k, dtype=torch.int32, device=dev) if want_perm else None,
+            "aux": torch.empty(1, dtype=torch.float32, device=dev),
+            "logits": torch.empty(T, E, dtype=torch.float32, device=dev) if want_logits else None,
+        }
+        if b_r is not None:
+            assert b_r.dtype == torch.float32 and b_r.numel() == E
+        if logits_in is not None:
+            assert logits_in.dtype == torch.float32 and tuple(logits_in.shape) == (T, E) and logits_in.is_contiguous()
+        rc = self.lib.moe_forward(self.h, T, _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(logits_in), _ptr(W_gate), _ptr(W_up),
+                                  _ptr(W_down), _ptr(out["y"]), _ptr(out["idx"]), _ptr(out["gates"]),
+                                  _ptr(out["counts"]), _ptr(out["perm"]), _ptr(out["aux"]), _ptr(out["logits"]),
+                                  _ptr(self.ws), self.ws.numel(), self._stream())
+        _check(self.lib, rc, "moe_forward")
+        self._saved = (x, W_r, W_gate, W_up, W_down)
+        return out
+
+    def backward(self, dy, d_aux: float, want_db: bool = False, grads=None):
+        """Gradients for the last forward().  `grads` may carry preallocated output tensors."""
+        import torch
+        x, W_r, W_gate, W_up, W_down = self._saved
+        T = x.shape[0]
+        d, E, f = self.d, self.E, self.f
+        assert dy.dtype == torch.bfloat16 and tuple(dy.shape) == (T, d) and dy.is_contiguous()
+        dev = x.device
+        g = grads or {}
+        out = {
+            "dx": g.get("dx", None) if g.get("dx", None) is not None else torch.empty(T, d, dtype=torch.bfloat16, device=dev),
+            "dW_r": g.get("dW_r") if g.get("dW_r") is not None else torch.empty(d, E, dtype=torch.float32, device=dev),
+            "db_r": torch.empty(E, dtype=torch.float32, device=dev) if want_db else None,
+            "dW_gate": g.get("dW_gate") if g.get("dW_gate") is not None else torch.empty(E, d, f, dtype=torch.bfloat16, device=dev),
+            "dW_up": g.get("dW_up") if g.get("dW_up") is not None else torch.empty(E, d, f, dtype=torch.bfloat16, device=dev),
+            "dW_down": g.get("dW_down") if g.get("dW_down") is not None else torch.empty(E, f, d, dtype=torch.bfloat16, device=dev),
+        }
+        rc = self.lib.moe_backward(self.h, T, _ptr(dy), C.c_float(d_aux), _ptr(x), _ptr(W_r), _ptr(W_gate), _ptr(W_up),
+                                   _ptr(W_down), _ptr(out["dx"]), _ptr(out["dW_r"]), _ptr(out["db_r"]),
+                                   _ptr(out["dW_gate"]), _ptr(out["dW_up"]), _ptr(out["dW_down"]), _ptr(self.ws),
+                                   self.ws.numel(), self._stream())
+        _check(self.lib, rc, "moe_backward")
+        return out
+
+    def poll(self) -> None:
+        """Synchronises and raises if a device-side bounded wait ran out."""
+        _check(self.lib, self.lib.moe_poll_status(self.h, _ptr(self.ws), self._stream()), "device status")
+
+    def set_profiling(self, on: bool) -> None:
+        _check(self.lib, self.lib.moe_set_profiling(self.h, 1 if on else 0), "moe_set_profiling")
+
+    def stage_times(self, acc=None):
+        """Adds the per-stage milliseconds of the last forward+backward to `acc` (list of NUM_STAGES floats)."""
+        arr = (C.c_float * NUM_STAGES)(*(acc or [0.0] * NUM_STAGES))
+        _check(self.lib, self.lib.moe_stage_times(self.h, arr), "moe_stage_times")
+        return list(arr)
+
+    # ---- host-buffer step (end-to-end timing)
+    def e2e_device_bytes(self, T: int) -> int:
+        return int(self.lib.moe_e2e_device_bytes(self.h, T))
+
+    def step_host(self, T, dev_buf, host, d_aux: float, copy_weights: bool):
+        """host: dict of pinned CPU tensors x, W_r, W_gate, W_up, W_down, dy and outputs y, aux, dx, dW_r, dW_gate,
+        dW_up, dW_down.  dev_buf: uint8 CUDA tensor of e2e_device_bytes(T)."""
+        hp = lambda n: None if host.get(n) is None else C.c_void_p(host[n].data_ptr())
+        rc = self.lib.moe_step_host(self.h, T, 1 if copy_weights else 0, hp("x"), hp("W_r"), hp("W_gate"), hp("W_up"),
+                                    hp("W_down"), hp("dy"), C.c_float(d_aux), hp("y"), hp("aux"), hp("dx"), hp("dW_r"),
+                                    hp("dW_gate"), hp("dW_up"), hp("dW_down"), _ptr(dev_buf), dev_buf.numel(),
+                                    self._stream())
+        _check(self.lib, rc, "moe_step_host")

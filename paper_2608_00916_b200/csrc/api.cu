@@ -1,0 +1,423 @@
+// C ABI of the MoE layer library (see include/moe.h): argument checks, workspace layout, kernel sequencing.
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace moe {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+WsLayout make_layout(const Shape& s, int64_t T) {
+  WsLayout L;
+  memset(&L, 0, sizeof(L));
+  const int64_t R = T * s.k;
+  L.max_m_tiles = (R + ROW_PAD - 1) / ROW_PAD + s.E;
+  L.rows_max = L.max_m_tiles * ROW_PAD;
+  L.tok_tiles = (T + TOK_TILE - 1) / TOK_TILE;
+  L.router_blocks = (T + ROUTER_TOK - 1) / ROUTER_TOK;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  L.status = take(sizeof(int32_t) * 16);
+  L.counts = take(sizeof(int32_t) * s.E);
+  L.offsets = take(sizeof(int32_t) * (s.E + 1));
+  L.pad_offsets = take(sizeof(int32_t) * (s.E + 1));
+  L.sched = take(sizeof(int32_t) * 4);
+  L.tile_expert = take(sizeof(int32_t) * L.max_m_tiles);
+  L.tile_counts = take(sizeof(int32_t) * (L.tok_tiles + 1) * s.E);
+  L.psum_part = take(sizeof(float) * (L.router_blocks + 1) * s.E);
+  L.psum = take(sizeof(float) * s.E);
+  L.logits = take(sizeof(float) * T * s.E);
+  L.idx = take(sizeof(int32_t) * R);
+  L.gates = take(sizeof(float) * R);
+  L.inv = take(sizeof(int32_t) * R);
+  L.row_token = take(sizeof(int32_t) * L.rows_max);
+  L.dg = take(sizeof(float) * R);
+  L.dl = take(sizeof(float) * T * s.E);
+  L.dwr_part = take(sizeof(float) * DWR_SPLIT * s.d * s.E);
+  const size_t rows_d = sizeof(uint16_t) * L.rows_max * s.d, rows_f = sizeof(uint16_t) * L.rows_max * s.f;
+  L.xp = take(rows_d);
+  L.hg = take(rows_f);
+  L.hu = take(rows_f);
+  L.act = take(rows_f);
+  L.o = take(rows_d);
+  L.dhg = take(rows_f);
+  L.dhu = take(rows_f);
+  L.dxp = take(rows_d);
+  L.total = off;
+  return L;
+}
+
+static moe_status ensure_device(moe_ctx_impl* c) {
+  if (c->encode_fn) return MOE_OK;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return MOE_ERR_CUDA;
+  if (prop.major != 10) return MOE_ERR_UNSUPPORTED;  // tcgen05 / TMEM kernels: sm_100a only, no fallback
+  c->device = dev;
+  c->sm_count = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess)
+    return MOE_ERR_CUDA;
+  c->encode_fn = fn;
+  return MOE_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct StageTimer {
+  moe_ctx_impl* c;
+  cudaStream_t st;
+  int stage;
+  StageTimer(moe_ctx_impl* c_, cudaStream_t st_, int stage_) : c(c_), st(st_), stage(stage_) {
+    if (c->profiling) {
+      cudaEventRecord(c->ev[stage][0], st);
+    }
+  }
+  ~StageTimer() {
+    if (c->profiling) {
+      cudaEventRecord(c->ev[stage][1], st);
+      c->ev_used[stage] = 1;
+    }
+  }
+};
+
+}  // namespace moe
+
+using namespace moe;
+
+extern "C" {
+
+moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
+  if (!cfg || !out) return MOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->d <= 0 || cfg->f <= 0 || cfg->d % 64 != 0 || cfg->f % 64 != 0) return MOE_ERR_INVALID_ARG;
+  if (cfg->E < 1 || cfg->E > MAX_E) return MOE_ERR_INVALID_ARG;
+  if (cfg->top_k < 1 || cfg->top_k > cfg->E || cfg->top_k > MAX_K) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = new (std::nothrow) moe_ctx_impl;
+  if (!c) return MOE_ERR_INVALID_ARG;
+  memset(c, 0, sizeof(*c));
+  c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
+  *out = reinterpret_cast<moe_ctx*>(c);
+  return MOE_OK;
+}
+
+void moe_destroy(moe_ctx* ctx) {
+  if (!ctx) return;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  if (c->ev_created)
+    for (int i = 0; i < MOE_NUM_STAGES; ++i) {
+      cudaEventDestroy(c->ev[i][0]);
+      cudaEventDestroy(c->ev[i][1]);
+    }
+  delete c;
+}
+
+size_t moe_workspace_bytes(const moe_ctx* ctx, int64_t T) {
+  if (!ctx || T < 0) return 0;
+  const moe_ctx_impl* c = reinterpret_cast<const moe_ctx_impl*>(ctx);
+  return make_layout(c->s, T).total;
+}
+
+moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char* name, size_t* offset, size_t* bytes) {
+  if (!ctx || !name || !offset || !bytes || T < 0) return MOE_ERR_INVALID_ARG;
+  const moe_ctx_impl* c = reinterpret_cast<const moe_ctx_impl*>(ctx);
+  const Shape& s = c->s;
+  const WsLayout L = make_layout(s, T);
+  const size_t R = static_cast<size_t>(T) * s.k;
+  const size_t rows_d = sizeof(uint16_t) * L.rows_max * s.d, rows_f = sizeof(uint16_t) * L.rows_max * s.f;
+  struct Ent {
+    const char* n;
+    size_t off, sz;
+  } tab[] = {{"counts", L.counts, sizeof(int32_t) * s.E},
+             {"offsets", L.offsets, sizeof(int32_t) * (s.E + 1)},
+             {"pad_offsets", L.pad_offsets, sizeof(int32_t) * (s.E + 1)},
+             {"logits", L.logits, sizeof(float) * T * s.E},
+             {"idx", L.idx, sizeof(int32_t) * R},
+             {"gates", L.gates, sizeof(float) * R},
+             {"inv", L.inv, sizeof(int32_t) * R},
+             {"row_token", L.row_token, sizeof(int32_t) * L.rows_max},
+             {"xp", L.xp, rows_d},
+             {"hg", L.hg, rows_f},
+             {"hu", L.hu, rows_f},
+             {"act", L.act, rows_f},
+             {"o", L.o, rows_d},
+             {"dhg", L.dhg, rows_f},
+             {"dhu", L.dhu, rows_f},
+             {"dxp", L.dxp, rows_d},
+             {"dg", L.dg, sizeof(float) * R},
+             {"dl", L.dl, sizeof(float) * T * s.E},
+             {"status", L.status, sizeof(int32_t) * 16}};
+  for (const Ent& e : tab)
+    if (strcmp(e.n, name) == 0) {
+      *offset = e.off;
+      *bytes = e.sz;
+      return MOE_OK;
+    }
+  return MOE_ERR_INVALID_ARG;
+}
+
+const char* moe_status_string(moe_status s) {
+  switch (s) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_ERR_UNSUPPORTED: return "unsupported device or configuration (sm_100a required)";
+    case MOE_ERR_WORKSPACE: return "workspace too small";
+    case MOE_ERR_CUDA: return "CUDA call failed";
+    case MOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_stream) {
+  if (!ctx || !workspace) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  const WsLayout L = make_layout(c->s, 0);
+  int32_t st[2] = {0, 0};
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(st, static_cast<const char*>(workspace) + L.status, sizeof(st), cudaMemcpyDeviceToHost, s) !=
+      cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return MOE_ERR_CUDA;
+  return st[0] == DEV_OK ? MOE_OK : MOE_ERR_DEVICE_TIMEOUT;
+}
+
+moe_status moe_set_profiling(moe_ctx* ctx, int enable) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  if (enable && !c->ev_created) {
+    for (int i = 0; i < MOE_NUM_STAGES; ++i)
+      if (cudaEventCreate(&c->ev[i][0]) != cudaSuccess || cudaEventCreate(&c->ev[i][1]) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    c->ev_created = 1;
+  }
+  c->profiling = enable ? 1 : 0;
+  return MOE_OK;
+}
+
+moe_status moe_stage_times(moe_ctx* ctx, float* ms) {
+  if (!ctx || !ms) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  for (int i = 0; i < MOE_NUM_STAGES; ++i) {
+    if (!c->ev_used[i]) continue;
+    if (cudaEventSynchronize(c->ev[i][1]) != cudaSuccess) return MOE_ERR_CUDA;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, c->ev[i][0], c->ev[i][1]) != cudaSuccess) return MOE_ERR_CUDA;
+    ms[i] += t;
+  }
+  return MOE_OK;
+}
+
+moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                       const float* logits_in, const uint16_t* W_gate, const uint16_t* W_up,
+                       const uint16_t* W_down, uint16_t* y, int32_t* topk_idx, float* topk_w,
+                       int32_t* expert_counts, int32_t* perm, float* aux_loss, float* logits_out,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  const Shape& s = c->s;
+  if (!W_gate || !W_up || !W_down || !expert_counts || !aux_loss || !workspace) return MOE_ERR_INVALID_ARG;
+  if (T > 0 && (!x || !y || !topk_idx || !topk_w || (!W_r && !logits_in))) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_gate) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(y) ||
+      !aligned16(workspace) || !aligned16(W_r))
+    return MOE_ERR_INVALID_ARG;
+  if (T * s.k > (int64_t(1) << 30)) return MOE_ERR_UNSUPPORTED;
+  const WsLayout L = make_layout(s, T);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE;
+  moe_status rc = ensure_device(c);
+  if (rc != MOE_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  {
+    StageTimer tm(c, st, 0);
+    launch_router(s, T, x, W_r, b_r, logits_in, reinterpret_cast<float*>(ws + L.logits),
+                  reinterpret_cast<int32_t*>(ws + L.idx), reinterpret_cast<float*>(ws + L.gates), topk_idx, topk_w,
+                  logits_out, reinterpret_cast<float*>(ws + L.psum_part), st);
+  }
+  {
+    StageTimer tm(c, st, 1);
+    launch_permute(s, T, L, ws, x, expert_counts, perm, aux_loss, st);
+  }
+  if (T > 0) {
+    {
+      StageTimer tm(c, st, 2);
+      rc = launch_grouped_gemm(c, GEMM_F3, T, L, ws, W_gate, W_up, W_down, nullptr, nullptr, nullptr, st);
+    }
+    if (rc != MOE_OK) return rc;
+    {
+      StageTimer tm(c, st, 3);
+      rc = launch_grouped_gemm(c, GEMM_F4, T, L, ws, W_gate, W_up, W_down, nullptr, nullptr, nullptr, st);
+    }
+    if (rc != MOE_OK) return rc;
+    {
+      StageTimer tm(c, st, 4);
+      launch_combine(s, T, reinterpret_cast<const uint16_t*>(ws + L.o), reinterpret_cast<const float*>(ws + L.gates),
+                     reinterpret_cast<const int32_t*>(ws + L.inv), y, st);
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
+                        const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                        const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
+                        uint16_t* dW_up, uint16_t* dW_down, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+  if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  const Shape& s = c->s;
+  if (!W_r || !W_gate || !W_up || !W_down || !dW_r || !dW_gate || !dW_up || !dW_down || !workspace)
+    return MOE_ERR_INVALID_ARG;
+  if (T > 0 && (!dy || !x || !dx)) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(W_r) || !aligned16(W_gate) || !aligned16(W_up) ||
+      !aligned16(W_down) || !aligned16(dx) || !aligned16(dW_gate) || !aligned16(dW_up) || !aligned16(dW_down) ||
+      !aligned16(workspace))
+    return MOE_ERR_INVALID_ARG;
+  const WsLayout L = make_layout(s, T);
+  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE;
+  moe_status rc = ensure_device(c);
+  if (rc != MOE_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  float* dl = reinterpret_cast<float*>(ws + L.dl);
+  const int32_t* inv = reinterpret_cast<const int32_t*>(ws + L.inv);
+  const float* gates = reinterpret_cast<const float*>(ws + L.gates);
+  {
+    StageTimer tm(c, st, 5);
+    launch_combine_bwd(s, T, dy, reinterpret_cast<uint16_t*>(ws + L.o), gates, inv,
+                       reinterpret_cast<float*>(ws + L.dg), st);
+  }
+  if (T > 0) {
+    StageTimer tm(c, st, 6);
+    rc = launch_grouped_gemm(c, GEMM_B2, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+  }
+  if (rc != MOE_OK) return rc;
+  {
+    StageTimer tm(c, st, 7);
+    rc = launch_grouped_gemm(c, GEMM_B3, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+  }
+  if (rc != MOE_OK) return rc;
+  if (T > 0) {
+    StageTimer tm(c, st, 8);
+    rc = launch_grouped_gemm(c, GEMM_B4, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+  }
+  if (rc != MOE_OK) return rc;
+  {
+    StageTimer tm(c, st, 9);
+    rc = launch_grouped_gemm(c, GEMM_B5, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+  }
+  if (rc != MOE_OK) return rc;
+  {
+    StageTimer tm(c, st, 10);
+    launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
+                      gates, reinterpret_cast<const float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts),
+                      d_aux, dl, st);
+  }
+  {
+    StageTimer tm(c, st, 11);
+    launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, st);
+  }
+  {
+    StageTimer tm(c, st, 12);
+    launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, st);
+  }
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------ host-buffer step
+struct E2ELayout {
+  size_t x, dy, y, dx, W_r, Wg, Wu, Wd, dWr, dWg, dWu, dWd, idx, gates, counts, aux, ws, total;
+};
+static E2ELayout e2e_layout(const Shape& s, int64_t T) {
+  E2ELayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t td = sizeof(uint16_t) * T * s.d, w = sizeof(uint16_t) * s.E * s.d * s.f;
+  L.x = take(td); L.dy = take(td); L.y = take(td); L.dx = take(td);
+  L.W_r = take(sizeof(uint16_t) * s.d * s.E);
+  L.Wg = take(w); L.Wu = take(w); L.Wd = take(w);
+  L.dWr = take(sizeof(float) * s.d * s.E);
+  L.dWg = take(w); L.dWu = take(w); L.dWd = take(w);
+  L.idx = take(sizeof(int32_t) * T * s.k);
+  L.gates = take(sizeof(float) * T * s.k);
+  L.counts = take(sizeof(int32_t) * s.E);
+  L.aux = take(256);
+  L.ws = take(make_layout(s, T).total);
+  L.total = off;
+  return L;
+}
+
+size_t moe_e2e_device_bytes(const moe_ctx* ctx, int64_t T) {
+  if (!ctx || T < 0) return 0;
+  return e2e_layout(reinterpret_cast<const moe_ctx_impl*>(ctx)->s, T).total;
+}
+
+moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16_t* x, const uint16_t* W_r,
+                         const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
+                         const uint16_t* dy, float d_aux, uint16_t* y, float* aux_loss, uint16_t* dx,
+                         float* dW_r, uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, void* dev,
+                         size_t dev_bytes, void* cuda_stream) {
+  if (!ctx || T < 0 || !dev || !x || !dy || !y || !dx || !aux_loss) return MOE_ERR_INVALID_ARG;
+  if (copy_weights && (!W_r || !W_gate || !W_up || !W_down || !dW_r || !dW_gate || !dW_up || !dW_down))
+    return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  const Shape& s = c->s;
+  const E2ELayout L = e2e_layout(s, T);
+  if (dev_bytes < L.total) return MOE_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* D = static_cast<char*>(dev);
+  const size_t td = sizeof(uint16_t) * T * s.d, w = sizeof(uint16_t) * s.E * s.d * s.f;
+  bool ok = true;
+  auto h2d = [&](size_t off, const void* src, size_t n) {
+    ok = ok && cudaMemcpyAsync(D + off, src, n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  };
+  auto d2h = [&](void* dst, size_t off, size_t n) {
+    ok = ok && cudaMemcpyAsync(dst, D + off, n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  };
+  h2d(L.x, x, td);
+  h2d(L.dy, dy, td);
+  if (copy_weights) {
+    h2d(L.W_r, W_r, sizeof(uint16_t) * s.d * s.E);
+    h2d(L.Wg, W_gate, w);
+    h2d(L.Wu, W_up, w);
+    h2d(L.Wd, W_down, w);
+  }
+  if (!ok) return MOE_ERR_CUDA;
+  const size_t wsb = make_layout(s, T).total;
+  auto U = [&](size_t off) { return reinterpret_cast<uint16_t*>(D + off); };
+  moe_status rc = moe_forward(ctx, T, U(L.x), U(L.W_r), nullptr, nullptr, U(L.Wg), U(L.Wu), U(L.Wd), U(L.y),
+                              reinterpret_cast<int32_t*>(D + L.idx), reinterpret_cast<float*>(D + L.gates),
+                              reinterpret_cast<int32_t*>(D + L.counts), nullptr, reinterpret_cast<float*>(D + L.aux),
+                              nullptr, D + L.ws, wsb, cuda_stream);
+  if (rc != MOE_OK) return rc;
+  rc = moe_backward(ctx, T, U(L.dy), d_aux, U(L.x), U(L.W_r), U(L.Wg), U(L.Wu), U(L.Wd), U(L.dx),
+                    reinterpret_cast<float*>(D + L.dWr), nullptr, U(L.dWg), U(L.dWu), U(L.dWd), D + L.ws, wsb,
+                    cuda_stream);
+  if (rc != MOE_OK) return rc;
+  d2h(y, L.y, td);
+  d2h(dx, L.dx, td);
+  d2h(aux_loss, L.aux, sizeof(float));
+  if (copy_weights) {
+    d2h(dW_r, L.dWr, sizeof(float) * s.d * s.E);
+    d2h(dW_gate, L.dWg, w);
+    d2h(dW_up, L.dWu, w);
+    d2h(dW_down, L.dWd, w);
+  }
+  if (!ok) return MOE_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
+  return moe_poll_status(ctx, D + L.ws, cuda_stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Shared declarations of the MoE layer library: workspace layout, launcher prototypes, small device helpers.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/moe.h"
+
+namespace moe {
+
+constexpr int ROW_PAD = 128;     // every expert's row segment starts and ends on a multiple of this
+constexpr int TOK_TILE = 256;    // tokens per block in the histogram / scatter kernels (8 warps x 32)
+constexpr int ROUTER_TOK = 16;   // tokens per block in the router kernel
+constexpr int MAX_E = 256;
+constexpr int MAX_K = 32;
+constexpr int DWR_SPLIT = 8;     // token slices of the dW_r contraction
+
+// status word values written by kernels
+constexpr int DEV_OK = 0;
+constexpr int DEV_TIMEOUT = 1;
+
+struct Shape {
+  int d, E, f, k;
+};
+
+// Byte offsets of every internal buffer inside the caller's workspace (all 256-byte aligned).
+struct WsLayout {
+  size_t status;       // int32[16]   [0] device status, [1] where it happened
+  size_t counts;       // int32[E]    rows per expert
+  size_t offsets;      // int32[E+1]  exclusive scan of counts (canonical, unpadded)
+  size_t pad_offsets;  // int32[E+1]  exclusive scan of counts rounded up to ROW_PAD
+  size_t sched;        // int32[4]    [0] number of 128-row tiles, [1] padded row total
+  size_t tile_expert;  // int32[max_m_tiles] expert of every 128-row tile
+  size_t tile_counts;  // int32[tok_tiles * E] per token-tile histogram, turned into a prefix along tiles
+  size_t psum_part;    // float[router_blocks * E] per-block column sums of p
+  size_t psum;         // float[E]
+  size_t logits;       // float[T*E]
+  size_t idx;          // int32[T*k]
+  size_t gates;        // float[T*k]
+  size_t inv;          // int32[T*k]  padded row of pair (t, j)
+  size_t row_token;    // int32[rows_max] token of a padded row, -1 for pad rows
+  size_t dg;           // float[T*k]
+  size_t dl;           // float[T*E]
+  size_t dwr_part;     // float[DWR_SPLIT * d * E]
+  size_t xp;           // bf16[rows_max * d]
+  size_t hg, hu, act;  // bf16[rows_max * f]
+  size_t o;            // bf16[rows_max * d]   o in forward, overwritten by d_o in backward
+  size_t dhg, dhu;     // bf16[rows_max * f]
+  size_t dxp;          // bf16[rows_max * d]
+  size_t total;
+  int64_t rows_max;    // upper bound of the padded row total for T tokens
+  int64_t max_m_tiles;
+  int64_t tok_tiles;
+  int64_t router_blocks;
+};
+
+WsLayout make_layout(const Shape& s, int64_t T);
+
+struct moe_ctx_impl {
+  Shape s;
+  int sm_count;
+  int device;
+  void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
+  int profiling;
+  cudaEvent_t ev[MOE_NUM_STAGES + 4][2];
+  int ev_used[MOE_NUM_STAGES + 4];
+  int ev_created;
+};
+
+// ---- launchers (route.cu)
+void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                   const float* logits_in, float* logits, int32_t* idx, float* gates, int32_t* idx_out,
+                   float* gates_out, float* logits_out, float* psum_part, cudaStream_t st);
+void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
+                    int32_t* perm_out, float* aux_out, cudaStream_t st);
+// ---- launchers (combine.cu)
+void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
+                    uint16_t* y, cudaStream_t st);
+void launch_combine_bwd(const Shape& s, int64_t T, const uint16_t* dy, uint16_t* o_to_do, const float* gates,
+                        const int32_t* inv, float* dg, cudaStream_t st);
+void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
+                       const float* dg, const int32_t* counts, float d_aux, float* dl, cudaStream_t st);
+void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
+                float* db_r, cudaStream_t st);
+void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const float* dl,
+                          const uint16_t* W_r, uint16_t* dx, cudaStream_t st);
+// ---- launchers (gemm.cu); each returns a CUDA / driver error as moe_status
+enum GemmKind { GEMM_F3 = 0, GEMM_F4, GEMM_B2, GEMM_B3, GEMM_B4, GEMM_B5 };
+moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
+                               const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
+                               uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, cudaStream_t st);
+
+// ---- device helpers
+__device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // .x = lo (low 16 bits), .y = hi
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi) {
+  lo = __uint_as_float(w << 16);
+  hi = __uint_as_float(w & 0xFFFF0000u);
+}
+
+}  // namespace moe

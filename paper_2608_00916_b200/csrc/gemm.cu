@@ -1,0 +1,536 @@
+// Grouped GEMMs of the MoE layer on tcgen05 tensor cores (sm_100a).
+//
+// One persistent, warp-specialised kernel template serves the six contractions of the layer:
+//   F3  [hg|hu] = xp  W_gate[e] | W_up[e]          + SwiGLU epilogue (writes hg, hu, act)
+//   F4  o       = act W_down[e]
+//   B2  da      = d_o W_down[e]^T                   + SwiGLU-backward epilogue (reads hg, hu; writes dhg, dhu)
+//   B4  dxp     = dhg W_gate[e]^T + dhu W_up[e]^T   (one accumulator, two K segments)
+//   B3  dW_down[e]          = act_e^T d_o_e         (K = rows of expert e, one CTA owns a whole output tile)
+//   B5  dW_gate[e]|dW_up[e] = xp_e^T [dhg_e|dhu_e]
+// Tiles are 128 x 256 with K steps of 64; operands arrive by TMA into 128-byte-swizzled shared memory (4 stages),
+// the accumulator lives in tensor memory (2 x 256 columns, so the epilogue of one tile overlaps the main loop
+// of the next).  Operand major-ness replaces every transpose: row-major [rows, K] is a K-major operand,
+// row-major [K, cols] is an MN-major operand, and the UMMA instruction takes either.
+// Row buffers are expert-major with each expert's segment padded to 128 rows of zeros, so an M tile never
+// straddles two experts and the ragged K of the weight gradients needs no masking.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer (owns the TMEM allocation), warps 2..5 epilogue.
+// Every mbarrier wait is bounded; on a timeout the kernel records it in the status word and leaves.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace moe {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;       // 16 KB
+constexpr int B_BYTES = BN * BK * 2;       // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-major tile: 8 KB
+constexpr int GEMM_THREADS = 192;
+constexpr int ACC_COLS = 256;
+constexpr int TMEM_COLS = 512;
+constexpr size_t GEMM_SMEM = static_cast<size_t>(STAGES) * STAGE_BYTES + 1024;
+
+struct GemmParams {
+  CUtensorMap mapA0, mapA1, mapB0, mapB1;
+  const int32_t* sched;        // [0] number of 128-row tiles
+  const int32_t* tile_expert;  // expert of each 128-row tile
+  const int32_t* pad_offsets;  // padded segment starts, E + 1 entries
+  int32_t* status;
+  int n_tiles;   // output tiles along N
+  int m_tiles;   // weight gradients: output tiles along M per expert
+  int E;
+  int k_blocks;  // row GEMMs: K blocks per segment
+  int M_total;   // weight gradients: rows of one expert's output
+  int N_total;   // columns of the output
+  uint16_t* out0;
+  uint16_t* out1;
+  uint16_t* out2;
+  const uint16_t* in0;
+  const uint16_t* in1;
+  int64_t ld_out;
+  int64_t expert_stride;
+};
+
+template <int KIND>
+struct Traits {
+  static constexpr bool WGRAD = (KIND == GEMM_B3 || KIND == GEMM_B5);
+  static constexpr int A_MN = WGRAD ? 1 : 0;
+  static constexpr int B_MN = (KIND == GEMM_B2 || KIND == GEMM_B4) ? 0 : 1;
+  static constexpr int NSEG = (KIND == GEMM_B4) ? 2 : 1;
+  // width of output covered by one N tile (F3 / B5 pair a 128-wide gate tile with the matching up tile)
+  static constexpr int N_SPAN = (KIND == GEMM_F3 || KIND == GEMM_B5) ? 128 : 256;
+};
+
+struct Tile {
+  int e, row0, m0, n0, nkb;
+};
+
+template <int KIND>
+__device__ __forceinline__ int total_tiles(const GemmParams& p) {
+  if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;
+  return p.sched[0] * p.n_tiles;
+}
+
+template <int KIND>
+__device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
+  Tile tl;
+  if (Traits<KIND>::WGRAD) {
+    const int per = p.m_tiles * p.n_tiles;
+    tl.e = t / per;
+    const int rem = t - tl.e * per;
+    tl.m0 = (rem / p.n_tiles) * BM;
+    tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.row0 = p.pad_offsets[tl.e];
+    tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
+  } else {
+    const int mt = t / p.n_tiles;
+    tl.e = p.tile_expert[mt];
+    tl.row0 = mt * BM;
+    tl.m0 = 0;
+    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
+  }
+  return tl;
+}
+
+template <int KIND>
+__device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl, int kb, uint32_t sA, uint32_t sB,
+                                            uint32_t bar) {
+  if (KIND == GEMM_F3) {
+    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+      tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
+    }
+  } else if (KIND == GEMM_F4) {
+    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+  } else if (KIND == GEMM_B2) {
+    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
+  } else if (KIND == GEMM_B4) {
+    const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
+    tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
+    tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
+  } else if (KIND == GEMM_B3) {
+    const int row = tl.row0 + kb * BK;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
+  } else {  // GEMM_B5
+    const int row = tl.row0 + kb * BK;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+      tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
+      tma_load_2d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, row);
+    }
+  }
+}
+
+__device__ __forceinline__ void store_bf16x32(uint16_t* dst, const float (&v)[32]) {
+  uint4* q = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint4 w;
+    w.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);
+    w.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
+    w.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
+    w.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
+    q[i] = w;
+  }
+}
+__device__ __forceinline__ void load_bf16x32(const uint16_t* src, float (&v)[32]) {
+  const uint4* q = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint4 w = q[i];
+    unpack_bf16x2(w.x, v[8 * i + 0], v[8 * i + 1]);
+    unpack_bf16x2(w.y, v[8 * i + 2], v[8 * i + 3]);
+    unpack_bf16x2(w.z, v[8 * i + 4], v[8 * i + 5]);
+    unpack_bf16x2(w.w, v[8 * i + 6], v[8 * i + 7]);
+  }
+}
+__device__ __forceinline__ float fast_sigmoid(float h) { return __fdividef(1.f, 1.f + __expf(-h)); }
+
+template <int KIND>
+__global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __grid_constant__ GemmParams p) {
+  using TR = Traits<KIND>;
+  extern __shared__ unsigned char gemm_smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ uint32_t tmem_base_slot;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = (smem_u32(gemm_smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 128);
+    }
+    fence_mbar_init();
+    tma_prefetch_desc(&p.mapA0);
+    tma_prefetch_desc(&p.mapB0);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const int ntiles = total_tiles<KIND>(p);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+      const Tile tl = get_tile<KIND>(p, t);
+      for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u)) {
+          ok = false;
+          break;
+        }
+        if (lane == 0) {
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t sA = smem_base + s * STAGE_BYTES;
+          issue_loads<KIND>(p, tl, kb, sA, sA + A_BYTES, full_bar(s));
+        }
+        __syncwarp();
+      }
+    }
+    if (!ok && lane == 0) {
+      atomicExch(p.status, DEV_TIMEOUT);
+      p.status[1] = 100 + KIND;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc = umma_idesc(BM, BN, TR::A_MN, TR::B_MN);
+    constexpr uint32_t A_LBO = TR::A_MN ? CHUNK_BYTES : 0, B_LBO = TR::B_MN ? CHUNK_BYTES : 0;
+    constexpr uint32_t A_KSTEP = TR::A_MN ? 2048 : 32, B_KSTEP = TR::B_MN ? 2048 : 32;  // bytes per K = 16
+    uint32_t it = 0, tc = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+      const Tile tl = get_tile<KIND>(p, t);
+      if (tl.nkb == 0) continue;
+      const int acc = tc & 1;
+      const uint32_t aph = (tc >> 1) & 1u;
+      ++tc;
+      if (!mbar_wait(tempty_bar(acc), aph ^ 1u)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
+      for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1u;
+        if (!mbar_wait(full_bar(s), ph)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t sA = smem_base + s * STAGE_BYTES;
+          const uint32_t sB = sA + A_BYTES;
+#pragma unroll
+          for (int ks = 0; ks < BK / 16; ++ks) {
+            const uint64_t da = smem_desc(sA + ks * A_KSTEP, A_LBO, 1024);
+            const uint64_t db = smem_desc(sB + ks * B_KSTEP, B_LBO, 1024);
+            umma_bf16(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar(s));
+        }
+        __syncwarp();
+      }
+      if (ok && lane == 0) umma_commit(tfull_bar(acc));
+      __syncwarp();
+    }
+    if (!ok && lane == 0) {
+      atomicExch(p.status, DEV_TIMEOUT);
+      p.status[1] = 200 + KIND;
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps, 128 TMEM lanes)
+    const int ew = warp & 3;  // TMEM lane quadrant this warp may read
+    uint32_t tc = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+      const Tile tl = get_tile<KIND>(p, t);
+      const int rin = ew * 32 + lane;  // row inside the tile
+      if (tl.nkb == 0) {
+        // weight gradient of an expert without tokens: zeros
+        if (TR::WGRAD) {
+          const int m = tl.m0 + rin;
+          if (m < p.M_total) {
+            float z[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) z[i] = 0.f;
+            for (int c = 0; c < 8; ++c) {
+              uint16_t* base = p.out0;
+              int col = tl.n0 + c * 32;
+              if (KIND == GEMM_B5) {
+                base = (c >= 4) ? p.out1 : p.out0;
+                col = tl.n0 + (c & 3) * 32;
+              }
+              if (col < p.N_total)
+                store_bf16x32(base + tl.e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, z);
+            }
+          }
+        }
+        continue;
+      }
+      const int acc = tc & 1;
+      const uint32_t aph = (tc >> 1) & 1u;
+      ++tc;
+      if (!mbar_wait(tfull_bar(acc), aph)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + acc * ACC_COLS;
+      const int64_t row = static_cast<int64_t>(tl.row0) + rin;
+      if (KIND == GEMM_F3) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t rg[32], ru[32];
+          tmem_ld32(taddr + c * 32, rg);
+          tmem_ld32(taddr + 128 + c * 32, ru);
+          tmem_ld_wait();
+          const int col = tl.n0 + c * 32;
+          if (col < p.N_total) {
+            float hg[32], hu[32], a[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              hg[i] = __uint_as_float(rg[i]);
+              hu[i] = __uint_as_float(ru[i]);
+              a[i] = hg[i] * fast_sigmoid(hg[i]) * hu[i];
+            }
+            const int64_t off = row * p.ld_out + col;
+            store_bf16x32(p.out0 + off, hg);
+            store_bf16x32(p.out1 + off, hu);
+            store_bf16x32(p.out2 + off, a);
+          }
+        }
+      } else if (KIND == GEMM_B2) {
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          uint32_t rd[32];
+          tmem_ld32(taddr + c * 32, rd);
+          tmem_ld_wait();
+          const int col = tl.n0 + c * 32;
+          if (col < p.N_total) {
+            const int64_t off = row * p.ld_out + col;
+            float hg[32], hu[32], dhg[32], dhu[32];
+            load_bf16x32(p.in0 + off, hg);
+            load_bf16x32(p.in1 + off, hu);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float da = __uint_as_float(rd[i]);
+              const float sg = fast_sigmoid(hg[i]);
+              dhg[i] = da * hu[i] * sg * (1.f + hg[i] * (1.f - sg));
+              dhu[i] = da * hg[i] * sg;
+            }
+            store_bf16x32(p.out0 + off, dhg);
+            store_bf16x32(p.out1 + off, dhu);
+          }
+        }
+      } else {
+        // plain bf16 store: F4, B4 (row GEMMs), B3, B5 (weight gradients)
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          uint32_t rd[32];
+          tmem_ld32(taddr + c * 32, rd);
+          tmem_ld_wait();
+          float v[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rd[i]);
+          if (TR::WGRAD) {
+            const int m = tl.m0 + rin;
+            uint16_t* base = p.out0;
+            int col = tl.n0 + c * 32;
+            if (KIND == GEMM_B5) {
+              base = (c >= 4) ? p.out1 : p.out0;
+              col = tl.n0 + (c & 3) * 32;
+            }
+            if (m < p.M_total && col < p.N_total)
+              store_bf16x32(base + tl.e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, v);
+          } else {
+            const int col = tl.n0 + c * 32;
+            if (col < p.N_total) store_bf16x32(p.out0 + row * p.ld_out + col, v);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(acc));
+    }
+    if (!ok && lane == 0) {
+      atomicExch(p.status, DEV_TIMEOUT);
+      p.status[1] = 300 + KIND;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 row-major [rows, width] -> 2D map with box {64, box_rows}
+static bool map_2d(void* fn, CUtensorMap* m, const void* base, int64_t rows, int64_t width, int box_rows) {
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(width), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(width) * 2};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t es[2] = {1, 1};
+  return reinterpret_cast<EncodeTiledFn>(fn)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                                             strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// bf16 [E, rows, width] -> 3D map with box {64, box_rows, 1}
+static bool map_3d(void* fn, CUtensorMap* m, const void* base, int64_t E, int64_t rows, int64_t width,
+                   int box_rows) {
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(width), static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(E)};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(width) * 2, static_cast<cuuint64_t>(width) * rows * 2};
+  cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return reinterpret_cast<EncodeTiledFn>(fn)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
+                                             strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int KIND>
+static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream_t st) {
+  static bool attr_done[8] = {false};
+  if (!attr_done[KIND]) {
+    if (cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(GEMM_SMEM)) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done[KIND] = true;
+  }
+  grouped_gemm_kernel<KIND><<<ctx->sm_count, GEMM_THREADS, GEMM_SMEM, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
+                               const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
+                               uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, cudaStream_t st) {
+  const Shape& s = ctx->s;
+  const int d = s.d, f = s.f, E = s.E;
+  const int64_t R = L.rows_max;
+  void* fn = ctx->encode_fn;
+  uint16_t* xp = reinterpret_cast<uint16_t*>(ws + L.xp);
+  uint16_t* hg = reinterpret_cast<uint16_t*>(ws + L.hg);
+  uint16_t* hu = reinterpret_cast<uint16_t*>(ws + L.hu);
+  uint16_t* act = reinterpret_cast<uint16_t*>(ws + L.act);
+  uint16_t* o = reinterpret_cast<uint16_t*>(ws + L.o);
+  uint16_t* dhg = reinterpret_cast<uint16_t*>(ws + L.dhg);
+  uint16_t* dhu = reinterpret_cast<uint16_t*>(ws + L.dhu);
+  uint16_t* dxp = reinterpret_cast<uint16_t*>(ws + L.dxp);
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.sched = reinterpret_cast<const int32_t*>(ws + L.sched);
+  p.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
+  p.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+  p.status = reinterpret_cast<int32_t*>(ws + L.status);
+  p.E = E;
+  bool ok = true;
+  switch (kind) {
+    case GEMM_F3:
+      ok = map_2d(fn, &p.mapA0, xp, R, d, 128) && map_3d(fn, &p.mapB0, W_gate, E, d, f, 64) &&
+           map_3d(fn, &p.mapB1, W_up, E, d, f, 64);
+      p.mapA1 = p.mapA0;
+      p.n_tiles = (f + 127) / 128;
+      p.k_blocks = d / BK;
+      p.N_total = f;
+      p.out0 = hg; p.out1 = hu; p.out2 = act;
+      p.ld_out = f;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_F3>(ctx, p, st);
+    case GEMM_F4:
+      ok = map_2d(fn, &p.mapA0, act, R, f, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.n_tiles = (d + 255) / 256;
+      p.k_blocks = f / BK;
+      p.N_total = d;
+      p.out0 = o;
+      p.ld_out = d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_F4>(ctx, p, st);
+    case GEMM_B2:
+      ok = map_2d(fn, &p.mapA0, o, R, d, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, 256);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.n_tiles = (f + 255) / 256;
+      p.k_blocks = d / BK;
+      p.N_total = f;
+      p.in0 = hg; p.in1 = hu;
+      p.out0 = dhg; p.out1 = dhu;
+      p.ld_out = f;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B2>(ctx, p, st);
+    case GEMM_B4:
+      ok = map_2d(fn, &p.mapA0, dhg, R, f, 128) && map_2d(fn, &p.mapA1, dhu, R, f, 128) &&
+           map_3d(fn, &p.mapB0, W_gate, E, d, f, 256) && map_3d(fn, &p.mapB1, W_up, E, d, f, 256);
+      p.n_tiles = (d + 255) / 256;
+      p.k_blocks = f / BK;
+      p.N_total = d;
+      p.out0 = dxp;
+      p.ld_out = d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B4>(ctx, p, st);
+    case GEMM_B3:
+      ok = map_2d(fn, &p.mapA0, act, R, f, 64) && map_2d(fn, &p.mapB0, o, R, d, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.m_tiles = (f + 127) / 128;
+      p.n_tiles = (d + 255) / 256;
+      p.M_total = f;
+      p.N_total = d;
+      p.out0 = dW_down;
+      p.ld_out = d;
+      p.expert_stride = static_cast<int64_t>(f) * d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B3>(ctx, p, st);
+    case GEMM_B5:
+      ok = map_2d(fn, &p.mapA0, xp, R, d, 64) && map_2d(fn, &p.mapB0, dhg, R, f, 64) &&
+           map_2d(fn, &p.mapB1, dhu, R, f, 64);
+      p.mapA1 = p.mapA0;
+      p.m_tiles = (d + 127) / 128;
+      p.n_tiles = (f + 127) / 128;
+      p.M_total = d;
+      p.N_total = f;
+      p.out0 = dW_gate; p.out1 = dW_up;
+      p.ld_out = f;
+      p.expert_stride = static_cast<int64_t>(d) * f;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B5>(ctx, p, st);
+  }
+  (void)T;
+  return MOE_ERR_INVALID_ARG;
+}
+
+}  // namespace moe

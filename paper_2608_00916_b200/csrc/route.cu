@@ -1,0 +1,357 @@
+// Router (fp32 logits, softmax, top-k with lowest-index tie-break, renormalised gates) and the
+// deterministic token permutation (per-tile histogram, prefix scan, stable scatter, row gather).
+#include "common.cuh"
+
+namespace moe {
+
+// ------------------------------------------------------------------------------------------ router
+// One block routes ROUTER_TOK tokens.  Contraction: thread = (expert, group of 8 tokens), x staged in shared
+// memory as fp32 (transposed so that the 8 tokens of a group are two float4), W_r read coalesced over
+// experts.  bf16 x bf16 products are exact in fp32, so the logits are fp32 sums of exact terms.
+// Then one warp per token: k rounds of (max value, lowest index) warp reduction on the logits, full
+// softmax for the auxiliary loss statistics, gates = softmax over the selected logits.
+constexpr int RT_CH = 256;  // columns of x staged per step
+
+__global__ void __launch_bounds__(256) router_kernel(int64_t T, int d, int E, int k, const uint16_t* __restrict__ x,
+                                                     const uint16_t* __restrict__ W_r, const float* __restrict__ b_r,
+                                                     const float* __restrict__ logits_in, float* __restrict__ logits,
+                                                     int32_t* __restrict__ idx, float* __restrict__ gates,
+                                                     int32_t* __restrict__ idx_out, float* __restrict__ gates_out,
+                                                     float* __restrict__ logits_out, float* __restrict__ psum_part) {
+  extern __shared__ __align__(16) unsigned char rt_smem[];
+  float* xs = reinterpret_cast<float*>(rt_smem);           // [RT_CH][ROUTER_TOK]
+  float* ls = xs + RT_CH * ROUTER_TOK;                     // [ROUTER_TOK][E]
+  float* pw = ls + ROUTER_TOK * E;                         // [8 warps][E]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * ROUTER_TOK;
+  constexpr int TG = ROUTER_TOK / 8;
+  const int items = E * TG;
+
+  if (logits_in != nullptr) {
+    for (int i = tid; i < ROUTER_TOK * E; i += 256) {
+      int tok = i / E, e = i % E;
+      int64_t t = t0 + tok;
+      ls[i] = (t < T) ? logits_in[t * E + e] : 0.f;
+    }
+  } else {
+    // each thread owns up to 2 items (E <= 256, TG = 2 -> at most 512 items)
+    float acc[2][8];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[a][i] = 0.f;
+    for (int c0 = 0; c0 < d; c0 += RT_CH) {
+      __syncthreads();
+      for (int i = tid; i < ROUTER_TOK * RT_CH / 2; i += 256) {
+        int tok = i / (RT_CH / 2), cp = i % (RT_CH / 2);
+        int64_t t = t0 + tok;
+        int c = c0 + 2 * cp;
+        float lo = 0.f, hi = 0.f;
+        if (t < T && c < d) {
+          uint32_t w = *reinterpret_cast<const uint32_t*>(x + t * d + c);
+          unpack_bf16x2(w, lo, hi);
+        }
+        xs[(2 * cp) * ROUTER_TOK + tok] = lo;
+        xs[(2 * cp + 1) * ROUTER_TOK + tok] = hi;
+      }
+      __syncthreads();
+      const int cmax = min(RT_CH, d - c0);
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        int item = tid + a * 256;
+        if (item < items) {
+          int tg = item / E, e = item % E;
+          const uint16_t* wp = W_r + static_cast<int64_t>(c0) * E + e;
+#pragma unroll 4
+          for (int c = 0; c < cmax; ++c) {
+            float w = bf16_to_f32(wp[static_cast<int64_t>(c) * E]);
+            const float4 xa = *reinterpret_cast<const float4*>(xs + c * ROUTER_TOK + tg * 8);
+            const float4 xb = *reinterpret_cast<const float4*>(xs + c * ROUTER_TOK + tg * 8 + 4);
+            acc[a][0] = fmaf(xa.x, w, acc[a][0]);
+            acc[a][1] = fmaf(xa.y, w, acc[a][1]);
+            acc[a][2] = fmaf(xa.z, w, acc[a][2]);
+            acc[a][3] = fmaf(xa.w, w, acc[a][3]);
+            acc[a][4] = fmaf(xb.x, w, acc[a][4]);
+            acc[a][5] = fmaf(xb.y, w, acc[a][5]);
+            acc[a][6] = fmaf(xb.z, w, acc[a][6]);
+            acc[a][7] = fmaf(xb.w, w, acc[a][7]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      int item = tid + a * 256;
+      if (item < items) {
+        int tg = item / E, e = item % E;
+        float b = b_r ? b_r[e] : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ls[(tg * 8 + i) * E + e] = acc[a][i] + b;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- per token: selection, softmax, gates (one warp per token)
+  const int NQ = (E + 31) / 32;
+  float psum_acc[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) psum_acc[q] = 0.f;
+  for (int tok = warp; tok < ROUTER_TOK; tok += 8) {
+    const int64_t t = t0 + tok;
+    if (t >= T) break;  // warp-uniform
+    float v[8];
+    uint32_t taken = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      int e = lane + 32 * q;
+      if (q < NQ && e < E) {
+        v[q] = ls[tok * E + e];
+        logits[t * E + e] = v[q];
+        if (logits_out) logits_out[t * E + e] = v[q];
+      } else {
+        v[q] = -INFINITY;
+        taken |= 1u << q;
+      }
+    }
+    int my_e = 0;
+    float my_v = 0.f, vmax = 0.f;
+    for (int j = 0; j < k; ++j) {
+      float bv = -INFINITY;
+      int bi = 0x7FFFFFFF;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (!((taken >> q) & 1u) && (bi == 0x7FFFFFFF || v[q] > bv)) {
+          bv = v[q];
+          bi = lane + 32 * q;
+        }
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off);
+        int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
+        bool better = (oi != 0x7FFFFFFF) && (bi == 0x7FFFFFFF || ov > bv || (ov == bv && oi < bi));
+        if (better) {
+          bv = ov;
+          bi = oi;
+        }
+      }
+      if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+      if (lane == j) {
+        my_e = bi;
+        my_v = bv;
+      }
+      if (j == 0) vmax = bv;
+    }
+    // full softmax (statistics for the auxiliary loss)
+    float z = 0.f, pe[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      int e = lane + 32 * q;
+      pe[q] = (q < NQ && e < E) ? expf(v[q] - vmax) : 0.f;
+      z += pe[q];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
+    const float rz = 1.f / z;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) psum_acc[q] += pe[q] * rz;
+    // gates over the selection
+    float ge = (lane < k) ? expf(my_v - vmax) : 0.f;
+    float zs = ge;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) zs += __shfl_xor_sync(0xFFFFFFFFu, zs, off);
+    if (lane < k) {
+      float g = ge / zs;
+      idx[t * k + lane] = my_e;
+      gates[t * k + lane] = g;
+      idx_out[t * k + lane] = my_e;
+      gates_out[t * k + lane] = g;
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    int e = lane + 32 * q;
+    if (q < NQ && e < E) pw[warp * E + e] = psum_acc[q];
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += 256) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += pw[w * E + e];
+    psum_part[static_cast<int64_t>(blockIdx.x) * E + e] = s;
+  }
+}
+
+void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                   const float* logits_in, float* logits, int32_t* idx, float* gates, int32_t* idx_out,
+                   float* gates_out, float* logits_out, float* psum_part, cudaStream_t st) {
+  if (T == 0) return;
+  const int blocks = static_cast<int>((T + ROUTER_TOK - 1) / ROUTER_TOK);
+  const size_t smem = sizeof(float) * (RT_CH * ROUTER_TOK + ROUTER_TOK * s.E + 8 * s.E);
+  router_kernel<<<blocks, 256, smem, st>>>(T, s.d, s.E, s.k, x, W_r, b_r, logits_in, logits, idx, gates, idx_out,
+                                           gates_out, logits_out, psum_part);
+}
+
+// ------------------------------------------------------------------------------------------ permutation
+// Stable counting sort of the (token, slot) pairs by expert.  A token takes an expert at most once, so
+// the order inside an expert is the token order.  Each warp covers 32 consecutive tokens and records, per
+// expert, the 32-bit mask of its tokens that chose it (atomicOr: order-free, hence deterministic); ranks
+// are population counts of mask prefixes.  Tiles of TOK_TILE tokens are combined by a column scan.
+__device__ __forceinline__ void build_masks(uint32_t* masks /* [8][E] */, const int32_t* __restrict__ idx, int64_t T,
+                                            int E, int k, int64_t tile_t0) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int i = tid; i < 8 * E; i += TOK_TILE) masks[i] = 0u;
+  __syncthreads();
+  const int64_t t = tile_t0 + tid;
+  if (t < T) {
+    for (int j = 0; j < k; ++j) {
+      int e = idx[t * k + j];
+      atomicOr(&masks[warp * E + e], 1u << lane);
+    }
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(TOK_TILE) hist_kernel(int64_t T, int E, int k, const int32_t* __restrict__ idx,
+                                                        int32_t* __restrict__ tile_counts) {
+  extern __shared__ uint32_t hist_masks[];
+  build_masks(hist_masks, idx, T, E, k, static_cast<int64_t>(blockIdx.x) * TOK_TILE);
+  for (int e = threadIdx.x; e < E; e += TOK_TILE) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) c += __popc(hist_masks[w * E + e]);
+    tile_counts[static_cast<int64_t>(blockIdx.x) * E + e] = c;
+  }
+}
+
+// One block: column scan of tile_counts (in place -> exclusive prefix along tiles), counts, canonical and
+// padded offsets, tile -> expert table, and the auxiliary loss from the per-block column sums of p.
+__global__ void __launch_bounds__(256) scan_kernel(int64_t T, int E, int k, int tok_tiles, int router_blocks,
+                                                   int32_t* __restrict__ tile_counts, int32_t* __restrict__ counts,
+                                                   int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
+                                                   int32_t* __restrict__ sched, int32_t* __restrict__ tile_expert,
+                                                   const float* __restrict__ psum_part, float* __restrict__ psum,
+                                                   int32_t* __restrict__ counts_out, float* __restrict__ aux_out,
+                                                   int32_t* __restrict__ status) {
+  __shared__ int s_cnt[MAX_E];
+  __shared__ int s_pad[MAX_E + 1];
+  __shared__ float s_term[MAX_E];
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    status[0] = DEV_OK;
+    status[1] = 0;
+  }
+  for (int e = tid; e < E; e += 256) {
+    int run = 0;
+    for (int tl = 0; tl < tok_tiles; ++tl) {
+      int c = tile_counts[static_cast<int64_t>(tl) * E + e];
+      tile_counts[static_cast<int64_t>(tl) * E + e] = run;
+      run += c;
+    }
+    s_cnt[e] = run;
+    counts[e] = run;
+    counts_out[e] = run;
+    float ps = 0.f;
+    for (int b = 0; b < router_blocks; ++b) ps += psum_part[static_cast<int64_t>(b) * E + e];
+    psum[e] = ps;
+    // aux term: (c_e / (T k)) * (Psum_e / T)
+    s_term[e] = (T > 0) ? (static_cast<float>(run) / static_cast<float>(T * k)) * (ps / static_cast<float>(T)) : 0.f;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int off = 0, poff = 0;
+    float aux = 0.f;
+    for (int e = 0; e < E; ++e) {
+      offsets[e] = off;
+      pad_offsets[e] = poff;
+      s_pad[e] = poff;
+      off += s_cnt[e];
+      poff += (s_cnt[e] + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
+      aux += s_term[e];
+    }
+    offsets[E] = off;
+    pad_offsets[E] = poff;
+    s_pad[E] = poff;
+    sched[0] = poff / ROW_PAD;
+    sched[1] = poff;
+    aux_out[0] = aux * static_cast<float>(E);
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += 256) {
+    for (int m = s_pad[e] / ROW_PAD; m < s_pad[e + 1] / ROW_PAD; ++m) tile_expert[m] = e;
+  }
+}
+
+__global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int k, const int32_t* __restrict__ idx,
+                                                           const int32_t* __restrict__ tile_base,
+                                                           const int32_t* __restrict__ offsets,
+                                                           const int32_t* __restrict__ pad_offsets,
+                                                           int32_t* __restrict__ inv, int32_t* __restrict__ row_token,
+                                                           int32_t* __restrict__ perm_out) {
+  extern __shared__ uint32_t sc_masks[];
+  const int64_t tile_t0 = static_cast<int64_t>(blockIdx.x) * TOK_TILE;
+  build_masks(sc_masks, idx, T, E, k, tile_t0);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t t = tile_t0 + tid;
+  if (t >= T) return;
+  for (int j = 0; j < k; ++j) {
+    const int e = idx[t * k + j];
+    int rank = tile_base[static_cast<int64_t>(blockIdx.x) * E + e];
+    for (int w = 0; w < warp; ++w) rank += __popc(sc_masks[w * E + e]);
+    rank += __popc(sc_masks[warp * E + e] & ((1u << lane) - 1u));
+    const int r = pad_offsets[e] + rank;
+    inv[t * k + j] = r;
+    row_token[r] = static_cast<int32_t>(t);
+    if (perm_out) perm_out[offsets[e] + rank] = static_cast<int32_t>(t * k + j);
+  }
+}
+
+// xp[r,:] = x[row_token[r],:], zero for pad rows.  One warp per row, 16-byte accesses.
+__global__ void __launch_bounds__(256) gather_rows_kernel(int d, const uint16_t* __restrict__ x,
+                                                          const int32_t* __restrict__ row_token,
+                                                          const int32_t* __restrict__ sched,
+                                                          uint16_t* __restrict__ xp) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (r >= sched[1]) return;
+  const int t = row_token[r];
+  uint4* dst = reinterpret_cast<uint4*>(xp + r * d);
+  const int n16 = d / 8;
+  if (t < 0) {
+    for (int i = lane; i < n16; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
+  } else {
+    const uint4* src = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(t) * d);
+    for (int i = lane; i < n16; i += 32) dst[i] = __ldg(src + i);
+  }
+}
+
+void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
+                    int32_t* perm_out, float* aux_out, cudaStream_t st) {
+  int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
+  int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
+  int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
+  const int tiles = static_cast<int>(L.tok_tiles);
+  const size_t msm = sizeof(uint32_t) * 8 * s.E;
+  cudaMemsetAsync(row_token, 0xFF, sizeof(int32_t) * L.rows_max, st);
+  if (tiles > 0) hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
+  scan_kernel<<<1, 256, 0, st>>>(T, s.E, s.k, tiles, static_cast<int>(L.router_blocks), tile_counts,
+                                 reinterpret_cast<int32_t*>(ws + L.counts), reinterpret_cast<int32_t*>(ws + L.offsets),
+                                 reinterpret_cast<int32_t*>(ws + L.pad_offsets),
+                                 reinterpret_cast<int32_t*>(ws + L.sched),
+                                 reinterpret_cast<int32_t*>(ws + L.tile_expert),
+                                 reinterpret_cast<const float*>(ws + L.psum_part),
+                                 reinterpret_cast<float*>(ws + L.psum), counts_out, aux_out,
+                                 reinterpret_cast<int32_t*>(ws + L.status));
+  if (tiles > 0) {
+    scatter_kernel<<<tiles, TOK_TILE, msm, st>>>(
+        T, s.E, s.k, idx, tile_counts, reinterpret_cast<const int32_t*>(ws + L.offsets),
+        reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<int32_t*>(ws + L.inv), row_token,
+        perm_out);
+    const int gblocks = static_cast<int>((L.rows_max + 7) / 8);
+    gather_rows_kernel<<<gblocks, 256, 0, st>>>(s.d, x, row_token, reinterpret_cast<const int32_t*>(ws + L.sched),
+                                                reinterpret_cast<uint16_t*>(ws + L.xp));
+  }
+}
+
+}  // namespace moe
