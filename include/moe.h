@@ -90,13 +90,16 @@ MOE_API const char* moe_status_string(moe_status s);
 MOE_API moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_stream);
 
 /* Per-stage timing.  With enable != 0, moe_forward / moe_backward record CUDA events between their
- * kernels on the caller's stream.  moe_stage_times synchronises on those events and adds, for each stage,
- * the milliseconds of the last forward+backward pair to ms[0..MOE_NUM_STAGES) (host array).
+ * kernels on the caller's stream, one event set per forward+backward pair, in a ring of MOE_PROF_RING sets.
+ * moe_stage_times waits for the recorded events, ADDS to ms[s] (host array of MOE_NUM_STAGES floats) the
+ * milliseconds stage s took summed over the pairs recorded since the previous call (the last MOE_PROF_RING
+ * of them if there were more), stores that number of pairs in *steps, and starts a new window.
  * Stage order: 0 router, 1 permute (histogram, scan, scatter, gather), 2 gate/up GEMM + SwiGLU,
  * 3 down GEMM, 4 combine, 5 combine-bwd, 6 dgrad-down + SwiGLU-bwd, 7 wgrad-down, 8 dgrad gate/up,
  * 9 wgrad gate/up, 10 router-bwd (dl), 11 dW_r, 12 unpermute-bwd (dx), 13..15 unused. */
+#define MOE_PROF_RING 64
 MOE_API moe_status moe_set_profiling(moe_ctx* ctx, int enable);
-MOE_API moe_status moe_stage_times(moe_ctx* ctx, float* ms /* host, MOE_NUM_STAGES floats */);
+MOE_API moe_status moe_stage_times(moe_ctx* ctx, float* ms /* host */, int32_t* steps /* host */);
 
 /* Forward pass over T tokens (T >= 0).
  *   x          [T,d]   bf16

@@ -51,7 +51,7 @@ def load_library() -> C.CDLL:
     lib.moe_poll_status.restype = C.c_int
     lib.moe_set_profiling.argtypes = [vp, C.c_int]
     lib.moe_set_profiling.restype = C.c_int
-    lib.moe_stage_times.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.moe_stage_times.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.moe_stage_times.restype = C.c_int
     lib.moe_forward.argtypes = [vp, i64] + [vp] * 14 + [vp, sz, vp]
     lib.moe_forward.restype = C.c_int
@@ -189,10 +189,12 @@ class MoELayer:
         _check(self.lib, self.lib.moe_set_profiling(self.h, 1 if on else 0), "moe_set_profiling")
 
     def stage_times(self, acc=None):
-        """Adds the per-stage milliseconds of the last forward+backward to `acc` (list of NUM_STAGES floats)."""
+        """Adds to `acc` the per-stage milliseconds summed over the forward+backward pairs recorded since the last
+        call; returns (list of NUM_STAGES floats, number of pairs)."""
         arr = (C.c_float * NUM_STAGES)(*(acc or [0.0] * NUM_STAGES))
-        _check(self.lib, self.lib.moe_stage_times(self.h, arr), "moe_stage_times")
-        return list(arr)
+        n = C.c_int32(0)
+        _check(self.lib, self.lib.moe_stage_times(self.h, arr, C.byref(n)), "moe_stage_times")
+        return list(arr), n.value
 
     # ---- host-buffer step (end-to-end timing)
     def e2e_device_bytes(self, T: int) -> int:

@@ -78,14 +78,12 @@ struct StageTimer {
   cudaStream_t st;
   int stage;
   StageTimer(moe_ctx_impl* c_, cudaStream_t st_, int stage_) : c(c_), st(st_), stage(stage_) {
-    if (c->profiling) {
-      cudaEventRecord(c->ev[stage][0], st);
-    }
+    if (c->profiling) cudaEventRecord(c->ev[c->prof_step % MOE_PROF_RING][stage][0], st);
   }
   ~StageTimer() {
     if (c->profiling) {
-      cudaEventRecord(c->ev[stage][1], st);
-      c->ev_used[stage] = 1;
+      cudaEventRecord(c->ev[c->prof_step % MOE_PROF_RING][stage][1], st);
+      c->ev_used[c->prof_step % MOE_PROF_RING][stage] = 1;
     }
   }
 };
@@ -114,10 +112,11 @@ void moe_destroy(moe_ctx* ctx) {
   if (!ctx) return;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   if (c->ev_created)
-    for (int i = 0; i < MOE_NUM_STAGES; ++i) {
-      cudaEventDestroy(c->ev[i][0]);
-      cudaEventDestroy(c->ev[i][1]);
-    }
+    for (int r = 0; r < MOE_PROF_RING; ++r)
+      for (int i = 0; i < MOE_NUM_STAGES; ++i) {
+        cudaEventDestroy(c->ev[r][i][0]);
+        cudaEventDestroy(c->ev[r][i][1]);
+      }
   delete c;
 }
 
@@ -194,25 +193,36 @@ moe_status moe_set_profiling(moe_ctx* ctx, int enable) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   if (enable && !c->ev_created) {
-    for (int i = 0; i < MOE_NUM_STAGES; ++i)
-      if (cudaEventCreate(&c->ev[i][0]) != cudaSuccess || cudaEventCreate(&c->ev[i][1]) != cudaSuccess)
-        return MOE_ERR_CUDA;
+    for (int r = 0; r < MOE_PROF_RING; ++r)
+      for (int i = 0; i < MOE_NUM_STAGES; ++i)
+        if (cudaEventCreate(&c->ev[r][i][0]) != cudaSuccess || cudaEventCreate(&c->ev[r][i][1]) != cudaSuccess)
+          return MOE_ERR_CUDA;
     c->ev_created = 1;
   }
   c->profiling = enable ? 1 : 0;
+  c->prof_read = c->prof_step;
+  memset(c->ev_used, 0, sizeof(c->ev_used));
   return MOE_OK;
 }
 
-moe_status moe_stage_times(moe_ctx* ctx, float* ms) {
-  if (!ctx || !ms) return MOE_ERR_INVALID_ARG;
+moe_status moe_stage_times(moe_ctx* ctx, float* ms, int32_t* steps) {
+  if (!ctx || !ms || !steps) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
-  for (int i = 0; i < MOE_NUM_STAGES; ++i) {
-    if (!c->ev_used[i]) continue;
-    if (cudaEventSynchronize(c->ev[i][1]) != cudaSuccess) return MOE_ERR_CUDA;
-    float t = 0.f;
-    if (cudaEventElapsedTime(&t, c->ev[i][0], c->ev[i][1]) != cudaSuccess) return MOE_ERR_CUDA;
-    ms[i] += t;
+  int64_t first = c->prof_read;
+  if (c->prof_step - first > MOE_PROF_RING) first = c->prof_step - MOE_PROF_RING;
+  *steps = static_cast<int32_t>(c->prof_step - first);
+  for (int64_t sidx = first; sidx < c->prof_step; ++sidx) {
+    const int r = static_cast<int>(sidx % MOE_PROF_RING);
+    for (int i = 0; i < MOE_NUM_STAGES; ++i) {
+      if (!c->ev_used[r][i]) continue;
+      c->ev_used[r][i] = 0;
+      if (cudaEventSynchronize(c->ev[r][i][1]) != cudaSuccess) return MOE_ERR_CUDA;
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, c->ev[r][i][0], c->ev[r][i][1]) != cudaSuccess) return MOE_ERR_CUDA;
+      ms[i] += t;
+    }
   }
+  c->prof_read = c->prof_step;
   return MOE_OK;
 }
 
@@ -329,6 +339,7 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
     StageTimer tm(c, st, 12);
     launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, st);
   }
+  if (c->profiling) c->prof_step++;
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

@@ -72,27 +72,35 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(int d, int k, const ui
     unpack_bf16x2(dv.y, dyv[2], dyv[3]);
     unpack_bf16x2(dv.z, dyv[4], dyv[5]);
     unpack_bf16x2(dv.w, dyv[6], dyv[7]);
+    // groups of 8 slots: all row loads of a group are issued before the first store, so they overlap
 #pragma unroll
-    for (int j = 0; j < MAX_K; ++j) {
-      if (j < k) {
-        uint4* po = reinterpret_cast<uint4*>(o + static_cast<int64_t>(sr[j]) * d + c);
-        const uint4 v = *po;
-        float ov[8];
-        unpack_bf16x2(v.x, ov[0], ov[1]);
-        unpack_bf16x2(v.y, ov[2], ov[3]);
-        unpack_bf16x2(v.z, ov[4], ov[5]);
-        unpack_bf16x2(v.w, ov[6], ov[7]);
-        float s = 0.f;
+    for (int j0 = 0; j0 < MAX_K; j0 += 8) {
+      if (j0 < k) {
+        uint4 v[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) s = fmaf(dyv[i], ov[i], s);
-        dot[j] += s;
-        const float g = sg[j];
-        uint4 w;
-        w.x = pack_bf16x2(g * dyv[0], g * dyv[1]);
-        w.y = pack_bf16x2(g * dyv[2], g * dyv[3]);
-        w.z = pack_bf16x2(g * dyv[4], g * dyv[5]);
-        w.w = pack_bf16x2(g * dyv[6], g * dyv[7]);
-        *po = w;
+        for (int jj = 0; jj < 8; ++jj)
+          if (j0 + jj < k) v[jj] = *reinterpret_cast<const uint4*>(o + static_cast<int64_t>(sr[j0 + jj]) * d + c);
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          if (j0 + jj < k) {
+            float ov[8];
+            unpack_bf16x2(v[jj].x, ov[0], ov[1]);
+            unpack_bf16x2(v[jj].y, ov[2], ov[3]);
+            unpack_bf16x2(v[jj].z, ov[4], ov[5]);
+            unpack_bf16x2(v[jj].w, ov[6], ov[7]);
+            float s = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) s = fmaf(dyv[i], ov[i], s);
+            dot[j0 + jj] += s;
+            const float g = sg[j0 + jj];
+            uint4 w;
+            w.x = pack_bf16x2(g * dyv[0], g * dyv[1]);
+            w.y = pack_bf16x2(g * dyv[2], g * dyv[3]);
+            w.z = pack_bf16x2(g * dyv[4], g * dyv[5]);
+            w.w = pack_bf16x2(g * dyv[6], g * dyv[7]);
+            *reinterpret_cast<uint4*>(o + static_cast<int64_t>(sr[j0 + jj]) * d + c) = w;
+          }
+        }
       }
     }
   }

@@ -64,9 +64,11 @@ struct moe_ctx_impl {
   int device;
   void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
   int profiling;
-  cudaEvent_t ev[MOE_NUM_STAGES + 4][2];
-  int ev_used[MOE_NUM_STAGES + 4];
+  cudaEvent_t ev[MOE_PROF_RING][MOE_NUM_STAGES][2];
+  unsigned char ev_used[MOE_PROF_RING][MOE_NUM_STAGES];
   int ev_created;
+  int64_t prof_step;   // forward+backward pairs recorded so far
+  int64_t prof_read;   // pairs already reported by moe_stage_times
 };
 
 // ---- launchers (route.cu)

@@ -1,0 +1,83 @@
+"""The C-ABI library loads and exports every symbol include/moe.h declares; host-side argument checks and the
+workspace arithmetic run without a GPU (no kernel is launched here)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2608_00916_b200 import binding
+from paper_2608_00916_b200 import build as pbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    pbuild.build()
+    return binding.load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "moe.h")).read()
+    return re.findall(r"MOE_API\s+[\w\s\*]+?\b(moe_\w+)\s*\(", text)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(names) == sorted(binding.EXPORTS)
+
+
+def test_create_validates_arguments(lib):
+    h = C.c_void_p()
+    for bad in [(100, 8, 128, 2), (128, 0, 128, 1), (128, 300, 128, 2), (128, 8, 128, 9), (128, 8, 100, 2),
+                (128, 64, 128, 33)]:
+        cfg = binding.MoEConfig(*bad, 0)
+        assert lib.moe_create(C.byref(cfg), C.byref(h)) == -1, bad
+    cfg = binding.MoEConfig(2048, 128, 768, 8, 0)
+    assert lib.moe_create(C.byref(cfg), C.byref(h)) == 0
+    lib.moe_destroy(h)
+    assert lib.moe_status_string(0) == b"ok" and b"workspace" in lib.moe_status_string(-3)
+
+
+def test_workspace_arithmetic(lib):
+    layer = binding.MoELayer(2048, 128, 768, 8)
+    sizes = [layer.workspace_bytes(T) for T in (0, 1, 1000, 16384, 65536)]
+    assert all(a < b for a, b in zip(sizes, sizes[1:]))
+    assert lib.moe_workspace_bytes(None, 5) == 0 and layer.workspace_bytes(-1) == 0
+    T = 16384
+    rows_max = ((T * 8 + 127) // 128 + 128) * 128
+    off, n = layer.find(T, "xp")
+    assert n == rows_max * 2048 * 2 and off % 256 == 0
+    off2, n2 = layer.find(T, "act")
+    assert n2 == rows_max * 768 * 2 and off2 >= off + n
+    assert layer.workspace_bytes(T) < 3 * 2**30  # saved activations of the Qwen shape fit in a few GB
+    with pytest.raises(binding.MoEError):
+        layer.find(T, "nonsense")
+    # regions do not overlap
+    spans = sorted(layer.find(T, nm) for nm in ("counts", "offsets", "pad_offsets", "logits", "idx", "gates", "inv",
+                                                 "row_token", "xp", "hg", "hu", "act", "o", "dhg", "dhu", "dxp", "dg",
+                                                 "dl"))
+    for (o1, n1), (o2, _) in zip(spans, spans[1:]):
+        assert o1 + n1 <= o2
+
+
+def test_forward_rejects_bad_arguments_before_launch(lib):
+    layer = binding.MoELayer(128, 8, 128, 2)
+    vp = C.c_void_p
+    fake = vp(4096)  # aligned non-null pointer; never dereferenced because the checks fail first
+    # T < 0
+    args = [layer.h, -1] + [fake] * 14 + [fake, 1 << 30, None]
+    assert lib.moe_forward(*args) == -1
+    # workspace too small
+    args = [layer.h, 64] + [fake] * 14 + [fake, 16, None]
+    assert lib.moe_forward(*args) == -3
+    # misaligned x
+    args = [layer.h, 64, vp(4098)] + [fake] * 13 + [fake, 1 << 30, None]
+    assert lib.moe_forward(*args) == -1
+    # missing weights
+    args = [layer.h, 64, fake, fake, None, None, None, fake, fake] + [fake] * 7 + [fake, 1 << 30, None]
+    assert lib.moe_forward(*args) == -1

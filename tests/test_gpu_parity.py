@@ -1,0 +1,215 @@
+"""Parity of the CUDA layer (called through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bars: routing indices, per-expert counts and the permutation are bit-exact; gates |d| <= 1e-5; logits
+|d| <= 1e-5 max|l|; aux relative <= 1e-4; relative Frobenius error <= 1e-2 for y and every gradient (bf16
+storage of the intermediates puts the expected error near 3e-3); weight-gradient slabs of experts that received
+tokens <= 2e-2 each, and exactly zero for experts without tokens."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_00916_b200 import synth
+from gpu_util import Run, from_dev_bf16, oracle_run, rel_fro
+from oracle import moe_oracle as orc
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def check_routing(fw, ofw):
+    assert np.array_equal(fw["idx"].cpu().numpy(), ofw["idx"])
+    assert np.array_equal(fw["counts"].cpu().numpy(), ofw["counts"])
+    assert np.array_equal(fw["perm"].cpu().numpy(), ofw["perm"])
+    assert np.abs(fw["gates"].cpu().numpy() - ofw["gates"]).max() <= 1e-5
+    lg = fw["logits"].cpu().numpy()
+    assert np.abs(lg - ofw["logits"]).max() <= 1e-5 * max(1.0, np.abs(ofw["logits"]).max())
+    assert float(fw["aux"].cpu()[0]) == pytest.approx(ofw["aux"], rel=1e-4)
+
+
+def check_all(r: Run, ofw, obw, d_aux, stages=True):
+    fw = r.forward()
+    check_routing(fw, ofw)
+    d, f, k, E = r.d, r.f, r.k, r.E
+    if stages:
+        for nm, w in (("xp", d), ("hg", f), ("hu", f), ("act", f), ("o", d)):
+            got, pad = r.rows(nm, w)
+            assert rel_fro(got, ofw[nm]) <= (0.0 if nm == "xp" else TOL), nm
+            assert not pad.any(), f"pad rows of {nm} are not zero"
+    assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+    bw = r.backward(d_aux)
+    if stages:
+        assert rel_fro(r.layer.buffer("dg", torch.float32).cpu().numpy().reshape(-1, k), obw["dg"]) <= TOL
+        for nm, w, on in (("o", d, "d_o"), ("dhg", f, "dhg"), ("dhu", f, "dhu"), ("dxp", d, "dxp")):
+            got, pad = r.rows(nm, w)
+            assert rel_fro(got, obw[on]) <= TOL, on
+            assert not pad.any(), f"pad rows of {on} are not zero"
+        assert rel_fro(r.layer.buffer("dl", torch.float32).cpu().numpy().reshape(-1, E), obw["dl"]) <= TOL
+    for nm in ("dx", "dW_gate", "dW_up", "dW_down"):
+        assert rel_fro(from_dev_bf16(bw[nm]), obw[nm]) <= TOL, nm
+    assert rel_fro(bw["dW_r"].cpu().numpy(), obw["dW_r"]) <= TOL
+    assert rel_fro(bw["db_r"].cpu().numpy(), obw["db_r"]) <= TOL
+    # per-expert slabs
+    for nm in ("dW_gate", "dW_up", "dW_down"):
+        g = from_dev_bf16(bw[nm])
+        for e in range(E):
+            if ofw["counts"][e] == 0:
+                assert not g[e].any(), (nm, e)
+            else:
+                assert rel_fro(g[e], obw[nm][e]) <= 2e-2, (nm, e)
+    return fw, bw
+
+
+def test_tiny_config_stage_by_stage():
+    inp = synth.make_config("tiny")
+    ofw, obw = oracle_run(inp, 2, inp["d_aux"])
+    check_all(Run(inp, 2), ofw, obw, inp["d_aux"])
+
+
+@pytest.mark.parametrize("T,d,E,k,f,seed", [
+    (1, 64, 4, 2, 64, 11),        # a single token
+    (7, 128, 8, 3, 192, 12),      # fewer tokens than experts*k: several empty experts
+    (255, 256, 8, 2, 320, 13),    # one short of a token tile; f not a multiple of 128 or 256
+    (1000, 512, 16, 4, 384, 14),  # several row tiles per expert, ragged tails
+    (333, 192, 5, 5, 320, 15),    # k = E: every expert takes every token; d not a multiple of 128
+    (300, 128, 1, 1, 256, 16),    # E = 1, k = 1: dense SwiGLU MLP
+    (2049, 256, 32, 8, 128, 17),  # more than 8 token tiles, k = 8
+    (520, 320, 256, 6, 64, 18),   # the largest expert count
+])
+def test_odd_shapes(T, d, E, k, f, seed):
+    shape = synth.MoEShape(T, d, E, k, f)
+    inp = synth.make_inputs(shape, seed, x_std=1.0)
+    ofw, obw = oracle_run(inp, k, 0.05)
+    check_all(Run(inp, k), ofw, obw, 0.05)
+
+
+def test_skewed_small_with_bias_and_empty_experts():
+    shape = synth.MoEShape(2048, 256, 32, 4, 256)
+    inp = synth.make_inputs(shape, 7, x_std=1.0, skew=True)
+    ofw, obw = oracle_run(inp, 4, 0.1)
+    assert (ofw["counts"] == 0).sum() >= 3
+    check_all(Run(inp, 4), ofw, obw, 0.1)
+
+
+def test_exact_ties_through_logits_in():
+    """Routing from caller-supplied logits with many exact ties must match the oracle bit for bit."""
+    shape = synth.MoEShape(512, 128, 16, 4, 128)
+    inp = synth.make_inputs(shape, 21, guard=False)
+    rng = np.random.default_rng(3)
+    logits = rng.integers(-2, 3, size=(512, 16)).astype(np.float32)
+    logits[:64] = 0.0  # all-ties rows: idx must be 0..k-1
+    ofw, obw = oracle_run(inp, 4, 0.0, logits_in=logits)
+    r = Run(inp, 4, logits_in=logits)
+    fw = r.forward()
+    check_routing(fw, ofw)
+    assert np.array_equal(fw["idx"].cpu().numpy()[:64], np.tile(np.arange(4, dtype=np.int32), (64, 1)))
+    assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+
+
+def test_all_ties_closed_form_on_gpu():
+    """W_r = 0: idx = (0..k-1) for every token, gates 1/k, aux = 1 exactly."""
+    shape = synth.MoEShape(300, 128, 8, 3, 128)
+    inp = synth.make_inputs(shape, 22, guard=False)
+    inp["W_r"] = np.zeros_like(inp["W_r"])
+    r = Run(inp, 3)
+    fw = r.forward()
+    assert np.array_equal(fw["idx"].cpu().numpy(), np.tile(np.arange(3, dtype=np.int32), (300, 1)))
+    np.testing.assert_allclose(fw["gates"].cpu().numpy(), 1.0 / 3.0, rtol=1e-6)
+    assert float(fw["aux"].cpu()[0]) == pytest.approx(1.0, rel=1e-6)
+    assert fw["counts"].cpu().numpy().tolist() == [300, 300, 300, 0, 0, 0, 0, 0]
+
+
+def test_zero_tokens():
+    shape = synth.MoEShape(0, 128, 8, 2, 128)
+    inp = synth.make_inputs(shape, 23, guard=False)
+    r = Run(inp, 2)
+    fw = r.forward()
+    assert fw["counts"].cpu().numpy().sum() == 0 and fw["y"].shape[0] == 0
+    bw = r.backward(0.0)
+    for nm in ("dW_gate", "dW_up", "dW_down"):
+        assert not bw[nm].float().cpu().numpy().any()
+    assert not bw["dW_r"].cpu().numpy().any()
+
+
+def test_repeated_calls_are_bitwise_reproducible():
+    inp = synth.make_inputs(synth.MoEShape(700, 256, 16, 4, 256), 24)
+    r = Run(inp, 4)
+    a = r.forward()
+    ga = r.backward(0.02)
+    b = r.forward()
+    gb = r.backward(0.02)
+    for n in ("y", "idx", "gates", "perm", "aux"):
+        assert torch.equal(a[n], b[n]), n
+    for n in ("dx", "dW_r", "dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(ga[n], gb[n]), n
+
+
+def test_midsize_qwen_shape_full_oracle():
+    """The Qwen3-30B-A3B expert shape with fewer tokens, full oracle in float32 mode."""
+    shape = synth.MoEShape(2048, 2048, 128, 8, 768)
+    inp = synth.make_inputs(shape, 31, x_std=1.0)
+    ofw, obw = oracle_run(inp, 8, 0.01, dtype=np.float32)
+    check_all(Run(inp, 8), ofw, obw, 0.01, stages=False)
+
+
+# ------------------------------------------------------------------------------------------ full-size configurations
+def sampled_parity(name, n_tokens=48):
+    """Full-size workloads in the launch configuration the benchmark times.  The oracle routes every token
+    (cheap) and computes y rows for sampled tokens plus complete weight gradients of four experts (hottest,
+    median, coldest non-empty, one empty if present); properties cover the rest."""
+    shape, seed, x_std, skew = synth.CONFIGS[name]
+    inp = synth.make_inputs(shape, seed, x_std=x_std, skew=skew)
+    k, E, T = shape.k, shape.E, shape.T
+    rt = orc.route_only(inp["x"], inp["W_r"], k, E, b_r=inp.get("b_r"))
+    r = Run(inp, k)
+    fw = r.forward()
+    check_routing(fw, rt)
+    perm = fw["perm"].cpu().numpy()
+    assert np.array_equal(np.sort(perm), np.arange(T * k))
+    inv = r.ints("inv")
+    pad = r.ints("pad_offsets")
+    assert (np.diff(pad) % 128 == 0).all() and np.array_equal(np.diff(pad) >= fw["counts"].cpu().numpy(), np.ones(E, bool))
+    assert len(np.unique(inv)) == T * k
+    rng = np.random.default_rng(seed)
+    toks = rng.choice(T, size=n_tokens, replace=False)
+    y = from_dev_bf16(fw["y"][torch.from_numpy(toks).cuda()])
+    ref = np.stack([orc.token_rows(int(t), rt, inp["x"], inp["W_gate"], inp["W_up"], inp["W_down"]) for t in toks])
+    assert rel_fro(y, ref) <= TOL
+    bw = r.backward(inp["d_aux"])
+    counts = rt["counts"]
+    order = np.argsort(counts)
+    nonempty = order[counts[order] > 0]
+    picks = {int(nonempty[-1]), int(nonempty[len(nonempty) // 2]), int(nonempty[0])}
+    if (counts == 0).any():
+        picks.add(int(order[0]))
+    for e in sorted(picks):
+        gg, gu, gd = orc.expert_grads(e, rt, inp["dy"], inp["x"], inp["W_gate"], inp["W_up"], inp["W_down"],
+                                      dtype=np.float32)
+        for nm, ref_e in (("dW_gate", gg), ("dW_up", gu), ("dW_down", gd)):
+            got = from_dev_bf16(bw[nm][e])
+            if counts[e] == 0:
+                assert not got.any()
+            else:
+                assert rel_fro(got, ref_e) <= 2e-2, (nm, e, int(counts[e]))
+    # dW_r against x^T dl with the GPU's own dl (host fp64 contraction), dl rows of sampled tokens sum to zero
+    dl = r.layer.buffer("dl", torch.float32).view(T, E).double().cpu().numpy()
+    assert np.abs(dl.sum(1)).max() <= 1e-4 * max(1.0, np.abs(dl).max())
+    ref_dwr = synth.bf16_bits_to_f64(inp["x"]).T @ dl
+    assert rel_fro(bw["dW_r"].cpu().numpy(), ref_dwr) <= 1e-3
+    assert torch.isfinite(bw["dx"].float()).all()
+
+
+def test_full_qwen_config_sampled():
+    sampled_parity("qwen")
+
+
+def test_full_skewed_config_sampled():
+    sampled_parity("skewed")
+
+
+def test_full_coarse_config_sampled():
+    sampled_parity("coarse", n_tokens=8)
+
+
+@pytest.mark.parametrize("name", ["sweep_T1000", "sweep_T8191"])
+def test_sweep_sampled(name):
+    sampled_parity(name, n_tokens=24)

@@ -1,0 +1,54 @@
+"""The N > 1 path of the benchmark is data parallel over tokens with replicated experts and no data-path
+collective; its host logic (rendezvous, per-rank token draws, barrier, max-over-ranks timing, whole-job
+throughput) runs here as two gloo ranks on CPU."""
+import os
+import sys
+
+import numpy as np
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    from oracle import moe_oracle as orc
+    from paper_2608_00916_b200 import dist as pdist
+    from paper_2608_00916_b200 import synth
+    pdist.init(world, rank, backend="gloo")
+    shape = synth.MoEShape(64, 64, 8, 2, 64)
+    base = synth.make_inputs(shape, 500, threads=1)          # weights: same seed on every rank
+    mine = synth.make_inputs(shape, pdist.shard_seed(500, rank), threads=1)
+    fw = orc.forward(mine["x"], base["W_r"], base["W_gate"], base["W_up"], base["W_down"], 2)
+    pdist.barrier()
+    ms = 10.0 * (rank + 1)  # pretend rank r took 10 (r + 1) ms
+    q.put((rank, pdist.max_over_ranks(ms), pdist.job_throughput(shape.T, ms), float(np.abs(fw["y"]).sum()),
+           int(base["W_gate"].view(np.uint16).sum()), int(mine["x"].view(np.uint16).sum())))
+    pdist.finish()
+
+
+def test_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29650 + os.getpid() % 200
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (r0, max0, thr0, y0, w0, x0), (r1, max1, thr1, y1, w1, x1) = res
+    assert max0 == max1 == 20.0                      # slowest rank decides
+    assert thr0 == thr1 == (64 + 64) / 0.020          # tokens of all ranks over that time
+    assert w0 == w1                                   # replicated weights
+    assert x0 != x1 and y0 != y1                      # different token batches per rank
+
+
+def test_token_split_is_balanced():
+    from paper_2608_00916_b200 import dist as pdist
+    for total, world in ((16384, 8), (8191, 4), (5, 8)):
+        parts = [pdist.tokens_per_rank(total, world, r) for r in range(world)]
+        assert sum(parts) == total and max(parts) - min(parts) <= 1
