@@ -39,6 +39,8 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.row_token = take(sizeof(int32_t) * L.rows_max);
   L.dg = take(sizeof(float) * R);
   L.dl = take(sizeof(float) * T * s.E);
+  L.dl_hi = take(sizeof(uint16_t) * (T * s.E + 64));
+  L.dl_lo = take(sizeof(uint16_t) * (T * s.E + 64));
   L.dwr_part = take(sizeof(float) * DWR_SPLIT * s.d * s.E);
   const size_t rows_d = sizeof(uint16_t) * L.rows_max * s.d, rows_f = sizeof(uint16_t) * L.rows_max * s.f;
   L.xp = take(rows_d);
@@ -49,6 +51,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.dhg = take(rows_f);
   L.dhu = take(rows_f);
   L.dxp = take(rows_d);
+  L.dxr = take(sizeof(uint16_t) * T * s.d);
   L.total = off;
   return L;
 }
@@ -152,6 +155,7 @@ moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char* name, s
              {"dhg", L.dhg, rows_f},
              {"dhu", L.dhu, rows_f},
              {"dxp", L.dxp, rows_d},
+             {"dxr", L.dxr, sizeof(uint16_t) * T * s.d},
              {"dg", L.dg, sizeof(float) * R},
              {"dl", L.dl, sizeof(float) * T * s.E},
              {"status", L.status, sizeof(int32_t) * 16}};
@@ -246,25 +250,35 @@ moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
+  GemmIO io;
+  io.x = x; io.W_r = W_r; io.b_r = b_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
+  io.idx_out = topk_idx; io.gates_out = topk_w; io.logits_out = logits_out;
+  const bool tc_router = router_on_tensor_cores(s) && logits_in == nullptr;
   {
     StageTimer tm(c, st, 0);
-    launch_router(s, T, x, W_r, b_r, logits_in, reinterpret_cast<float*>(ws + L.logits),
-                  reinterpret_cast<int32_t*>(ws + L.idx), reinterpret_cast<float*>(ws + L.gates), topk_idx, topk_w,
-                  logits_out, reinterpret_cast<float*>(ws + L.psum_part), st);
+    if (T > 0 && tc_router) {
+      rc = launch_grouped_gemm(c, GEMM_RT, T, L, ws, io, st);
+      if (rc != MOE_OK) return rc;
+    } else {
+      launch_router(s, T, x, W_r, b_r, logits_in, reinterpret_cast<float*>(ws + L.logits),
+                    reinterpret_cast<int32_t*>(ws + L.idx), reinterpret_cast<float*>(ws + L.gates), topk_idx, topk_w,
+                    logits_out, reinterpret_cast<float*>(ws + L.psum_part), st);
+    }
   }
   {
     StageTimer tm(c, st, 1);
-    launch_permute(s, T, L, ws, x, expert_counts, perm, aux_loss, st);
+    launch_permute(s, T, L, ws, x, expert_counts, perm, aux_loss,
+                   static_cast<int>(router_psum_rows(s, T, logits_in != nullptr)), st);
   }
   if (T > 0) {
     {
       StageTimer tm(c, st, 2);
-      rc = launch_grouped_gemm(c, GEMM_F3, T, L, ws, W_gate, W_up, W_down, nullptr, nullptr, nullptr, st);
+      rc = launch_grouped_gemm(c, GEMM_F3, T, L, ws, io, st);
     }
     if (rc != MOE_OK) return rc;
     {
       StageTimer tm(c, st, 3);
-      rc = launch_grouped_gemm(c, GEMM_F4, T, L, ws, W_gate, W_up, W_down, nullptr, nullptr, nullptr, st);
+      rc = launch_grouped_gemm(c, GEMM_F4, T, L, ws, io, st);
     }
     if (rc != MOE_OK) return rc;
     {
@@ -300,6 +314,10 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   float* dl = reinterpret_cast<float*>(ws + L.dl);
   const int32_t* inv = reinterpret_cast<const int32_t*>(ws + L.inv);
   const float* gates = reinterpret_cast<const float*>(ws + L.gates);
+  GemmIO io;
+  io.x = x; io.W_r = W_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
+  io.dW_gate = dW_gate; io.dW_up = dW_up; io.dW_down = dW_down; io.dx = dx;
+  const bool tc_router = router_on_tensor_cores(s);
   {
     StageTimer tm(c, st, 5);
     launch_combine_bwd(s, T, dy, reinterpret_cast<uint16_t*>(ws + L.o), gates, inv,
@@ -307,37 +325,49 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   }
   if (T > 0) {
     StageTimer tm(c, st, 6);
-    rc = launch_grouped_gemm(c, GEMM_B2, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+    rc = launch_grouped_gemm(c, GEMM_B2, T, L, ws, io, st);
   }
   if (rc != MOE_OK) return rc;
   {
     StageTimer tm(c, st, 7);
-    rc = launch_grouped_gemm(c, GEMM_B3, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+    rc = launch_grouped_gemm(c, GEMM_B3, T, L, ws, io, st);
   }
   if (rc != MOE_OK) return rc;
   if (T > 0) {
     StageTimer tm(c, st, 8);
-    rc = launch_grouped_gemm(c, GEMM_B4, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+    rc = launch_grouped_gemm(c, GEMM_B4, T, L, ws, io, st);
   }
   if (rc != MOE_OK) return rc;
   {
     StageTimer tm(c, st, 9);
-    rc = launch_grouped_gemm(c, GEMM_B5, T, L, ws, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, st);
+    rc = launch_grouped_gemm(c, GEMM_B5, T, L, ws, io, st);
   }
   if (rc != MOE_OK) return rc;
   {
     StageTimer tm(c, st, 10);
     launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
                       gates, reinterpret_cast<const float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts),
-                      d_aux, dl, st);
+                      d_aux, dl, reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo),
+                      st);
   }
   {
     StageTimer tm(c, st, 11);
-    launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, st);
+    if (tc_router && T > 0) {
+      rc = launch_grouped_gemm(c, GEMM_DWR, T, L, ws, io, st);
+      if (rc != MOE_OK) return rc;
+    }
+    launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, tc_router && T > 0, st);
   }
   {
     StageTimer tm(c, st, 12);
-    launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, st);
+    if (tc_router && T > 0) {
+      rc = launch_grouped_gemm(c, GEMM_DX, T, L, ws, io, st);
+      if (rc != MOE_OK) return rc;
+      launch_unpermute_sum(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv,
+                           reinterpret_cast<const uint16_t*>(ws + L.dxr), dx, st);
+    } else {
+      launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, st);
+    }
   }
   if (c->profiling) c->prof_step++;
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;

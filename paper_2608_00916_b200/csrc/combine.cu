@@ -136,7 +136,8 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
                                                          const int32_t* __restrict__ idx,
                                                          const float* __restrict__ gates, const float* __restrict__ dg,
                                                          const int32_t* __restrict__ counts, float d_aux,
-                                                         float* __restrict__ dl) {
+                                                         float* __restrict__ dl, uint16_t* __restrict__ dl_hi,
+                                                         uint16_t* __restrict__ dl_lo) {
   const int lane = threadIdx.x & 31;
   const int64_t t = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (t >= T) return;
@@ -198,15 +199,23 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
     int e = lane + 32 * q;
-    if (q < NQ && e < E) dl[t * E + e] = out[q];
+    if (q < NQ && e < E) {
+      dl[t * E + e] = out[q];
+      // exact two-term bf16 split (hi + lo reproduces dl to about 2^-17 relative) for the tensor-core contractions
+      const __nv_bfloat16 h = __float2bfloat16_rn(out[q]);
+      const __nv_bfloat16 l = __float2bfloat16_rn(out[q] - __bfloat162float(h));
+      dl_hi[t * E + e] = *reinterpret_cast<const uint16_t*>(&h);
+      dl_lo[t * E + e] = *reinterpret_cast<const uint16_t*>(&l);
+    }
   }
 }
 
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
-                       const float* dg, const int32_t* counts, float d_aux, float* dl, cudaStream_t st) {
+                       const float* dg, const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi,
+                       uint16_t* dl_lo, cudaStream_t st) {
   if (T == 0) return;
   router_bwd_kernel<<<static_cast<unsigned>((T + 7) / 8), 256, 0, st>>>(T, s.E, s.k, logits, idx, gates, dg, counts,
-                                                                        d_aux, dl);
+                                                                        d_aux, dl, dl_hi, dl_lo);
 }
 
 // ------------------------------------------------------------------------------------------ dW_r, db_r
@@ -302,10 +311,12 @@ __global__ void __launch_bounds__(256) dbr_kernel(int64_t T, int E, const float*
 }
 
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
-                float* db_r, cudaStream_t st) {
+                float* db_r, bool partials_ready, cudaStream_t st) {
   const int64_t n = static_cast<int64_t>(s.d) * s.E;
-  dim3 grid(s.d / DW_BM, DWR_SPLIT);
-  dwr_partial_kernel<<<grid, 256, sizeof(float) * DW_BK * s.E, st>>>(T, s.d, s.E, x, dl, part);
+  if (!partials_ready) {
+    dim3 grid(s.d / DW_BM, DWR_SPLIT);
+    dwr_partial_kernel<<<grid, 256, sizeof(float) * DW_BK * s.E, st>>>(T, s.d, s.E, x, dl, part);
+  }
   dwr_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(n, part, dW_r);
   if (db_r) dbr_kernel<<<(s.E + 31) / 32, 256, 0, st>>>(T, s.E, dl, db_r);
 }
@@ -400,6 +411,48 @@ __global__ void __launch_bounds__(256) unpermute_bwd_kernel(int64_t T, int d, in
       }
     }
   }
+}
+
+// dx[t,:] = dxr[t,:] + sum_j dxp[inv[t,j],:]; one block per token, 16-byte accesses, all row loads in flight at once.
+__global__ void __launch_bounds__(256) unpermute_sum_kernel(int d, int k, const uint16_t* __restrict__ dxp,
+                                                            const int32_t* __restrict__ inv,
+                                                            const uint16_t* __restrict__ dxr,
+                                                            uint16_t* __restrict__ dx) {
+  const int64_t t = blockIdx.x;
+  __shared__ int sr[MAX_K];
+  if (threadIdx.x < k) sr[threadIdx.x] = inv[t * k + threadIdx.x];
+  __syncthreads();
+  for (int c = threadIdx.x * 8; c < d; c += 256 * 8) {
+    float acc[8];
+    {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(dxr + t * d + c));
+      unpack_bf16x2(v.x, acc[0], acc[1]);
+      unpack_bf16x2(v.y, acc[2], acc[3]);
+      unpack_bf16x2(v.z, acc[4], acc[5]);
+      unpack_bf16x2(v.w, acc[6], acc[7]);
+    }
+#pragma unroll 8
+    for (int j = 0; j < k; ++j) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(dxp + static_cast<int64_t>(sr[j]) * d + c));
+      float a, b;
+      unpack_bf16x2(v.x, a, b); acc[0] += a; acc[1] += b;
+      unpack_bf16x2(v.y, a, b); acc[2] += a; acc[3] += b;
+      unpack_bf16x2(v.z, a, b); acc[4] += a; acc[5] += b;
+      unpack_bf16x2(v.w, a, b); acc[6] += a; acc[7] += b;
+    }
+    uint4 w;
+    w.x = pack_bf16x2(acc[0], acc[1]);
+    w.y = pack_bf16x2(acc[2], acc[3]);
+    w.z = pack_bf16x2(acc[4], acc[5]);
+    w.w = pack_bf16x2(acc[6], acc[7]);
+    *reinterpret_cast<uint4*>(dx + t * d + c) = w;
+  }
+}
+
+void launch_unpermute_sum(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const uint16_t* dxr,
+                          uint16_t* dx, cudaStream_t st) {
+  if (T == 0) return;
+  unpermute_sum_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, dxp, inv, dxr, dx);
 }
 
 void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const float* dl,

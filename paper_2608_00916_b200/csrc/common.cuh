@@ -43,12 +43,14 @@ struct WsLayout {
   size_t row_token;    // int32[rows_max] token of a padded row, -1 for pad rows
   size_t dg;           // float[T*k]
   size_t dl;           // float[T*E]
+  size_t dl_hi, dl_lo; // bf16[T*E]   dl split into two bf16 terms (hi + lo) for the tensor-core contractions
   size_t dwr_part;     // float[DWR_SPLIT * d * E]
   size_t xp;           // bf16[rows_max * d]
   size_t hg, hu, act;  // bf16[rows_max * f]
   size_t o;            // bf16[rows_max * d]   o in forward, overwritten by d_o in backward
   size_t dhg, dhu;     // bf16[rows_max * f]
   size_t dxp;          // bf16[rows_max * d]
+  size_t dxr;          // bf16[T * d]  router term of dx (dl W_r^T)
   size_t total;
   int64_t rows_max;    // upper bound of the padded row total for T tokens
   int64_t max_m_tiles;
@@ -76,23 +78,49 @@ void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t*
                    const float* logits_in, float* logits, int32_t* idx, float* gates, int32_t* idx_out,
                    float* gates_out, float* logits_out, float* psum_part, cudaStream_t st);
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
-                    int32_t* perm_out, float* aux_out, cudaStream_t st);
+                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st);
 // ---- launchers (combine.cu)
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
                     uint16_t* y, cudaStream_t st);
 void launch_combine_bwd(const Shape& s, int64_t T, const uint16_t* dy, uint16_t* o_to_do, const float* gates,
                         const int32_t* inv, float* dg, cudaStream_t st);
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
-                       const float* dg, const int32_t* counts, float d_aux, float* dl, cudaStream_t st);
+                       const float* dg, const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi,
+                       uint16_t* dl_lo, cudaStream_t st);
+// SIMT dW_r (any E) and the shared partial reduction / db_r
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
-                float* db_r, cudaStream_t st);
+                float* db_r, bool partials_ready, cudaStream_t st);
 void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const float* dl,
                           const uint16_t* W_r, uint16_t* dx, cudaStream_t st);
+// dx[t,:] = dxr[t,:] + sum_j dxp[inv[t,j],:]  (router term already contracted on the tensor cores)
+void launch_unpermute_sum(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const uint16_t* dxr,
+                          uint16_t* dx, cudaStream_t st);
 // ---- launchers (gemm.cu); each returns a CUDA / driver error as moe_status
-enum GemmKind { GEMM_F3 = 0, GEMM_F4, GEMM_B2, GEMM_B3, GEMM_B4, GEMM_B5 };
+enum GemmKind { GEMM_F3 = 0, GEMM_F4, GEMM_B2, GEMM_B3, GEMM_B4, GEMM_B5, GEMM_RT, GEMM_DX, GEMM_DWR, GEMM_KINDS };
+// Caller tensors a grouped-GEMM launch may need besides the workspace.
+struct GemmIO {
+  const uint16_t* x = nullptr;
+  const uint16_t* W_r = nullptr;
+  const float* b_r = nullptr;
+  const uint16_t* W_gate = nullptr;
+  const uint16_t* W_up = nullptr;
+  const uint16_t* W_down = nullptr;
+  uint16_t* dW_gate = nullptr;
+  uint16_t* dW_up = nullptr;
+  uint16_t* dW_down = nullptr;
+  uint16_t* dx = nullptr;
+  int32_t* idx_out = nullptr;
+  float* gates_out = nullptr;
+  float* logits_out = nullptr;
+};
 moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
-                               const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
-                               uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, cudaStream_t st);
+                               const GemmIO& io, cudaStream_t st);
+// true when the tensor-core router / dW_r / dx kernels apply (their TMA maps need E % 8 == 0)
+inline bool router_on_tensor_cores(const Shape& s) { return s.E % 8 == 0; }
+// psum_part rows written by the router: one per warp of a 128-token tile (tensor cores) or per ROUTER_TOK tokens (SIMT)
+inline int64_t router_psum_rows(const Shape& s, int64_t T, bool logits_given) {
+  return (router_on_tensor_cores(s) && !logits_given) ? 4 * ((T + 127) / 128) : (T + ROUTER_TOK - 1) / ROUTER_TOK;
+}
 
 // ---- device helpers
 __device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }

@@ -7,6 +7,11 @@
 //   B4  dxp     = dhg W_gate[e]^T + dhu W_up[e]^T   (one accumulator, two K segments)
 //   B3  dW_down[e]          = act_e^T d_o_e         (K = rows of expert e, one CTA owns a whole output tile)
 //   B5  dW_gate[e]|dW_up[e] = xp_e^T [dhg_e|dhu_e]
+// and the three contractions of the router, whose operands are bf16 (or fp32 split exactly into two bf16 terms),
+// so that a bf16 MMA with fp32 accumulation is an fp32 contraction up to summation order:
+//   RT  logits = x W_r (+ b_r)                      + routing epilogue (top-k, gates, softmax column sums)
+//   DX  dxr    = dl_hi W_r^T + dl_lo W_r^T          (router term of dx; the unpermute kernel adds the dxp rows)
+//   DWR dW_r partial[s] = x_s^T (dl_hi + dl_lo)_s   (token slices s; partials are summed by a small kernel)
 // Tiles are 128 x 256 with K steps of 64; operands arrive by TMA into 128-byte-swizzled shared memory (4 stages),
 // the accumulator lives in tensor memory (2 x 256 columns, so the epilogue of one tile overlaps the main loop
 // of the next).  Operand major-ness replaces every transpose: row-major [rows, K] is a K-major operand,
@@ -50,16 +55,32 @@ struct GemmParams {
   const uint16_t* in1;
   int64_t ld_out;
   int64_t expert_stride;
+  // router kinds
+  int static_m_tiles;   // RT, DX: number of 128-token tiles
+  int split_rows;       // DWR: tokens per slice (multiple of 64)
+  int rows_total;       // DWR: tokens rounded up to 64
+  int top_k;
+  int64_t T;
+  const float* bias;    // RT: [E] or null
+  float* logits;        // RT: [T,E] saved logits
+  float* logits_out;    // RT: optional copy for the caller
+  int32_t* idx;         // RT: [T,k] (workspace) and idx_out (caller)
+  int32_t* idx_out;
+  float* gates;
+  float* gates_out;
+  float* psum_part;     // RT: [4 * tiles, E] per-warp column sums of p
+  float* outf;          // DWR: [slices, d, E] fp32 partials
 };
 
 template <int KIND>
 struct Traits {
-  static constexpr bool WGRAD = (KIND == GEMM_B3 || KIND == GEMM_B5);
+  static constexpr bool WGRAD = (KIND == GEMM_B3 || KIND == GEMM_B5 || KIND == GEMM_DWR);
+  static constexpr bool STATIC_M = (KIND == GEMM_RT || KIND == GEMM_DX);  // token tiles, no expert lookup
   static constexpr int A_MN = WGRAD ? 1 : 0;
-  static constexpr int B_MN = (KIND == GEMM_B2 || KIND == GEMM_B4) ? 0 : 1;
-  static constexpr int NSEG = (KIND == GEMM_B4) ? 2 : 1;
-  // width of output covered by one N tile (F3 / B5 pair a 128-wide gate tile with the matching up tile)
-  static constexpr int N_SPAN = (KIND == GEMM_F3 || KIND == GEMM_B5) ? 128 : 256;
+  static constexpr int B_MN = (KIND == GEMM_B2 || KIND == GEMM_B4 || KIND == GEMM_DX) ? 0 : 1;
+  static constexpr int NSEG = (KIND == GEMM_B4 || KIND == GEMM_DX) ? 2 : 1;
+  // width of output covered by one N tile (F3 / B5 / DWR pair a 128-wide tile with a second 128-wide operand)
+  static constexpr int N_SPAN = (KIND == GEMM_F3 || KIND == GEMM_B5 || KIND == GEMM_DWR) ? 128 : 256;
 };
 
 struct Tile {
@@ -69,6 +90,7 @@ struct Tile {
 template <int KIND>
 __device__ __forceinline__ int total_tiles(const GemmParams& p) {
   if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;
+  if (Traits<KIND>::STATIC_M) return p.static_m_tiles * p.n_tiles;
   return p.sched[0] * p.n_tiles;
 }
 
@@ -81,8 +103,20 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     const int rem = t - tl.e * per;
     tl.m0 = (rem / p.n_tiles) * BM;
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
-    tl.row0 = p.pad_offsets[tl.e];
-    tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
+    if (KIND == GEMM_DWR) {  // "expert" = token slice
+      tl.row0 = tl.e * p.split_rows;
+      tl.nkb = max(0, min(p.split_rows, p.rows_total - tl.row0)) / BK;
+    } else {
+      tl.row0 = p.pad_offsets[tl.e];
+      tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
+    }
+  } else if (Traits<KIND>::STATIC_M) {
+    const int mt = t / p.n_tiles;
+    tl.e = 0;
+    tl.row0 = mt * BM;
+    tl.m0 = 0;
+    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
   } else {
     const int mt = t / p.n_tiles;
     tl.e = p.tile_expert[mt];
@@ -104,14 +138,14 @@ __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl,
       tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
       tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
     }
-  } else if (KIND == GEMM_F4) {
+  } else if (KIND == GEMM_F4 || KIND == GEMM_RT) {
     tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
 #pragma unroll
     for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
   } else if (KIND == GEMM_B2) {
     tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
     tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
-  } else if (KIND == GEMM_B4) {
+  } else if (KIND == GEMM_B4 || KIND == GEMM_DX) {
     const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
     tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
     tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
@@ -121,7 +155,7 @@ __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl,
     for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
 #pragma unroll
     for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
-  } else {  // GEMM_B5
+  } else {  // GEMM_B5, GEMM_DWR
     const int row = tl.row0 + kb * BK;
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
@@ -163,6 +197,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   extern __shared__ unsigned char gemm_smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
   __shared__ uint32_t tmem_base_slot;
+  __shared__ float s_bias[KIND == GEMM_RT ? MAX_E : 1];  // router bias (zero beyond E)
+  if (KIND == GEMM_RT)
+    for (int i = threadIdx.x; i < MAX_E; i += GEMM_THREADS) s_bias[i] = (p.bias && i < p.N_total) ? p.bias[i] : 0.f;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(gemm_smem_raw) + 1023u) & ~1023u;
@@ -277,7 +314,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       const int rin = ew * 32 + lane;  // row inside the tile
       if (tl.nkb == 0) {
         // weight gradient of an expert without tokens: zeros
-        if (TR::WGRAD) {
+        if (KIND == GEMM_DWR) {
+          const int m = tl.m0 + rin;
+          if (m < p.M_total)
+            for (int col = tl.n0; col < min(tl.n0 + 128, p.N_total); col += 4)
+              *reinterpret_cast<float4*>(p.outf + (static_cast<int64_t>(tl.e) * p.M_total + m) * p.N_total + col) =
+                  make_float4(0.f, 0.f, 0.f, 0.f);
+        } else if (TR::WGRAD) {
           const int m = tl.m0 + rin;
           if (m < p.M_total) {
             float z[32];
@@ -352,6 +395,122 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
             store_bf16x32(p.out1 + off, dhu);
           }
         }
+      } else if (KIND == GEMM_RT) {
+        // Routing epilogue: one thread per token; the row of E logits is re-read from tensor memory in every
+        // pass.  Pass j picks the largest logit that comes after pick j-1 in the order (value descending,
+        // index ascending), which is the rule "largest not taken yet, lowest index among equals".
+        const int64_t tok = row;
+        const bool valid = tok < p.T;
+        const int E = p.N_total, k = p.top_k;
+        const int nch = (E + 31) >> 5;
+        float selv[MAX_K];
+        int seli[MAX_K];
+        float pv = INFINITY;
+        int pi = -1;
+        for (int j = 0; j < k; ++j) {
+          float bv = -INFINITY;
+          int bi = 0x7FFFFFFF;
+          for (int c = 0; c < nch; ++c) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_ld_wait();
+            float val[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) val[i] = __uint_as_float(r[i]) + s_bias[c * 32 + i];
+            if (j == 0 && valid) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4) {
+                if (c * 32 + i < E) {
+                  const float4 w = make_float4(val[i], val[i + 1], val[i + 2], val[i + 3]);
+                  *reinterpret_cast<float4*>(p.logits + tok * E + c * 32 + i) = w;
+                  if (p.logits_out) *reinterpret_cast<float4*>(p.logits_out + tok * E + c * 32 + i) = w;
+                }
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int e = c * 32 + i;
+              const bool after = (val[i] < pv) || (val[i] == pv && e > pi);
+              if (e < E && after && val[i] > bv) {
+                bv = val[i];
+                bi = e;
+              }
+            }
+          }
+          selv[j] = bv;
+          seli[j] = bi;
+          pv = bv;
+          pi = bi;
+        }
+        const float vmax = selv[0];
+        float z = 0.f;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i < E) z += expf(__uint_as_float(r[i]) + s_bias[c * 32 + i] - vmax);
+        }
+        const float rz = valid ? 1.f / z : 0.f;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+          float pc[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            pc[i] = (c * 32 + i < E) ? expf(__uint_as_float(r[i]) + s_bias[c * 32 + i] - vmax) * rz : 0.f;
+          // column sums over the 32 tokens of this warp: butterfly transpose-reduce, lane L ends with column L
+#pragma unroll
+          for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              if (i < cnt) {
+                const bool up = (lane & off) != 0;
+                const float send = up ? pc[i] : pc[i + cnt];
+                const float keep = up ? pc[i + cnt] : pc[i];
+                pc[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
+              }
+            }
+          }
+          if (c * 32 + lane < E)
+            p.psum_part[(static_cast<int64_t>(tl.row0 / BM) * 4 + ew) * E + c * 32 + lane] = pc[0];
+        }
+        if (valid) {
+          float zs = 0.f;
+          for (int j = 0; j < k; ++j) zs += expf(selv[j] - vmax);
+          const float rzs = 1.f / zs;
+          for (int j = 0; j < k; ++j) {
+            const float g = expf(selv[j] - vmax) * rzs;
+            p.idx[tok * k + j] = seli[j];
+            p.gates[tok * k + j] = g;
+            p.idx_out[tok * k + j] = seli[j];
+            p.gates_out[tok * k + j] = g;
+          }
+        }
+      } else if (KIND == GEMM_DWR) {
+        // fp32 partial of dW_r for this token slice: hi and lo halves of dl share one accumulator pair
+        const int m = tl.m0 + rin;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t rh[32], rl[32];
+          tmem_ld32(taddr + c * 32, rh);
+          tmem_ld32(taddr + 128 + c * 32, rl);
+          tmem_ld_wait();
+          const int col = tl.n0 + c * 32;
+          if (m < p.M_total) {
+            float* dst = p.outf + (static_cast<int64_t>(tl.e) * p.M_total + m) * p.N_total + col;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              if (col + i < p.N_total)
+                *reinterpret_cast<float4*>(dst + i) = make_float4(
+                    __uint_as_float(rh[i]) + __uint_as_float(rl[i]), __uint_as_float(rh[i + 1]) + __uint_as_float(rl[i + 1]),
+                    __uint_as_float(rh[i + 2]) + __uint_as_float(rl[i + 2]),
+                    __uint_as_float(rh[i + 3]) + __uint_as_float(rl[i + 3]));
+            }
+          }
+        }
       } else {
         // plain bf16 store: F4, B4 (row GEMMs), B3, B5 (weight gradients)
 #pragma unroll 1
@@ -374,7 +533,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
               store_bf16x32(base + tl.e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, v);
           } else {
             const int col = tl.n0 + c * 32;
-            if (col < p.N_total) store_bf16x32(p.out0 + row * p.ld_out + col, v);
+            const bool in_rows = (KIND != GEMM_DX) || row < p.T;  // token tiles may overhang T
+            if (in_rows && col < p.N_total) store_bf16x32(p.out0 + row * p.ld_out + col, v);
           }
         }
       }
@@ -426,7 +586,7 @@ static bool map_3d(void* fn, CUtensorMap* m, const void* base, int64_t E, int64_
 
 template <int KIND>
 static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream_t st) {
-  static bool attr_done[8] = {false};
+  static bool attr_done[GEMM_KINDS] = {false};
   if (!attr_done[KIND]) {
     if (cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(GEMM_SMEM)) != cudaSuccess)
@@ -438,8 +598,9 @@ static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream
 }
 
 moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
-                               const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
-                               uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, cudaStream_t st) {
+                               const GemmIO& io, cudaStream_t st) {
+  const uint16_t *W_gate = io.W_gate, *W_up = io.W_up, *W_down = io.W_down;
+  uint16_t *dW_gate = io.dW_gate, *dW_up = io.dW_up, *dW_down = io.dW_down;
   const Shape& s = ctx->s;
   const int d = s.d, f = s.f, E = s.E;
   const int64_t R = L.rows_max;
@@ -528,6 +689,60 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.expert_stride = static_cast<int64_t>(d) * f;
       if (!ok) return MOE_ERR_CUDA;
       return launch_kind<GEMM_B5>(ctx, p, st);
+    case GEMM_RT:
+      // logits[T,E] = x[T,d] W_r[d,E]; W_r is read as a one-slab 3D tensor so the weight loaders apply
+      ok = map_2d(fn, &p.mapA0, io.x, T, d, 128) && map_3d(fn, &p.mapB0, io.W_r, 1, d, E, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.static_m_tiles = static_cast<int>((T + BM - 1) / BM);
+      p.n_tiles = 1;
+      p.k_blocks = d / BK;
+      p.N_total = E;
+      p.T = T;
+      p.top_k = s.k;
+      p.bias = io.b_r;
+      p.logits = reinterpret_cast<float*>(ws + L.logits);
+      p.logits_out = io.logits_out;
+      p.idx = reinterpret_cast<int32_t*>(ws + L.idx);
+      p.gates = reinterpret_cast<float*>(ws + L.gates);
+      p.idx_out = io.idx_out;
+      p.gates_out = io.gates_out;
+      p.psum_part = reinterpret_cast<float*>(ws + L.psum_part);
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_RT>(ctx, p, st);
+    case GEMM_DX:
+      // dxr[T,d] = dl_hi W_r^T + dl_lo W_r^T
+      ok = map_2d(fn, &p.mapA0, ws + L.dl_hi, T, E, 128) && map_2d(fn, &p.mapA1, ws + L.dl_lo, T, E, 128) &&
+           map_3d(fn, &p.mapB0, io.W_r, 1, d, E, 256);
+      p.mapB1 = p.mapB0;
+      p.static_m_tiles = static_cast<int>((T + BM - 1) / BM);
+      p.n_tiles = (d + 255) / 256;
+      p.k_blocks = (E + BK - 1) / BK;
+      p.N_total = d;
+      p.T = T;
+      p.top_k = s.k;
+      p.out0 = reinterpret_cast<uint16_t*>(ws + L.dxr);
+      p.ld_out = d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_DX>(ctx, p, st);
+    case GEMM_DWR: {
+      // partial[s][d,E] = x_s^T (dl_hi + dl_lo)_s over token slices of split_rows tokens
+      ok = map_2d(fn, &p.mapA0, io.x, T, d, 64) && map_2d(fn, &p.mapB0, ws + L.dl_hi, T, E, 64) &&
+           map_2d(fn, &p.mapB1, ws + L.dl_lo, T, E, 64);
+      p.mapA1 = p.mapA0;
+      const int64_t per = ((T + DWR_SPLIT - 1) / DWR_SPLIT + BK - 1) / BK * BK;
+      p.split_rows = static_cast<int>(per);
+      p.rows_total = static_cast<int>((T + BK - 1) / BK * BK);
+      p.E = DWR_SPLIT;  // slices play the role of experts in the tile list
+      p.m_tiles = (d + 127) / 128;
+      p.n_tiles = (E + 127) / 128;
+      p.M_total = d;
+      p.N_total = E;
+      p.outf = reinterpret_cast<float*>(ws + L.dwr_part);
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_DWR>(ctx, p, st);
+    }
+    default:
+      break;
   }
   (void)T;
   return MOE_ERR_INVALID_ARG;

@@ -226,23 +226,36 @@ __global__ void __launch_bounds__(TOK_TILE) hist_kernel(int64_t T, int E, int k,
 }
 
 // One block: column scan of tile_counts (in place -> exclusive prefix along tiles), counts, canonical and
-// padded offsets, tile -> expert table, and the auxiliary loss from the per-block column sums of p.
-__global__ void __launch_bounds__(256) scan_kernel(int64_t T, int E, int k, int tok_tiles, int router_blocks,
-                                                   int32_t* __restrict__ tile_counts, int32_t* __restrict__ counts,
-                                                   int32_t* __restrict__ offsets, int32_t* __restrict__ pad_offsets,
-                                                   int32_t* __restrict__ sched, int32_t* __restrict__ tile_expert,
-                                                   const float* __restrict__ psum_part, float* __restrict__ psum,
-                                                   int32_t* __restrict__ counts_out, float* __restrict__ aux_out,
-                                                   int32_t* __restrict__ status) {
+// padded offsets, tile -> expert table, and the auxiliary loss from the router's partial column sums of p
+// (summed in a fixed order: reproducible).
+constexpr int SCAN_THREADS = 1024;
+__global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, int k, int tok_tiles, int psum_rows,
+                                                            int32_t* __restrict__ tile_counts,
+                                                            int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                                                            int32_t* __restrict__ pad_offsets,
+                                                            int32_t* __restrict__ sched, int32_t* __restrict__ tile_expert,
+                                                            const float* __restrict__ psum_part,
+                                                            float* __restrict__ psum, int32_t* __restrict__ counts_out,
+                                                            float* __restrict__ aux_out, int32_t* __restrict__ status) {
   __shared__ int s_cnt[MAX_E];
   __shared__ int s_pad[MAX_E + 1];
   __shared__ float s_term[MAX_E];
+  __shared__ float s_ps[SCAN_THREADS];
   const int tid = threadIdx.x;
   if (tid == 0) {
     status[0] = DEV_OK;
     status[1] = 0;
   }
-  for (int e = tid; e < E; e += 256) {
+  // column sums of p: G groups of threads stride over the partial rows
+  const int G = SCAN_THREADS / E;
+  if (tid < G * E) {
+    const int g = tid / E, e = tid - g * E;
+    float ps = 0.f;
+    for (int b = g; b < psum_rows; b += G) ps += psum_part[static_cast<int64_t>(b) * E + e];
+    s_ps[tid] = ps;
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += SCAN_THREADS) {
     int run = 0;
     for (int tl = 0; tl < tok_tiles; ++tl) {
       int c = tile_counts[static_cast<int64_t>(tl) * E + e];
@@ -253,7 +266,7 @@ __global__ void __launch_bounds__(256) scan_kernel(int64_t T, int E, int k, int 
     counts[e] = run;
     counts_out[e] = run;
     float ps = 0.f;
-    for (int b = 0; b < router_blocks; ++b) ps += psum_part[static_cast<int64_t>(b) * E + e];
+    for (int g = 0; g < G; ++g) ps += s_ps[g * E + e];
     psum[e] = ps;
     // aux term: (c_e / (T k)) * (Psum_e / T)
     s_term[e] = (T > 0) ? (static_cast<float>(run) / static_cast<float>(T * k)) * (ps / static_cast<float>(T)) : 0.f;
@@ -278,7 +291,7 @@ __global__ void __launch_bounds__(256) scan_kernel(int64_t T, int E, int k, int 
     aux_out[0] = aux * static_cast<float>(E);
   }
   __syncthreads();
-  for (int e = tid; e < E; e += 256) {
+  for (int e = tid; e < E; e += SCAN_THREADS) {
     for (int m = s_pad[e] / ROW_PAD; m < s_pad[e + 1] / ROW_PAD; ++m) tile_expert[m] = e;
   }
 }
@@ -327,7 +340,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(int d, const uint16_t*
 }
 
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
-                    int32_t* perm_out, float* aux_out, cudaStream_t st) {
+                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st) {
   int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
   int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
   int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
@@ -335,7 +348,7 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
   const size_t msm = sizeof(uint32_t) * 8 * s.E;
   cudaMemsetAsync(row_token, 0xFF, sizeof(int32_t) * L.rows_max, st);
   if (tiles > 0) hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
-  scan_kernel<<<1, 256, 0, st>>>(T, s.E, s.k, tiles, static_cast<int>(L.router_blocks), tile_counts,
+  scan_kernel<<<1, SCAN_THREADS, 0, st>>>(T, s.E, s.k, tiles, psum_rows, tile_counts,
                                  reinterpret_cast<int32_t*>(ws + L.counts), reinterpret_cast<int32_t*>(ws + L.offsets),
                                  reinterpret_cast<int32_t*>(ws + L.pad_offsets),
                                  reinterpret_cast<int32_t*>(ws + L.sched),
