@@ -149,6 +149,29 @@ MOE_API moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, cons
                          float* dW_r, uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down,
                          void* dev /* device */, size_t dev_bytes, void* cuda_stream);
 
+/* Router weight gradient without any device allocation:  dW_r[d,E] = sum_t x[t,:]^T dl[t,:].
+ * (The paper has no counterpart of this call; it exists for integration reasons only.)
+ *
+ * Who it is for.  moe_backward needs a caller-provided workspace, which in practice means the caller can
+ * allocate device memory.  Some callers cannot: a plug-in running inside a host application that handed all device
+ * memory to its own pool at start-up, or a service loop that cannot afford the device-wide synchronisation that
+ * cudaMalloc and cudaFree imply.  For them this one call keeps its scratch (the per-token-slice partial sums)
+ * in a fixed array that is part of the library image, and calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   x  [T,d] bf16 (device),  dl [T,E] fp32 (device, the router-logit gradient),  dW_r [d,E] fp32 (device, overwritten).
+ *   d must be a multiple of 64, 1 <= E <= 256, and d * E <= MOE_STATIC_MAX_DE; larger shapes are refused with
+ *   MOE_ERR_UNSUPPORTED before anything is launched (use moe_backward with a workspace instead).
+ *
+ * Cost and rules.  The scratch is MOE_STATIC_MAX_DE * 8 floats = 8 MiB of device memory on every GPU that loads the
+ * library, held until the process ends.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call during start-up, ahead of any stream
+ * capture.  All calls on one GPU share the array: two calls whose kernels can overlap on the GPU (different streams,
+ * different threads) race on it and must be ordered by the caller.  The array keeps whatever the previous call
+ * left; that is harmless because each call overwrites every partial it later reads. */
+#define MOE_STATIC_MAX_DE 262144
+MOE_API moe_status moe_router_wgrad_static(int64_t T, int32_t d, int32_t E, const uint16_t* x, const float* dl,
+                                           float* dW_r, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -14,7 +14,8 @@ STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine"
                "unpermute_bwd"]
 EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
-           "moe_e2e_device_bytes", "moe_step_host"]
+           "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static"]
+STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
 class MoEConfig(C.Structure):
@@ -61,6 +62,8 @@ def load_library() -> C.CDLL:
     lib.moe_e2e_device_bytes.restype = sz
     lib.moe_step_host.argtypes = [vp, i64, C.c_int] + [vp] * 6 + [C.c_float] + [vp] * 7 + [vp, sz, vp]
     lib.moe_step_host.restype = C.c_int
+    lib.moe_router_wgrad_static.argtypes = [i64, C.c_int32, C.c_int32, vp, vp, vp, vp]
+    lib.moe_router_wgrad_static.restype = C.c_int
     _lib = lib
     return lib
 
@@ -72,6 +75,25 @@ def _check(lib, rc: int, what: str) -> None:
 
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def router_wgrad_static(x, dl, dW_r=None):
+    """dW_r = x^T dl through the entry point that allocates nothing inside the library (its scratch is a fixed
+    array in the library image).  x: bf16 [T,d] CUDA tensor, dl: fp32 [T,E] CUDA tensor.  The output tensor is the
+    caller's: pass dW_r (fp32 [d,E]) to reuse one, otherwise torch allocates it here, outside the library.
+    Raises MoEError (unsupported) when d * E exceeds STATIC_MAX_DE."""
+    import torch
+    lib = load_library()
+    T, d = x.shape
+    E = dl.shape[1]
+    assert x.dtype == torch.bfloat16 and dl.dtype == torch.float32 and x.is_contiguous() and dl.is_contiguous()
+    assert dl.shape[0] == T
+    if dW_r is None:
+        dW_r = torch.empty(d, E, dtype=torch.float32, device=x.device)
+    rc = lib.moe_router_wgrad_static(T, d, E, _ptr(x), _ptr(dl), _ptr(dW_r),
+                                     C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    _check(lib, rc, "moe_router_wgrad_static")
+    return dW_r
 
 
 class MoELayer:
