@@ -51,8 +51,12 @@ typedef struct {
   int32_t E;      /* experts,      1 <= E <= 256                                   */
   int32_t f;      /* expert width, multiple of 64                                  */
   int32_t top_k;  /* experts per token, 1 <= top_k <= E and top_k <= 32            */
-  int32_t flags;  /* reserved, pass 0                                              */
+  int32_t flags;  /* 0, or MOE_FLAG_SINGLE_CTA_TILES                               */
 } moe_config;
+
+/* Runs the expert GEMMs on one-CTA 128 x 256 tiles instead of the default CTA pairs (256 x 256 tiles, tcgen05
+ * cta_group::2).  Same results; kept for comparison measurements. */
+#define MOE_FLAG_SINGLE_CTA_TILES 1
 
 typedef struct moe_ctx moe_ctx; /* opaque, lives in host memory */
 

@@ -102,10 +102,10 @@ class MoELayer:
     forward() / backward() take and return torch CUDA tensors (bf16 for activations and weights); the
     tensors are only carriers of device pointers."""
 
-    def __init__(self, d: int, E: int, f: int, top_k: int):
+    def __init__(self, d: int, E: int, f: int, top_k: int, flags: int = 0):
         self.lib = load_library()
         self.d, self.E, self.f, self.k = d, E, f, top_k
-        cfg = MoEConfig(d, E, f, top_k, 0)
+        cfg = MoEConfig(d, E, f, top_k, flags)
         h = C.c_void_p()
         _check(self.lib, self.lib.moe_create(C.byref(cfg), C.byref(h)), "moe_create")
         self.h = h

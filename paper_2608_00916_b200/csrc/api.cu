@@ -29,6 +29,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.pad_offsets = take(sizeof(int32_t) * (s.E + 1));
   L.sched = take(sizeof(int32_t) * 4);
   L.tile_expert = take(sizeof(int32_t) * L.max_m_tiles);
+  L.pair_tab = take(sizeof(int32_t) * 4 * L.max_m_tiles);
   L.tile_counts = take(sizeof(int32_t) * (L.tok_tiles + 1) * s.E);
   L.psum_part = take(sizeof(float) * (L.router_blocks + 1) * s.E);
   L.psum = take(sizeof(float) * s.E);
@@ -107,6 +108,7 @@ moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
   if (!c) return MOE_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
   c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
+  c->single_cta = (cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 1 : 0;
   *out = reinterpret_cast<moe_ctx*>(c);
   return MOE_OK;
 }

@@ -31,8 +31,9 @@ struct WsLayout {
   size_t counts;       // int32[E]    rows per expert
   size_t offsets;      // int32[E+1]  exclusive scan of counts (canonical, unpadded)
   size_t pad_offsets;  // int32[E+1]  exclusive scan of counts rounded up to ROW_PAD
-  size_t sched;        // int32[4]    [0] number of 128-row tiles, [1] padded row total
+  size_t sched;        // int32[4]    [0] number of 128-row tiles, [1] padded row total, [2] number of block pairs
   size_t tile_expert;  // int32[max_m_tiles] expert of every 128-row tile
+  size_t pair_tab;     // int32[4 * max_m_tiles] pairs of 128-row blocks of one expert: {expert, first row, blocks, 0}
   size_t tile_counts;  // int32[tok_tiles * E] per token-tile histogram, turned into a prefix along tiles
   size_t psum_part;    // float[router_blocks * E] per-block column sums of p
   size_t psum;         // float[E]
@@ -65,6 +66,7 @@ struct moe_ctx_impl {
   int sm_count;
   int device;
   void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
+  int single_cta;   // 1: expert GEMMs on one-CTA tiles (128 x 256) instead of CTA pairs (256 x 256)
   int profiling;
   cudaEvent_t ev[MOE_PROF_RING][MOE_NUM_STAGES][2];
   unsigned char ev_used[MOE_PROF_RING][MOE_NUM_STAGES];
@@ -115,6 +117,8 @@ struct GemmIO {
 };
 moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
                                const GemmIO& io, cudaStream_t st);
+struct GemmParams;
+moe_status launch_pair_gemm(moe_ctx_impl* ctx, GemmKind kind, const GemmParams& p, cudaStream_t st);  // gemm2.cu
 // true when the tensor-core router / dW_r / dx kernels apply (their TMA maps need E % 8 == 0)
 inline bool router_on_tensor_cores(const Shape& s) { return s.E % 8 == 0; }
 // psum_part rows written by the router: one per warp of a 128-token tile (tensor cores) or per ROUTER_TOK tokens (SIMT)

@@ -20,176 +20,9 @@
 // straddles two experts and the ragged K of the weight gradients needs no masking.
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer (owns the TMEM allocation), warps 2..5 epilogue.
 // Every mbarrier wait is bounded; on a timeout the kernel records it in the status word and leaves.
-#include "common.cuh"
-#include "ptx.cuh"
+#include "gemm_common.cuh"
 
 namespace moe {
-
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;       // 16 KB
-constexpr int B_BYTES = BN * BK * 2;       // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-major tile: 8 KB
-constexpr int GEMM_THREADS = 192;
-constexpr int ACC_COLS = 256;
-constexpr int TMEM_COLS = 512;
-constexpr size_t GEMM_SMEM = static_cast<size_t>(STAGES) * STAGE_BYTES + 1024;
-
-struct GemmParams {
-  CUtensorMap mapA0, mapA1, mapB0, mapB1;
-  const int32_t* sched;        // [0] number of 128-row tiles
-  const int32_t* tile_expert;  // expert of each 128-row tile
-  const int32_t* pad_offsets;  // padded segment starts, E + 1 entries
-  int32_t* status;
-  int n_tiles;   // output tiles along N
-  int m_tiles;   // weight gradients: output tiles along M per expert
-  int E;
-  int k_blocks;  // row GEMMs: K blocks per segment
-  int M_total;   // weight gradients: rows of one expert's output
-  int N_total;   // columns of the output
-  uint16_t* out0;
-  uint16_t* out1;
-  uint16_t* out2;
-  const uint16_t* in0;
-  const uint16_t* in1;
-  int64_t ld_out;
-  int64_t expert_stride;
-  // router kinds
-  int static_m_tiles;   // RT, DX: number of 128-token tiles
-  int split_rows;       // DWR: tokens per slice (multiple of 64)
-  int rows_total;       // DWR: tokens rounded up to 64
-  int top_k;
-  int64_t T;
-  const float* bias;    // RT: [E] or null
-  float* logits;        // RT: [T,E] saved logits
-  float* logits_out;    // RT: optional copy for the caller
-  int32_t* idx;         // RT: [T,k] (workspace) and idx_out (caller)
-  int32_t* idx_out;
-  float* gates;
-  float* gates_out;
-  float* psum_part;     // RT: [4 * tiles, E] per-warp column sums of p
-  float* outf;          // DWR: [slices, d, E] fp32 partials
-};
-
-template <int KIND>
-struct Traits {
-  static constexpr bool WGRAD = (KIND == GEMM_B3 || KIND == GEMM_B5 || KIND == GEMM_DWR);
-  static constexpr bool STATIC_M = (KIND == GEMM_RT || KIND == GEMM_DX);  // token tiles, no expert lookup
-  static constexpr int A_MN = WGRAD ? 1 : 0;
-  static constexpr int B_MN = (KIND == GEMM_B2 || KIND == GEMM_B4 || KIND == GEMM_DX) ? 0 : 1;
-  static constexpr int NSEG = (KIND == GEMM_B4 || KIND == GEMM_DX) ? 2 : 1;
-  // width of output covered by one N tile (F3 / B5 / DWR pair a 128-wide tile with a second 128-wide operand)
-  static constexpr int N_SPAN = (KIND == GEMM_F3 || KIND == GEMM_B5 || KIND == GEMM_DWR) ? 128 : 256;
-};
-
-struct Tile {
-  int e, row0, m0, n0, nkb;
-};
-
-template <int KIND>
-__device__ __forceinline__ int total_tiles(const GemmParams& p) {
-  if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;
-  if (Traits<KIND>::STATIC_M) return p.static_m_tiles * p.n_tiles;
-  return p.sched[0] * p.n_tiles;
-}
-
-template <int KIND>
-__device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
-  Tile tl;
-  if (Traits<KIND>::WGRAD) {
-    const int per = p.m_tiles * p.n_tiles;
-    tl.e = t / per;
-    const int rem = t - tl.e * per;
-    tl.m0 = (rem / p.n_tiles) * BM;
-    tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
-    if (KIND == GEMM_DWR) {  // "expert" = token slice
-      tl.row0 = tl.e * p.split_rows;
-      tl.nkb = max(0, min(p.split_rows, p.rows_total - tl.row0)) / BK;
-    } else {
-      tl.row0 = p.pad_offsets[tl.e];
-      tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
-    }
-  } else if (Traits<KIND>::STATIC_M) {
-    const int mt = t / p.n_tiles;
-    tl.e = 0;
-    tl.row0 = mt * BM;
-    tl.m0 = 0;
-    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
-    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
-  } else {
-    const int mt = t / p.n_tiles;
-    tl.e = p.tile_expert[mt];
-    tl.row0 = mt * BM;
-    tl.m0 = 0;
-    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
-    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
-  }
-  return tl;
-}
-
-template <int KIND>
-__device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl, int kb, uint32_t sA, uint32_t sB,
-                                            uint32_t bar) {
-  if (KIND == GEMM_F3) {
-    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
-      tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
-    }
-  } else if (KIND == GEMM_F4 || KIND == GEMM_RT) {
-    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
-  } else if (KIND == GEMM_B2) {
-    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-    tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
-  } else if (KIND == GEMM_B4 || KIND == GEMM_DX) {
-    const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
-    tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
-    tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
-  } else if (KIND == GEMM_B3) {
-    const int row = tl.row0 + kb * BK;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
-  } else {  // GEMM_B5, GEMM_DWR
-    const int row = tl.row0 + kb * BK;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
-      tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
-      tma_load_2d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, row);
-    }
-  }
-}
-
-__device__ __forceinline__ void store_bf16x32(uint16_t* dst, const float (&v)[32]) {
-  uint4* q = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint4 w;
-    w.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);
-    w.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
-    w.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
-    w.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
-    q[i] = w;
-  }
-}
-__device__ __forceinline__ void load_bf16x32(const uint16_t* src, float (&v)[32]) {
-  const uint4* q = reinterpret_cast<const uint4*>(src);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint4 w = q[i];
-    unpack_bf16x2(w.x, v[8 * i + 0], v[8 * i + 1]);
-    unpack_bf16x2(w.y, v[8 * i + 2], v[8 * i + 3]);
-    unpack_bf16x2(w.z, v[8 * i + 4], v[8 * i + 5]);
-    unpack_bf16x2(w.w, v[8 * i + 6], v[8 * i + 7]);
-  }
-}
-__device__ __forceinline__ float fast_sigmoid(float h) { return __fdividef(1.f, 1.f + __expf(-h)); }
 
 template <int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __grid_constant__ GemmParams p) {
@@ -321,22 +154,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
               *reinterpret_cast<float4*>(p.outf + (static_cast<int64_t>(tl.e) * p.M_total + m) * p.N_total + col) =
                   make_float4(0.f, 0.f, 0.f, 0.f);
         } else if (TR::WGRAD) {
-          const int m = tl.m0 + rin;
-          if (m < p.M_total) {
-            float z[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) z[i] = 0.f;
-            for (int c = 0; c < 8; ++c) {
-              uint16_t* base = p.out0;
-              int col = tl.n0 + c * 32;
-              if (KIND == GEMM_B5) {
-                base = (c >= 4) ? p.out1 : p.out0;
-                col = tl.n0 + (c & 3) * 32;
-              }
-              if (col < p.N_total)
-                store_bf16x32(base + tl.e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, z);
-            }
-          }
+          wgrad_zero_fill<KIND>(p, tl.e, tl.m0 + rin, tl.n0);
         }
         continue;
       }
@@ -350,51 +168,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + acc * ACC_COLS;
       const int64_t row = static_cast<int64_t>(tl.row0) + rin;
-      if (KIND == GEMM_F3) {
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t rg[32], ru[32];
-          tmem_ld32(taddr + c * 32, rg);
-          tmem_ld32(taddr + 128 + c * 32, ru);
-          tmem_ld_wait();
-          const int col = tl.n0 + c * 32;
-          if (col < p.N_total) {
-            float hg[32], hu[32], a[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              hg[i] = __uint_as_float(rg[i]);
-              hu[i] = __uint_as_float(ru[i]);
-              a[i] = hg[i] * fast_sigmoid(hg[i]) * hu[i];
-            }
-            const int64_t off = row * p.ld_out + col;
-            store_bf16x32(p.out0 + off, hg);
-            store_bf16x32(p.out1 + off, hu);
-            store_bf16x32(p.out2 + off, a);
-          }
-        }
-      } else if (KIND == GEMM_B2) {
-#pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-          uint32_t rd[32];
-          tmem_ld32(taddr + c * 32, rd);
-          tmem_ld_wait();
-          const int col = tl.n0 + c * 32;
-          if (col < p.N_total) {
-            const int64_t off = row * p.ld_out + col;
-            float hg[32], hu[32], dhg[32], dhu[32];
-            load_bf16x32(p.in0 + off, hg);
-            load_bf16x32(p.in1 + off, hu);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float da = __uint_as_float(rd[i]);
-              const float sg = fast_sigmoid(hg[i]);
-              dhg[i] = da * hu[i] * sg * (1.f + hg[i] * (1.f - sg));
-              dhu[i] = da * hg[i] * sg;
-            }
-            store_bf16x32(p.out0 + off, dhg);
-            store_bf16x32(p.out1 + off, dhu);
-          }
-        }
+      if (KIND == GEMM_F3 || KIND == GEMM_B2) {
+        expert_epilogue<KIND>(p, tl.e, row, tl.m0 + rin, tl.n0, taddr, true);
       } else if (KIND == GEMM_RT) {
         // Routing epilogue: one thread per token; the row of E logits is re-read from tensor memory in every
         // pass.  Pass j picks the largest logit that comes after pick j-1 in the order (value descending,
@@ -512,31 +287,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
           }
         }
       } else {
-        // plain bf16 store: F4, B4 (row GEMMs), B3, B5 (weight gradients)
-#pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
-          uint32_t rd[32];
-          tmem_ld32(taddr + c * 32, rd);
-          tmem_ld_wait();
-          float v[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rd[i]);
-          if (TR::WGRAD) {
-            const int m = tl.m0 + rin;
-            uint16_t* base = p.out0;
-            int col = tl.n0 + c * 32;
-            if (KIND == GEMM_B5) {
-              base = (c >= 4) ? p.out1 : p.out0;
-              col = tl.n0 + (c & 3) * 32;
-            }
-            if (m < p.M_total && col < p.N_total)
-              store_bf16x32(base + tl.e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, v);
-          } else {
-            const int col = tl.n0 + c * 32;
-            const bool in_rows = (KIND != GEMM_DX) || row < p.T;  // token tiles may overhang T
-            if (in_rows && col < p.N_total) store_bf16x32(p.out0 + row * p.ld_out + col, v);
-          }
-        }
+        expert_epilogue<KIND>(p, tl.e, row, tl.m0 + rin, tl.n0, taddr, true);
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
@@ -618,6 +369,8 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.sched = reinterpret_cast<const int32_t*>(ws + L.sched);
   p.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
   p.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+  p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
+  const bool pair = !ctx->single_cta;  // expert GEMMs on CTA pairs (256 x 256 tiles)
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
   bool ok = true;
@@ -632,7 +385,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.out0 = hg; p.out1 = hu; p.out2 = act;
       p.ld_out = f;
       if (!ok) return MOE_ERR_CUDA;
-      return launch_kind<GEMM_F3>(ctx, p, st);
+      return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_F3>(ctx, p, st);
     case GEMM_F4:
       ok = map_2d(fn, &p.mapA0, act, R, f, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, 64);
       p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
@@ -642,9 +395,9 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.out0 = o;
       p.ld_out = d;
       if (!ok) return MOE_ERR_CUDA;
-      return launch_kind<GEMM_F4>(ctx, p, st);
+      return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_F4>(ctx, p, st);
     case GEMM_B2:
-      ok = map_2d(fn, &p.mapA0, o, R, d, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, 256);
+      ok = map_2d(fn, &p.mapA0, o, R, d, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, pair ? 128 : 256);
       p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
       p.n_tiles = (f + 255) / 256;
       p.k_blocks = d / BK;
@@ -653,21 +406,22 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.out0 = dhg; p.out1 = dhu;
       p.ld_out = f;
       if (!ok) return MOE_ERR_CUDA;
-      return launch_kind<GEMM_B2>(ctx, p, st);
+      return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B2>(ctx, p, st);
     case GEMM_B4:
       ok = map_2d(fn, &p.mapA0, dhg, R, f, 128) && map_2d(fn, &p.mapA1, dhu, R, f, 128) &&
-           map_3d(fn, &p.mapB0, W_gate, E, d, f, 256) && map_3d(fn, &p.mapB1, W_up, E, d, f, 256);
+           map_3d(fn, &p.mapB0, W_gate, E, d, f, pair ? 128 : 256) &&
+           map_3d(fn, &p.mapB1, W_up, E, d, f, pair ? 128 : 256);
       p.n_tiles = (d + 255) / 256;
       p.k_blocks = f / BK;
       p.N_total = d;
       p.out0 = dxp;
       p.ld_out = d;
       if (!ok) return MOE_ERR_CUDA;
-      return launch_kind<GEMM_B4>(ctx, p, st);
+      return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B4>(ctx, p, st);
     case GEMM_B3:
       ok = map_2d(fn, &p.mapA0, act, R, f, 64) && map_2d(fn, &p.mapB0, o, R, d, 64);
       p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
-      p.m_tiles = (f + 127) / 128;
+      p.m_tiles = pair ? (f + 255) / 256 : (f + 127) / 128;
       p.n_tiles = (d + 255) / 256;
       p.M_total = f;
       p.N_total = d;
@@ -675,12 +429,12 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.ld_out = d;
       p.expert_stride = static_cast<int64_t>(f) * d;
       if (!ok) return MOE_ERR_CUDA;
-      return launch_kind<GEMM_B3>(ctx, p, st);
+      return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B3>(ctx, p, st);
     case GEMM_B5:
       ok = map_2d(fn, &p.mapA0, xp, R, d, 64) && map_2d(fn, &p.mapB0, dhg, R, f, 64) &&
            map_2d(fn, &p.mapB1, dhu, R, f, 64);
       p.mapA1 = p.mapA0;
-      p.m_tiles = (d + 127) / 128;
+      p.m_tiles = pair ? (d + 255) / 256 : (d + 127) / 128;
       p.n_tiles = (f + 127) / 128;
       p.M_total = d;
       p.N_total = f;
@@ -688,7 +442,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.ld_out = f;
       p.expert_stride = static_cast<int64_t>(d) * f;
       if (!ok) return MOE_ERR_CUDA;
-      return launch_kind<GEMM_B5>(ctx, p, st);
+      return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B5>(ctx, p, st);
     case GEMM_RT:
       // logits[T,E] = x[T,d] W_r[d,E]; W_r is read as a one-slab 3D tensor so the weight loaders apply
       ok = map_2d(fn, &p.mapA0, io.x, T, d, 128) && map_3d(fn, &p.mapB0, io.W_r, 1, d, E, 64);

@@ -1,0 +1,289 @@
+// The six expert contractions on CTA pairs (cluster of 2, tcgen05 cta_group::2).
+//
+// Why pairs: with one CTA per 128 x 256 tile every SM stages 48 KB of operands per 64-deep K step, and the profile
+// of that kernel shows the tensor pipe about half busy with no memory unit saturated - the four-stage ring cannot
+// keep enough bytes in flight.  A pair computes a 256 x 256 tile: each CTA stages its own 128 rows of A and only
+// HALF of B (128 of the 256 columns); the MMA reads both halves from the two CTAs' shared memories.  Per SM that is
+// 32 KB per K step for the same MMA time, and the ring grows to six stages.
+//
+// Protocol (leader = cluster rank 0).  Both producers issue their own TMA loads, all credited to the LEADER's full
+// barrier (the leader's producer posts the expected byte count of both CTAs).  The leader's MMA thread issues
+// tcgen05.mma.cta_group::2 and commits to the empty / accumulator-full barriers of BOTH CTAs.  The epilogue warps of
+// both CTAs drain their own tensor memory (their 128 rows) and arrive on the leader's accumulator-empty barrier.
+// Tensor memory is allocated and freed by one warp of each CTA; cluster barriers bracket the kernel so that no CTA
+// leaves while its partner may still touch its shared memory, barriers or tensor memory.
+//
+// Row GEMMs pair two consecutive 128-row blocks of ONE expert; an expert with an odd number of blocks gets a pair
+// whose second half is a dummy (it loads whatever follows and stores nothing).  Weight gradients pair along M.
+#include "gemm_common.cuh"
+
+namespace moe {
+
+constexpr int STAGES2 = 6;
+constexpr int BH_BYTES = 128 * BK * 2;              // this CTA's half of B: 16 KB
+constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;    // 32 KB
+constexpr size_t GEMM2_SMEM = static_cast<size_t>(STAGES2) * STAGE2_BYTES + 1024;
+
+struct Tile2 {
+  int e, row0, m0, n0, nkb;
+  bool write;
+};
+
+template <int KIND>
+__device__ __forceinline__ int total_tiles2(const GemmParams& p) {
+  if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;  // m_tiles = 256-row pairs of the output
+  return p.sched[2] * p.n_tiles;                                // sched[2] = number of row-block pairs
+}
+
+template <int KIND>
+__device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank) {
+  Tile2 tl;
+  if (Traits<KIND>::WGRAD) {
+    const int per = p.m_tiles * p.n_tiles;
+    tl.e = t / per;
+    const int rem = t - tl.e * per;
+    tl.m0 = (rem / p.n_tiles) * 2 * BM + rank * BM;
+    tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.row0 = p.pad_offsets[tl.e];
+    tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
+    tl.write = true;
+  } else {
+    const int pr = t / p.n_tiles;
+    const int4 info = *reinterpret_cast<const int4*>(p.pair_tab + 4 * pr);  // expert, first row, blocks (1 or 2)
+    tl.e = info.x;
+    tl.row0 = info.y + rank * BM;
+    tl.write = rank < info.z;
+    tl.m0 = 0;
+    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
+  }
+  return tl;
+}
+
+// Loads of one K block for the CTA of rank `rank`: its rows of A and its 128-column half of B.
+template <int KIND>
+__device__ __forceinline__ void issue_loads2(const GemmParams& p, const Tile2& tl, int kb, int rank, uint32_t sA,
+                                             uint32_t sB, uint32_t bar) {
+  if (KIND == GEMM_F3) {
+    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    const CUtensorMap* mb = rank ? &p.mapB1 : &p.mapB0;  // leader: gate columns, partner: the matching up columns
+#pragma unroll
+    for (int c = 0; c < 2; ++c) tma_load_3d_pair(sB + c * CHUNK_BYTES, mb, bar, tl.n0 + c * 64, kb * BK, tl.e);
+  } else if (KIND == GEMM_F4) {
+    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+      tma_load_3d_pair(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + rank * 128 + c * 64, kb * BK, tl.e);
+  } else if (KIND == GEMM_B2) {
+    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    tma_load_3d_pair(sB, &p.mapB0, bar, kb * BK, tl.n0 + rank * 128, tl.e);
+  } else if (KIND == GEMM_B4) {
+    const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
+    tma_load_2d_pair(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
+    tma_load_3d_pair(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0 + rank * 128, tl.e);
+  } else if (KIND == GEMM_B3) {
+    const int row = tl.row0 + kb * BK;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tma_load_2d_pair(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+      tma_load_2d_pair(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + rank * 128 + c * 64, row);
+    }
+  } else {  // GEMM_B5
+    const int row = tl.row0 + kb * BK;
+    const CUtensorMap* mb = rank ? &p.mapB1 : &p.mapB0;  // leader: dhg columns, partner: dhu columns
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tma_load_2d_pair(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+      tma_load_2d_pair(sB + c * CHUNK_BYTES, mb, bar, tl.n0 + c * 64, row);
+    }
+  }
+}
+
+template <int KIND>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+    grouped_gemm_pair_kernel(const __grid_constant__ GemmParams p) {
+  using TR = Traits<KIND>;
+  extern __shared__ unsigned char gemm2_smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES2 + 4];
+  __shared__ uint32_t tmem_base_slot;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = static_cast<int>(cluster_ctarank());
+  const bool leader = rank == 0;
+  const uint32_t smem_base = (smem_u32(gemm2_smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES2 + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES2; ++s) {
+      mbar_init(full_bar(s), 1);   // used in the leader only: its producer's arrive + the bytes of both CTAs
+      mbar_init(empty_bar(s), 1);  // one commit from the leader's MMA thread
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);   // one commit from the leader's MMA thread
+      mbar_init(tempty_bar(a), 8);  // used in the leader only: 4 epilogue warps of each CTA
+    }
+    fence_mbar_init();
+    tma_prefetch_desc(&p.mapA0);
+    tma_prefetch_desc(&p.mapB0);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&tmem_base_slot), TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals across the pair
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const int ntiles = total_tiles2<KIND>(p);
+  const int cid = blockIdx.x >> 1, nclusters = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = cid; t < ntiles && ok; t += nclusters) {
+      const Tile2 tl = get_tile2<KIND>(p, t, rank);
+      for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
+        const int s = it % STAGES2;
+        const uint32_t ph = (it / STAGES2) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u)) {
+          ok = false;
+          break;
+        }
+        if (lane == 0) {
+          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
+          const uint32_t sA = smem_base + s * STAGE2_BYTES;
+          issue_loads2<KIND>(p, tl, kb, rank, sA, sA + A_BYTES, mapa_shared(full_bar(s), 0));
+        }
+        __syncwarp();
+      }
+    }
+    if (!ok && lane == 0) {
+      atomicExch(p.status, DEV_TIMEOUT);
+      p.status[1] = 1100 + KIND;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (leader) {
+      constexpr uint32_t idesc = umma_idesc(2 * BM, BN, TR::A_MN, TR::B_MN);
+      constexpr uint32_t A_LBO = TR::A_MN ? CHUNK_BYTES : 0, B_LBO = TR::B_MN ? CHUNK_BYTES : 0;
+      constexpr uint32_t A_KSTEP = TR::A_MN ? 2048 : 32, B_KSTEP = TR::B_MN ? 2048 : 32;
+      uint32_t it = 0, tc = 0;
+      bool ok = true;
+      for (int t = cid; t < ntiles && ok; t += nclusters) {
+        const Tile2 tl = get_tile2<KIND>(p, t, rank);
+        if (tl.nkb == 0) continue;
+        const int acc = tc & 1;
+        const uint32_t aph = (tc >> 1) & 1u;
+        ++tc;
+        if (!mbar_wait(tempty_bar(acc), aph ^ 1u)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
+        for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
+          const int s = it % STAGES2;
+          const uint32_t ph = (it / STAGES2) & 1u;
+          if (!mbar_wait(full_bar(s), ph)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          if (lane == 0) {
+            const uint32_t sA = smem_base + s * STAGE2_BYTES;
+            const uint32_t sB = sA + A_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < BK / 16; ++ks) {
+              const uint64_t da = smem_desc(sA + ks * A_KSTEP, A_LBO, 1024);
+              const uint64_t db = smem_desc(sB + ks * B_KSTEP, B_LBO, 1024);
+              umma_bf16_pair(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+            }
+            // the stage is free in both CTAs once these MMAs have read it
+            umma_commit_pair(mapa_shared(empty_bar(s), 0));
+            umma_commit_pair(mapa_shared(empty_bar(s), 1));
+          }
+          __syncwarp();
+        }
+        if (ok && lane == 0) {
+          umma_commit_pair(mapa_shared(tfull_bar(acc), 0));
+          umma_commit_pair(mapa_shared(tfull_bar(acc), 1));
+        }
+        __syncwarp();
+      }
+      if (!ok && lane == 0) {
+        atomicExch(p.status, DEV_TIMEOUT);
+        p.status[1] = 1200 + KIND;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps per CTA, own 128 rows)
+    const int ew = warp & 3;
+    uint32_t tc = 0;
+    bool ok = true;
+    for (int t = cid; t < ntiles && ok; t += nclusters) {
+      const Tile2 tl = get_tile2<KIND>(p, t, rank);
+      const int rin = ew * 32 + lane;
+      if (tl.nkb == 0) {
+        if (TR::WGRAD) wgrad_zero_fill<KIND>(p, tl.e, tl.m0 + rin, tl.n0);
+        continue;
+      }
+      const int acc = tc & 1;
+      const uint32_t aph = (tc >> 1) & 1u;
+      ++tc;
+      if (!mbar_wait(tfull_bar(acc), aph)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + acc * ACC_COLS;
+      expert_epilogue<KIND>(p, tl.e, static_cast<int64_t>(tl.row0) + rin, tl.m0 + rin, tl.n0, taddr, tl.write);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
+    }
+    if (!ok && lane == 0) {
+      atomicExch(p.status, DEV_TIMEOUT);
+      p.status[1] = 1300 + KIND;
+    }
+  }
+
+  tc_fence_before();
+  cluster_sync_all();  // the partner has stopped using this CTA's shared memory, barriers and tensor memory
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int KIND>
+static moe_status launch_pair_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream_t st) {
+  static bool attr_done[GEMM_KINDS] = {false};
+  if (!attr_done[KIND]) {
+    if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(GEMM2_SMEM)) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done[KIND] = true;
+  }
+  const int grid = ctx->sm_count & ~1;  // whole pairs
+  grouped_gemm_pair_kernel<KIND><<<grid, GEMM_THREADS, GEMM2_SMEM, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status launch_pair_gemm(moe_ctx_impl* ctx, GemmKind kind, const GemmParams& p, cudaStream_t st) {
+  switch (kind) {
+    case GEMM_F3: return launch_pair_kind<GEMM_F3>(ctx, p, st);
+    case GEMM_F4: return launch_pair_kind<GEMM_F4>(ctx, p, st);
+    case GEMM_B2: return launch_pair_kind<GEMM_B2>(ctx, p, st);
+    case GEMM_B3: return launch_pair_kind<GEMM_B3>(ctx, p, st);
+    case GEMM_B4: return launch_pair_kind<GEMM_B4>(ctx, p, st);
+    case GEMM_B5: return launch_pair_kind<GEMM_B5>(ctx, p, st);
+    default: return MOE_ERR_INVALID_ARG;
+  }
+}
+
+}  // namespace moe

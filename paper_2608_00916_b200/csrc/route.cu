@@ -234,11 +234,13 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
                                                             int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                                                             int32_t* __restrict__ pad_offsets,
                                                             int32_t* __restrict__ sched, int32_t* __restrict__ tile_expert,
+                                                            int32_t* __restrict__ pair_tab,
                                                             const float* __restrict__ psum_part,
                                                             float* __restrict__ psum, int32_t* __restrict__ counts_out,
                                                             float* __restrict__ aux_out, int32_t* __restrict__ status) {
   __shared__ int s_cnt[MAX_E];
   __shared__ int s_pad[MAX_E + 1];
+  __shared__ int s_pair[MAX_E + 1];
   __shared__ float s_term[MAX_E];
   __shared__ float s_ps[SCAN_THREADS];
   const int tid = threadIdx.x;
@@ -273,26 +275,36 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
   }
   __syncthreads();
   if (tid == 0) {
-    int off = 0, poff = 0;
+    int off = 0, poff = 0, npair = 0;
     float aux = 0.f;
     for (int e = 0; e < E; ++e) {
       offsets[e] = off;
       pad_offsets[e] = poff;
       s_pad[e] = poff;
+      s_pair[e] = npair;
+      const int blocks = (s_cnt[e] + ROW_PAD - 1) / ROW_PAD;
       off += s_cnt[e];
-      poff += (s_cnt[e] + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
+      poff += blocks * ROW_PAD;
+      npair += (blocks + 1) / 2;
       aux += s_term[e];
     }
     offsets[E] = off;
     pad_offsets[E] = poff;
     s_pad[E] = poff;
+    s_pair[E] = npair;
     sched[0] = poff / ROW_PAD;
     sched[1] = poff;
+    sched[2] = npair;
     aux_out[0] = aux * static_cast<float>(E);
   }
   __syncthreads();
   for (int e = tid; e < E; e += SCAN_THREADS) {
     for (int m = s_pad[e] / ROW_PAD; m < s_pad[e + 1] / ROW_PAD; ++m) tile_expert[m] = e;
+    // pairs of consecutive 128-row blocks of this expert; the last pair of an odd count has one block
+    const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_PAD;
+    for (int q = 0; q < s_pair[e + 1] - s_pair[e]; ++q)
+      *reinterpret_cast<int4*>(pair_tab + 4 * (s_pair[e] + q)) =
+          make_int4(e, s_pad[e] + 2 * q * ROW_PAD, min(2, blocks - 2 * q), 0);
   }
 }
 
@@ -353,6 +365,7 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
                                  reinterpret_cast<int32_t*>(ws + L.pad_offsets),
                                  reinterpret_cast<int32_t*>(ws + L.sched),
                                  reinterpret_cast<int32_t*>(ws + L.tile_expert),
+                                 reinterpret_cast<int32_t*>(ws + L.pair_tab),
                                  reinterpret_cast<const float*>(ws + L.psum_part),
                                  reinterpret_cast<float*>(ws + L.psum), counts_out, aux_out,
                                  reinterpret_cast<int32_t*>(ws + L.status));
