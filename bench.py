@@ -306,7 +306,7 @@ def main():
 
     cpu = None
     if not args.no_cpu_baseline:
-        sample_T = min(T, 4096)
+        sample_T = min(T, 16384)
         v, dt = oracle_sample_tokens_per_s(inp, shape, sample_T)
         cpu = {"value": v, "unit": "tokens/s", "cores": host_cores(), "kind": "oracle", "seconds": dt,
                "sample": f"first {sample_T} tokens of the batch through the fp32 numpy oracle, forward + backward, "

@@ -24,6 +24,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
     return o;
   };
   L.status = take(sizeof(int32_t) * 16);
+  L.timers = take(sizeof(long long) * 16 * 8);
   L.counts = take(sizeof(int32_t) * s.E);
   L.offsets = take(sizeof(int32_t) * (s.E + 1));
   L.pad_offsets = take(sizeof(int32_t) * (s.E + 1));
@@ -108,7 +109,7 @@ moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
   if (!c) return MOE_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
   c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
-  c->single_cta = (cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 1 : 0;
+  c->single_cta = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 0 : 1;
   *out = reinterpret_cast<moe_ctx*>(c);
   return MOE_OK;
 }
@@ -160,7 +161,8 @@ moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char* name, s
              {"dxr", L.dxr, sizeof(uint16_t) * T * s.d},
              {"dg", L.dg, sizeof(float) * R},
              {"dl", L.dl, sizeof(float) * T * s.E},
-             {"status", L.status, sizeof(int32_t) * 16}};
+             {"status", L.status, sizeof(int32_t) * 16},
+             {"timers", L.timers, sizeof(long long) * 16 * 8}};
   for (const Ent& e : tab)
     if (strcmp(e.n, name) == 0) {
       *offset = e.off;

@@ -28,6 +28,7 @@ struct Shape {
 // Byte offsets of every internal buffer inside the caller's workspace (all 256-byte aligned).
 struct WsLayout {
   size_t status;       // int32[16]   [0] device status, [1] where it happened
+  size_t timers;       // int64[GEMM_KINDS][8] cycle counters of the GEMM roles (filled only when MOE_GEMM_TIMERS is set)
   size_t counts;       // int32[E]    rows per expert
   size_t offsets;      // int32[E+1]  exclusive scan of counts (canonical, unpadded)
   size_t pad_offsets;  // int32[E+1]  exclusive scan of counts rounded up to ROW_PAD

@@ -20,6 +20,8 @@
 // straddles two experts and the ragged K of the weight gradients needs no masking.
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer (owns the TMEM allocation), warps 2..5 epilogue.
 // Every mbarrier wait is bounded; on a timeout the kernel records it in the status word and leaves.
+#include <stdlib.h>
+
 #include "gemm_common.cuh"
 
 namespace moe {
@@ -69,15 +71,18 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     // ------------------------------------------------------------------ TMA producer
     uint32_t it = 0;
     bool ok = true;
+    long long t_wait = 0, t_begin = clock64();
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
       const Tile tl = get_tile<KIND>(p, t);
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
+        const long long w0 = clock64();
         if (!mbar_wait(empty_bar(s), ph ^ 1u)) {
           ok = false;
           break;
         }
+        t_wait += clock64() - w0;
         if (lane == 0) {
           mbar_expect_tx(full_bar(s), STAGE_BYTES);
           const uint32_t sA = smem_base + s * STAGE_BYTES;
@@ -85,6 +90,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
         }
         __syncwarp();
       }
+    }
+    if (p.timers && lane == 0) {
+      atomicAdd(p.timers + 0, static_cast<unsigned long long>(clock64() - t_begin));  // producer: total
+      atomicAdd(p.timers + 1, static_cast<unsigned long long>(t_wait));               // producer: waiting for a free stage
     }
     if (!ok && lane == 0) {
       atomicExch(p.status, DEV_TIMEOUT);
@@ -97,25 +106,30 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     constexpr uint32_t A_KSTEP = TR::A_MN ? 2048 : 32, B_KSTEP = TR::B_MN ? 2048 : 32;  // bytes per K = 16
     uint32_t it = 0, tc = 0;
     bool ok = true;
+    long long t_acc = 0, t_full = 0, t_begin = clock64();
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
       const Tile tl = get_tile<KIND>(p, t);
       if (tl.nkb == 0) continue;
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
+      const long long w0 = clock64();
       if (!mbar_wait(tempty_bar(acc), aph ^ 1u)) {
         ok = false;
         break;
       }
+      t_acc += clock64() - w0;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
+        const long long w1 = clock64();
         if (!mbar_wait(full_bar(s), ph)) {
           ok = false;
           break;
         }
+        t_full += clock64() - w1;
         tc_fence_after();
         if (lane == 0) {
           const uint32_t sA = smem_base + s * STAGE_BYTES;
@@ -133,6 +147,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       if (ok && lane == 0) umma_commit(tfull_bar(acc));
       __syncwarp();
     }
+    if (p.timers && lane == 0) {
+      atomicAdd(p.timers + 2, static_cast<unsigned long long>(clock64() - t_begin));  // MMA issuer: total
+      atomicAdd(p.timers + 3, static_cast<unsigned long long>(t_acc));                // waiting for a drained accumulator
+      atomicAdd(p.timers + 4, static_cast<unsigned long long>(t_full));               // waiting for operands
+    }
     if (!ok && lane == 0) {
       atomicExch(p.status, DEV_TIMEOUT);
       p.status[1] = 200 + KIND;
@@ -140,8 +159,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps, 128 TMEM lanes)
     const int ew = warp & 3;  // TMEM lane quadrant this warp may read
+    EpiStage es{smem_base + STAGES * STAGE_BYTES + ew * (EPI_UNITS * EPI_UNIT_BYTES), 0u};
     uint32_t tc = 0;
     bool ok = true;
+    long long t_idle = 0, t_begin = clock64();
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
       const Tile tl = get_tile<KIND>(p, t);
       const int rin = ew * 32 + lane;  // row inside the tile
@@ -161,15 +182,19 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
+      const long long w0 = clock64();
       if (!mbar_wait(tfull_bar(acc), aph)) {
         ok = false;
         break;
       }
+      t_idle += clock64() - w0;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + acc * ACC_COLS;
       const int64_t row = static_cast<int64_t>(tl.row0) + rin;
       if (KIND == GEMM_F3 || KIND == GEMM_B2) {
-        expert_epilogue<KIND>(p, tl.e, row, tl.m0 + rin, tl.n0, taddr, true);
+        expert_epilogue<KIND>(p, tl.e, row, (TR::WGRAD ? tl.m0 : tl.row0) + ew * 32, tl.n0, taddr, true,
+                              TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
+                              es, lane);
       } else if (KIND == GEMM_RT) {
         // Routing epilogue: one thread per token; the row of E logits is re-read from tensor memory in every
         // pass.  Pass j picks the largest logit that comes after pick j-1 in the order (value descending,
@@ -287,10 +312,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
           }
         }
       } else {
-        expert_epilogue<KIND>(p, tl.e, row, tl.m0 + rin, tl.n0, taddr, true);
+        expert_epilogue<KIND>(p, tl.e, row, (TR::WGRAD ? tl.m0 : tl.row0) + ew * 32, tl.n0, taddr, true,
+                              TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
+                              es, lane);
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
+    }
+    if (p.timers && lane == 0 && ew == 0) {
+      atomicAdd(p.timers + 5, static_cast<unsigned long long>(clock64() - t_begin));  // epilogue warp: total
+      atomicAdd(p.timers + 6, static_cast<unsigned long long>(t_idle));               // waiting for a finished accumulator
+      atomicAdd(p.timers + 7, 1ull);                                                  // CTAs counted
     }
     if (!ok && lane == 0) {
       atomicExch(p.status, DEV_TIMEOUT);
@@ -370,6 +402,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
   p.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
   p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
+  p.timers = getenv("MOE_GEMM_TIMERS") ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
   const bool pair = !ctx->single_cta;  // expert GEMMs on CTA pairs (256 x 256 tiles)
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;

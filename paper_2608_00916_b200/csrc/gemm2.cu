@@ -20,9 +20,10 @@
 namespace moe {
 
 constexpr int STAGES2 = 6;
+constexpr int GEMM2_THREADS = GEMM_THREADS;
 constexpr int BH_BYTES = 128 * BK * 2;              // this CTA's half of B: 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;    // 32 KB
-constexpr size_t GEMM2_SMEM = static_cast<size_t>(STAGES2) * STAGE2_BYTES + 1024;
+constexpr size_t GEMM2_SMEM = static_cast<size_t>(STAGES2) * STAGE2_BYTES + EPI_BYTES + 1024;
 
 struct Tile2 {
   int e, row0, m0, n0, nkb;
@@ -100,7 +101,7 @@ __device__ __forceinline__ void issue_loads2(const GemmParams& p, const Tile2& t
 }
 
 template <int KIND>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
     grouped_gemm_pair_kernel(const __grid_constant__ GemmParams p) {
   using TR = Traits<KIND>;
   extern __shared__ unsigned char gemm2_smem_raw[];
@@ -145,15 +146,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     uint32_t it = 0;
     bool ok = true;
+    long long t_wait = 0, t_begin = clock64();
     for (int t = cid; t < ntiles && ok; t += nclusters) {
       const Tile2 tl = get_tile2<KIND>(p, t, rank);
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
         const int s = it % STAGES2;
         const uint32_t ph = (it / STAGES2) & 1u;
+        const long long w0 = clock64();
         if (!mbar_wait(empty_bar(s), ph ^ 1u)) {
           ok = false;
           break;
         }
+        t_wait += clock64() - w0;
         if (lane == 0) {
           if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
           const uint32_t sA = smem_base + s * STAGE2_BYTES;
@@ -161,6 +165,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
         }
         __syncwarp();
       }
+    }
+    if (p.timers && lane == 0 && leader) {
+      atomicAdd(p.timers + 0, static_cast<unsigned long long>(clock64() - t_begin));
+      atomicAdd(p.timers + 1, static_cast<unsigned long long>(t_wait));
     }
     if (!ok && lane == 0) {
       atomicExch(p.status, DEV_TIMEOUT);
@@ -174,25 +182,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
       constexpr uint32_t A_KSTEP = TR::A_MN ? 2048 : 32, B_KSTEP = TR::B_MN ? 2048 : 32;
       uint32_t it = 0, tc = 0;
       bool ok = true;
+      long long t_acc = 0, t_full = 0, t_begin = clock64();
       for (int t = cid; t < ntiles && ok; t += nclusters) {
         const Tile2 tl = get_tile2<KIND>(p, t, rank);
         if (tl.nkb == 0) continue;
         const int acc = tc & 1;
         const uint32_t aph = (tc >> 1) & 1u;
         ++tc;
+        const long long w0 = clock64();
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u)) {
           ok = false;
           break;
         }
+        t_acc += clock64() - w0;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
         for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
           const int s = it % STAGES2;
           const uint32_t ph = (it / STAGES2) & 1u;
+          const long long w1 = clock64();
           if (!mbar_wait(full_bar(s), ph)) {
             ok = false;
             break;
           }
+          t_full += clock64() - w1;
           tc_fence_after();
           if (lane == 0) {
             const uint32_t sA = smem_base + s * STAGE2_BYTES;
@@ -215,6 +228,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
         }
         __syncwarp();
       }
+      if (p.timers && lane == 0) {
+        atomicAdd(p.timers + 2, static_cast<unsigned long long>(clock64() - t_begin));
+        atomicAdd(p.timers + 3, static_cast<unsigned long long>(t_acc));
+        atomicAdd(p.timers + 4, static_cast<unsigned long long>(t_full));
+      }
       if (!ok && lane == 0) {
         atomicExch(p.status, DEV_TIMEOUT);
         p.status[1] = 1200 + KIND;
@@ -223,8 +241,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps per CTA, own 128 rows)
     const int ew = warp & 3;
+    EpiStage es{smem_base + STAGES2 * STAGE2_BYTES + ew * (EPI_UNITS * EPI_UNIT_BYTES), 0u};
     uint32_t tc = 0;
     bool ok = true;
+    long long t_idle = 0, t_begin = clock64();
     for (int t = cid; t < ntiles && ok; t += nclusters) {
       const Tile2 tl = get_tile2<KIND>(p, t, rank);
       const int rin = ew * 32 + lane;
@@ -235,16 +255,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
+      const long long w0 = clock64();
       if (!mbar_wait(tfull_bar(acc), aph)) {
         ok = false;
         break;
       }
+      t_idle += clock64() - w0;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + acc * ACC_COLS;
-      expert_epilogue<KIND>(p, tl.e, static_cast<int64_t>(tl.row0) + rin, tl.m0 + rin, tl.n0, taddr, tl.write);
+      expert_epilogue<KIND>(p, tl.e, static_cast<int64_t>(tl.row0) + rin, (TR::WGRAD ? tl.m0 : tl.row0) + ew * 32, tl.n0, taddr,
+                            tl.write, TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : 32, es, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
+    }
+    if (p.timers && lane == 0 && ew == 0 && leader) {
+      atomicAdd(p.timers + 5, static_cast<unsigned long long>(clock64() - t_begin));
+      atomicAdd(p.timers + 6, static_cast<unsigned long long>(t_idle));
+      atomicAdd(p.timers + 7, 1ull);
     }
     if (!ok && lane == 0) {
       atomicExch(p.status, DEV_TIMEOUT);
@@ -270,7 +298,7 @@ static moe_status launch_pair_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaS
     attr_done[KIND] = true;
   }
   const int grid = ctx->sm_count & ~1;  // whole pairs
-  grouped_gemm_pair_kernel<KIND><<<grid, GEMM_THREADS, GEMM2_SMEM, st>>>(p);
+  grouped_gemm_pair_kernel<KIND><<<grid, GEMM2_THREADS, GEMM2_SMEM, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

@@ -12,10 +12,15 @@ constexpr int A_BYTES = BM * BK * 2;       // 16 KB
 constexpr int B_BYTES = BN * BK * 2;       // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-major tile: 8 KB
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 192;  // warps: 0 TMA producer, 1 MMA issuer, 2..5 epilogue
 constexpr int ACC_COLS = 256;
 constexpr int TMEM_COLS = 512;
-constexpr size_t GEMM_SMEM = static_cast<size_t>(STAGES) * STAGE_BYTES + 1024;
+// Epilogue staging: every epilogue warp owns EPI_UNITS units of 32 rows x 32 bf16 columns (64-byte rows, XOR
+// swizzle) through which it transposes its results for coalesced global stores.
+constexpr int EPI_UNIT_BYTES = 32 * 64;
+constexpr int EPI_UNITS = 2;
+constexpr int EPI_BYTES = 4 * EPI_UNITS * EPI_UNIT_BYTES;  // 4 epilogue warps: 32 KB
+constexpr size_t GEMM_SMEM = static_cast<size_t>(STAGES) * STAGE_BYTES + EPI_BYTES + 1024;
 
 struct GemmParams {
   CUtensorMap mapA0, mapA1, mapB0, mapB1;
@@ -24,6 +29,7 @@ struct GemmParams {
   const int32_t* pad_offsets;  // padded segment starts, E + 1 entries
   const int32_t* pair_tab;     // CTA-pair kernels: per pair of row blocks {expert, first row, blocks (1|2), 0}
   int32_t* status;
+  unsigned long long* timers;  // null, or 8 counters of this kind: summed over CTAs (see gemm.cu)
   int n_tiles;   // output tiles along N
   int m_tiles;   // weight gradients: output tiles along M per expert
   int E;
@@ -110,40 +116,54 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
   return tl;
 }
 
+// Loads of one K block: the A tile and the B tile of the stage, all credited to the stage's full barrier.
+// (Issuing A and B from two producer warps was tried: the producer's time is back-pressure from the L2 -> SM
+// path, not instruction issue, so it gained nothing.)
 template <int KIND>
 __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl, int kb, uint32_t sA, uint32_t sB,
                                             uint32_t bar) {
+  constexpr bool DO_A = true, DO_B = true;
   if (KIND == GEMM_F3) {
-    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (DO_B) {
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
-      tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
+      for (int c = 0; c < 2; ++c) {
+        tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+        tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
+      }
     }
   } else if (KIND == GEMM_F4 || KIND == GEMM_RT) {
-    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (DO_B) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+      for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+    }
   } else if (KIND == GEMM_B2) {
-    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-    tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
+    if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (DO_B) tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
   } else if (KIND == GEMM_B4 || KIND == GEMM_DX) {
     const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
-    tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
-    tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
+    if (DO_A) tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
+    if (DO_B) tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
   } else if (KIND == GEMM_B3) {
     const int row = tl.row0 + kb * BK;
+    if (DO_A) {
 #pragma unroll
-    for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+      for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+    }
+    if (DO_B) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
+      for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
+    }
   } else {  // GEMM_B5, GEMM_DWR
     const int row = tl.row0 + kb * BK;
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
-      tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
-      tma_load_2d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, row);
+      if (DO_A) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+      if (DO_B) {
+        tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
+        tma_load_2d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, row);
+      }
     }
   }
 }
@@ -175,13 +195,52 @@ __device__ __forceinline__ float fast_sigmoid(float h) { return __fdividef(1.f, 
 
 
 // ---------------------------------------------------------------------------------------------- expert epilogues
-// One thread owns one accumulator row (TMEM lane) of a 128 x 256 tile.  `taddr` addresses that thread's lane
-// quadrant and accumulator buffer; `row` is the row of the padded row buffers (row GEMMs), `m` the row of the
-// expert's weight-gradient slab (weight gradients); `write` is false for a tile whose rows do not exist.
-// All tcgen05.ld are executed by every lane (they are warp-collective); only the stores are predicated.
+// One thread owns one accumulator row (TMEM lane) of a 128 x 256 tile; a warp owns a slab of 32 rows.  Results
+// leave through shared memory: the warp writes a 32 x 32 bf16 unit (lane = row; 16-byte pieces placed with a
+// 64-byte XOR swizzle so both directions are conflict-free), then reads it back transposed - four consecutive lanes
+// hold one 64-byte row segment - and stores that to global memory, eight full row segments per instruction.
+// Measured alternatives on the Qwen shape: 16-byte stores from each lane to its own row cost one memory wavefront
+// per lane (GEMMs at 0.66 of their store-free speed); TMA stores from the same staging queue up behind the
+// producer's deep ring of TMA loads and stall the accumulator hand-off (0.72).
+struct EpiStage {
+  uint32_t base;  // shared address of this warp's two units (2 KB each)
+  uint32_t n;     // units written so far
+};
+
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+// out points at (first row of the slab, first of the 32 columns); rows_valid = rows of the slab inside the tensor.
+__device__ __forceinline__ void stage_store32(EpiStage& es, uint16_t* out, int64_t ld, int rows_valid,
+                                              const float (&v)[32], int lane) {
+  const uint32_t unit = es.base + (es.n & 1u) * EPI_UNIT_BYTES;
+  ++es.n;
+  const uint32_t rowaddr = unit + lane * 64;
+  const uint32_t sw = (lane >> 1) & 3;
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    st_shared_v4(rowaddr + ((j ^ sw) << 4), pack_bf16x2(v[8 * j + 0], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                 pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+  __syncwarp();  // also orders this unit's reads of two calls ago before its reuse
+  const int ch = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = (lane >> 2) + 8 * i;
+    const uint4 w = ld_shared_v4(unit + r * 64 + ((ch ^ ((r >> 1) & 3)) << 4));
+    if (r < rows_valid) *reinterpret_cast<uint4*>(out + r * ld + ch * 8) = w;
+  }
+}
+
+// `slab` is the first output row of the warp's 32-row slab (row of the padded row buffers for row GEMMs, row of
+// the expert's weight-gradient slab for weight gradients); `row` is the thread's own row (only the SwiGLU-backward
+// epilogue reads through it).  `write` (warp-uniform) is false for a tile half whose rows do not exist; `rows_valid`
+// clips a slab that overhangs the tensor.  Every tcgen05.ld is executed by all lanes.
 template <int KIND>
-__device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int64_t row, int m, int n0, uint32_t taddr,
-                                                bool write) {
+__device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int64_t row, int slab, int n0,
+                                                uint32_t taddr, bool write, int rows_valid, EpiStage& es, int lane) {
   if (KIND == GEMM_F3) {
 #pragma unroll 1
     for (int c = 0; c < 4; ++c) {
@@ -191,44 +250,80 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       tmem_ld_wait();
       const int col = n0 + c * 32;
       if (write && col < p.N_total) {
-        float hg[32], hu[32], a[32];
+        float t[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(rg[i]);
+        stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(ru[i]);
+        stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          hg[i] = __uint_as_float(rg[i]);
-          hu[i] = __uint_as_float(ru[i]);
-          a[i] = hg[i] * fast_sigmoid(hg[i]) * hu[i];
+          const float hg = __uint_as_float(rg[i]);
+          t[i] = hg * fast_sigmoid(hg) * __uint_as_float(ru[i]);
         }
-        const int64_t off = row * p.ld_out + col;
-        store_bf16x32(p.out0 + off, hg);
-        store_bf16x32(p.out1 + off, hu);
-        store_bf16x32(p.out2 + off, a);
+        stage_store32(es, p.out2 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
       }
     }
   } else if (KIND == GEMM_B2) {
+    // hg, hu of the thread's row are read straight from global memory, one 32-column chunk ahead of their use
+    uint4 nh[4], nu[4];
+    const bool rd0 = write && n0 < p.N_total;
+    if (rd0) {
+      const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + n0);
+      const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + n0);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        nh[i] = __ldg(qh + i);
+        nu[i] = __ldg(qu + i);
+      }
+    }
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
+      uint4 ch[4], cu[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        ch[i] = nh[i];
+        cu[i] = nu[i];
+      }
+      const int col = n0 + c * 32;
+      if (write && c + 1 < 8 && col + 32 < p.N_total) {
+        const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + col + 32);
+        const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + col + 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          nh[i] = __ldg(qh + i);
+          nu[i] = __ldg(qu + i);
+        }
+      }
       uint32_t rd[32];
       tmem_ld32(taddr + c * 32, rd);
       tmem_ld_wait();
-      const int col = n0 + c * 32;
       if (write && col < p.N_total) {
-        const int64_t off = row * p.ld_out + col;
-        float hg[32], hu[32], dhg[32], dhu[32];
-        load_bf16x32(p.in0 + off, hg);
-        load_bf16x32(p.in1 + off, hu);
+        float hg[32], hu[32], t[32];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          unpack_bf16x2(ch[i].x, hg[8 * i + 0], hg[8 * i + 1]);
+          unpack_bf16x2(ch[i].y, hg[8 * i + 2], hg[8 * i + 3]);
+          unpack_bf16x2(ch[i].z, hg[8 * i + 4], hg[8 * i + 5]);
+          unpack_bf16x2(ch[i].w, hg[8 * i + 6], hg[8 * i + 7]);
+          unpack_bf16x2(cu[i].x, hu[8 * i + 0], hu[8 * i + 1]);
+          unpack_bf16x2(cu[i].y, hu[8 * i + 2], hu[8 * i + 3]);
+          unpack_bf16x2(cu[i].z, hu[8 * i + 4], hu[8 * i + 5]);
+          unpack_bf16x2(cu[i].w, hu[8 * i + 6], hu[8 * i + 7]);
+        }
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const float da = __uint_as_float(rd[i]);
           const float sg = fast_sigmoid(hg[i]);
-          dhg[i] = da * hu[i] * sg * (1.f + hg[i] * (1.f - sg));
-          dhu[i] = da * hg[i] * sg;
+          hu[i] = __uint_as_float(rd[i]) * hu[i] * sg * (1.f + hg[i] * (1.f - sg));  // dhg
+          t[i] = __uint_as_float(rd[i]) * hg[i] * sg;                                 // dhu
         }
-        store_bf16x32(p.out0 + off, dhg);
-        store_bf16x32(p.out1 + off, dhu);
+        stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, hu, lane);
+        stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
       }
     }
   } else {
-    // plain bf16 store: F4, B4 (row GEMMs), B3, B5 (weight gradients)
+    // plain bf16 store: F4, B4, DX (row GEMMs), B3, B5 (weight gradients)
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
       uint32_t rd[32];
@@ -237,20 +332,15 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       float v[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rd[i]);
-      if (Traits<KIND>::WGRAD) {
-        uint16_t* base = p.out0;
-        int col = n0 + c * 32;
-        if (KIND == GEMM_B5) {
-          base = (c >= 4) ? p.out1 : p.out0;
-          col = n0 + (c & 3) * 32;
-        }
-        if (write && m < p.M_total && col < p.N_total)
-          store_bf16x32(base + e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, v);
-      } else {
-        const int col = n0 + c * 32;
-        const bool in_rows = (KIND != GEMM_DX) || row < p.T;  // token tiles may overhang T
-        if (write && in_rows && col < p.N_total) store_bf16x32(p.out0 + row * p.ld_out + col, v);
+      uint16_t* base = p.out0;
+      int col = n0 + c * 32;
+      if (KIND == GEMM_B5) {
+        base = (c >= 4) ? p.out1 : p.out0;
+        col = n0 + (c & 3) * 32;
       }
+      if (write && col < p.N_total)
+        stage_store32(es, base + e * p.expert_stride + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, v,
+                      lane);
     }
   }
 }

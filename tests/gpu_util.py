@@ -25,12 +25,12 @@ def rel_fro(got: np.ndarray, ref: np.ndarray) -> float:
 class Run:
     """Runs the CUDA layer on an instance from synth.make_inputs and keeps the device tensors."""
 
-    def __init__(self, inp: dict, k: int, logits_in=None):
+    def __init__(self, inp: dict, k: int, logits_in=None, flags: int = 0):
         self.inp = inp
         T, d = inp["x"].shape
         E, _, f = inp["W_gate"].shape
         self.T, self.d, self.E, self.f, self.k = T, d, E, f, k
-        self.layer = MoELayer(d, E, f, k)
+        self.layer = MoELayer(d, E, f, k, flags)
         self.dev = {n: to_dev_bf16(inp[n]) for n in ("x", "W_r", "W_gate", "W_up", "W_down", "dy")}
         self.b_r = None if inp.get("b_r") is None else torch.from_numpy(inp["b_r"]).cuda()
         self.logits_in = None if logits_in is None else torch.from_numpy(np.ascontiguousarray(logits_in, np.float32)).cuda()
