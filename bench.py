@@ -27,8 +27,8 @@ import numpy as np  # noqa: E402
 from paper_2608_00916_b200 import synth  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-LAUNCHES_PER_STEP = 17  # router, hist, scan, scatter, gather, 2 GEMMs, combine; combine-bwd, 4 GEMMs, router-bwd,
-#                         dW_r partial + reduce, unpermute-bwd
+LAUNCHES_PER_STEP = 19  # router, hist, scan, scatter, gather, 2 GEMMs, combine; gather(dy), 4 GEMMs, router-bwd,
+#                         dW_r GEMM + reduce, dx-router GEMM + unpermute-sum
 # dram bytes per launch of the dominant kernel taken from the committed ncu capture (profiles/), by stage name;
 # None where no capture has been taken for the workload.
 NCU_TRAFFIC = {}
@@ -53,7 +53,7 @@ def stage_work(shape: synth.MoEShape):
         "gemm_gateup_swiglu": ("tensor", 4 * R * d * f),
         "gemm_down": ("tensor", 2 * R * f * d),
         "combine": ("hbm", 2 * R * d + 2 * T * d + 8 * R),
-        "combine_bwd": ("hbm", 2 * T * d + 4 * R * d + 12 * R),
+        "combine_bwd": ("hbm", 2 * T * d + 2 * R * d + 4 * R),  # gather of dy rows (dg moved into the dgrad-down epilogue)
         "dgrad_down_swiglu_bwd": ("tensor", 2 * R * d * f),
         "wgrad_down": ("tensor", 2 * R * f * d),
         "dgrad_gateup": ("tensor", 4 * R * f * d),

@@ -86,7 +86,8 @@ MOE_API size_t moe_workspace_bytes(const moe_ctx* ctx, int64_t T);
  * Names: "counts" "offsets" "pad_offsets" "logits" "idx" "gates" "inv" "row_token" "xp" "hg" "hu" "act"
  * "o" "dhg" "dhu" "dxp" "dg" "dl".  Internal row buffers (xp, hg, hu, act, o, dhg, dhu, dxp) are laid out
  * expert-major with every expert's segment padded to a multiple of 128 rows ("pad_offsets"); pad rows
- * are zero.  Returns MOE_ERR_INVALID_ARG for an unknown name. */
+ * are zero.  "act" and "o" are stored already multiplied by the row's gate (so the combine is a plain sum); after
+ * moe_backward "o" holds the gathered rows of dy.  Returns MOE_ERR_INVALID_ARG for an unknown name. */
 MOE_API moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char* name /* host */,
                               size_t* offset /* host */, size_t* bytes /* host */);
 
@@ -101,7 +102,7 @@ MOE_API moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cu
  * milliseconds stage s took summed over the pairs recorded since the previous call (the last MOE_PROF_RING
  * of them if there were more), stores that number of pairs in *steps, and starts a new window.
  * Stage order: 0 router, 1 permute (histogram, scan, scatter, gather), 2 gate/up GEMM + SwiGLU,
- * 3 down GEMM, 4 combine, 5 combine-bwd, 6 dgrad-down + SwiGLU-bwd, 7 wgrad-down, 8 dgrad gate/up,
+ * 3 down GEMM, 4 combine, 5 combine-bwd (gather of dy rows), 6 dgrad-down + SwiGLU-bwd (+ dg), 7 wgrad-down, 8 dgrad gate/up,
  * 9 wgrad gate/up, 10 router-bwd (dl), 11 dW_r, 12 unpermute-bwd (dx), 13..15 unused. */
 #define MOE_PROF_RING 64
 MOE_API moe_status moe_set_profiling(moe_ctx* ctx, int enable);

@@ -39,6 +39,8 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.gates = take(sizeof(float) * R);
   L.inv = take(sizeof(int32_t) * R);
   L.row_token = take(sizeof(int32_t) * L.rows_max);
+  L.row_gate = take(sizeof(float) * L.rows_max);
+  L.dg_part = take(sizeof(float) * ((s.f + 255) / 256) * L.rows_max);
   L.dg = take(sizeof(float) * R);
   L.dl = take(sizeof(float) * T * s.E);
   L.dl_hi = take(sizeof(uint16_t) * (T * s.E + 64));
@@ -288,7 +290,7 @@ moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_
     {
       StageTimer tm(c, st, 4);
       launch_combine(s, T, reinterpret_cast<const uint16_t*>(ws + L.o), reinterpret_cast<const float*>(ws + L.gates),
-                     reinterpret_cast<const int32_t*>(ws + L.inv), y, st);
+                     reinterpret_cast<const int32_t*>(ws + L.inv), y, st);  // o already carries the gates
     }
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
@@ -322,10 +324,9 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   io.x = x; io.W_r = W_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
   io.dW_gate = dW_gate; io.dW_up = dW_up; io.dW_down = dW_down; io.dx = dx;
   const bool tc_router = router_on_tensor_cores(s);
-  {
+  if (T > 0) {
     StageTimer tm(c, st, 5);
-    launch_combine_bwd(s, T, dy, reinterpret_cast<uint16_t*>(ws + L.o), gates, inv,
-                       reinterpret_cast<float*>(ws + L.dg), st);
+    launch_gather_rows(s, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st);
   }
   if (T > 0) {
     StageTimer tm(c, st, 6);
@@ -350,9 +351,9 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   {
     StageTimer tm(c, st, 10);
     launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
-                      gates, reinterpret_cast<const float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts),
-                      d_aux, dl, reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo),
-                      st);
+                      gates, reinterpret_cast<const float*>(ws + L.dg_part), (s.f + 255) / 256, L.rows_max, inv,
+                      reinterpret_cast<float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts), d_aux, dl,
+                      reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo), st);
   }
   {
     StageTimer tm(c, st, 11);

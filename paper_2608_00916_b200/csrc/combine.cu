@@ -5,32 +5,29 @@
 namespace moe {
 
 // ------------------------------------------------------------------------------------------ combine
-// y[t,:] = sum_{j<k} g[t,j] * o[inv[t,j],:]   (fp32 accumulation in slot order, one bf16 rounding).
+// y[t,:] = sum_{j<k} o[inv[t,j],:] where the rows of o already carry their gate (the gate-up epilogue folds it into
+// the activation); fp32 accumulation in slot order, one bf16 rounding.
 // One block per token; a thread owns 8 consecutive columns (16 bytes) and issues the k row loads back to back.
 __global__ void __launch_bounds__(256) combine_kernel(int d, int k, const uint16_t* __restrict__ o,
                                                       const float* __restrict__ gates, const int32_t* __restrict__ inv,
                                                       uint16_t* __restrict__ y) {
   const int64_t t = blockIdx.x;
-  __shared__ float sg[MAX_K];
   __shared__ int sr[MAX_K];
-  if (threadIdx.x < k) {
-    sg[threadIdx.x] = gates[t * k + threadIdx.x];
-    sr[threadIdx.x] = inv[t * k + threadIdx.x];
-  }
+  (void)gates;
+  if (threadIdx.x < k) sr[threadIdx.x] = inv[t * k + threadIdx.x];
   __syncthreads();
   for (int c = threadIdx.x * 8; c < d; c += 256 * 8) {
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-#pragma unroll 4
+#pragma unroll 8
     for (int j = 0; j < k; ++j) {
       const uint4 v = __ldg(reinterpret_cast<const uint4*>(o + static_cast<int64_t>(sr[j]) * d + c));
-      const float g = sg[j];
       float a, b;
-      unpack_bf16x2(v.x, a, b); acc[0] = fmaf(g, a, acc[0]); acc[1] = fmaf(g, b, acc[1]);
-      unpack_bf16x2(v.y, a, b); acc[2] = fmaf(g, a, acc[2]); acc[3] = fmaf(g, b, acc[3]);
-      unpack_bf16x2(v.z, a, b); acc[4] = fmaf(g, a, acc[4]); acc[5] = fmaf(g, b, acc[5]);
-      unpack_bf16x2(v.w, a, b); acc[6] = fmaf(g, a, acc[6]); acc[7] = fmaf(g, b, acc[7]);
+      unpack_bf16x2(v.x, a, b); acc[0] += a; acc[1] += b;
+      unpack_bf16x2(v.y, a, b); acc[2] += a; acc[3] += b;
+      unpack_bf16x2(v.z, a, b); acc[4] += a; acc[5] += b;
+      unpack_bf16x2(v.w, a, b); acc[6] += a; acc[7] += b;
     }
     uint4 w;
     w.x = pack_bf16x2(acc[0], acc[1]);
@@ -47,94 +44,17 @@ void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* g
   combine_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, o, gates, inv, y);
 }
 
-// ------------------------------------------------------------------------------------------ combine backward
-// dg[t,j] = <dy[t,:], o[r,:]>,  d_o[r,:] = g[t,j] * dy[t,:]  with r = inv[t,j]; d_o overwrites o in place.
-__global__ void __launch_bounds__(256) combine_bwd_kernel(int d, int k, const uint16_t* __restrict__ dy,
-                                                          uint16_t* __restrict__ o, const float* __restrict__ gates,
-                                                          const int32_t* __restrict__ inv, float* __restrict__ dg) {
-  const int64_t t = blockIdx.x;
-  __shared__ float sg[MAX_K];
-  __shared__ int sr[MAX_K];
-  __shared__ float part[8][MAX_K];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x < k) {
-    sg[threadIdx.x] = gates[t * k + threadIdx.x];
-    sr[threadIdx.x] = inv[t * k + threadIdx.x];
-  }
-  __syncthreads();
-  float dot[MAX_K];
-#pragma unroll
-  for (int j = 0; j < MAX_K; ++j) dot[j] = 0.f;
-  for (int c = threadIdx.x * 8; c < d; c += 256 * 8) {
-    const uint4 dv = __ldg(reinterpret_cast<const uint4*>(dy + t * d + c));
-    float dyv[8];
-    unpack_bf16x2(dv.x, dyv[0], dyv[1]);
-    unpack_bf16x2(dv.y, dyv[2], dyv[3]);
-    unpack_bf16x2(dv.z, dyv[4], dyv[5]);
-    unpack_bf16x2(dv.w, dyv[6], dyv[7]);
-    // groups of 8 slots: all row loads of a group are issued before the first store, so they overlap
-#pragma unroll
-    for (int j0 = 0; j0 < MAX_K; j0 += 8) {
-      if (j0 < k) {
-        uint4 v[8];
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj)
-          if (j0 + jj < k) v[jj] = *reinterpret_cast<const uint4*>(o + static_cast<int64_t>(sr[j0 + jj]) * d + c);
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj) {
-          if (j0 + jj < k) {
-            float ov[8];
-            unpack_bf16x2(v[jj].x, ov[0], ov[1]);
-            unpack_bf16x2(v[jj].y, ov[2], ov[3]);
-            unpack_bf16x2(v[jj].z, ov[4], ov[5]);
-            unpack_bf16x2(v[jj].w, ov[6], ov[7]);
-            float s = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) s = fmaf(dyv[i], ov[i], s);
-            dot[j0 + jj] += s;
-            const float g = sg[j0 + jj];
-            uint4 w;
-            w.x = pack_bf16x2(g * dyv[0], g * dyv[1]);
-            w.y = pack_bf16x2(g * dyv[2], g * dyv[3]);
-            w.z = pack_bf16x2(g * dyv[4], g * dyv[5]);
-            w.w = pack_bf16x2(g * dyv[6], g * dyv[7]);
-            *reinterpret_cast<uint4*>(o + static_cast<int64_t>(sr[j0 + jj]) * d + c) = w;
-          }
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < MAX_K; ++j) {
-    if (j < k) {
-      float s = dot[j];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-      if (lane == 0) part[warp][j] = s;
-    }
-  }
-  __syncthreads();
-  if (threadIdx.x < k) {
-    float s = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
-    dg[t * k + threadIdx.x] = s;
-  }
-}
-
-void launch_combine_bwd(const Shape& s, int64_t T, const uint16_t* dy, uint16_t* o_to_do, const float* gates,
-                        const int32_t* inv, float* dg, cudaStream_t st) {
-  if (T == 0) return;
-  combine_bwd_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, dy, o_to_do, gates, inv, dg);
-}
-
 // ------------------------------------------------------------------------------------------ router backward
-// One warp per token.  p is recomputed from the saved logits.
+// One warp per token.  p is recomputed from the saved logits; dg[t,j] = <dy[t], o_tj> arrives as per-row partial
+// sums written by the dgrad-down epilogue (one slice per column tile) and is summed here in slice order.
 //   dl[t,e]  = p_e (dp_e - <p, dp>)                       auxiliary loss through P_e, dp_e = d_aux E c_e / (T k) / T
 //   dl[t,idx_j] += g_j (dg_j - sum_j' g_j' dg_j')         gates = softmax over the selected logits
 __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k, const float* __restrict__ logits,
                                                          const int32_t* __restrict__ idx,
-                                                         const float* __restrict__ gates, const float* __restrict__ dg,
+                                                         const float* __restrict__ gates,
+                                                         const float* __restrict__ dg_part, int dg_tiles,
+                                                         int64_t rows_max, const int32_t* __restrict__ inv,
+                                                         float* __restrict__ dg,
                                                          const int32_t* __restrict__ counts, float d_aux,
                                                          float* __restrict__ dl, uint16_t* __restrict__ dl_hi,
                                                          uint16_t* __restrict__ dl_lo) {
@@ -180,8 +100,10 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
   int ej = -1;
   if (lane < k) {
     g = gates[t * k + lane];
-    dgj = dg[t * k + lane];
     ej = idx[t * k + lane];
+    const int r = inv[t * k + lane];
+    for (int nt = 0; nt < dg_tiles; ++nt) dgj += dg_part[nt * rows_max + r];
+    dg[t * k + lane] = dgj;
   }
   float inner = g * dgj;
 #pragma unroll
@@ -211,11 +133,13 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
 }
 
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
-                       const float* dg, const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi,
-                       uint16_t* dl_lo, cudaStream_t st) {
+                       const float* dg_part, int dg_tiles, int64_t rows_max, const int32_t* inv, float* dg,
+                       const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi, uint16_t* dl_lo,
+                       cudaStream_t st) {
   if (T == 0) return;
-  router_bwd_kernel<<<static_cast<unsigned>((T + 7) / 8), 256, 0, st>>>(T, s.E, s.k, logits, idx, gates, dg, counts,
-                                                                        d_aux, dl, dl_hi, dl_lo);
+  router_bwd_kernel<<<static_cast<unsigned>((T + 7) / 8), 256, 0, st>>>(T, s.E, s.k, logits, idx, gates, dg_part,
+                                                                        dg_tiles, rows_max, inv, dg, counts, d_aux, dl,
+                                                                        dl_hi, dl_lo);
 }
 
 // ------------------------------------------------------------------------------------------ dW_r, db_r

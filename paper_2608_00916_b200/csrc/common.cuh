@@ -43,13 +43,15 @@ struct WsLayout {
   size_t gates;        // float[T*k]
   size_t inv;          // int32[T*k]  padded row of pair (t, j)
   size_t row_token;    // int32[rows_max] token of a padded row, -1 for pad rows
+  size_t row_gate;     // float[rows_max] gate of a padded row, 0 for pad rows
+  size_t dg_part;      // float[ceil(f/256) * rows_max] per-row partial sums of dg, one slice per dgrad-down column tile
   size_t dg;           // float[T*k]
   size_t dl;           // float[T*E]
   size_t dl_hi, dl_lo; // bf16[T*E]   dl split into two bf16 terms (hi + lo) for the tensor-core contractions
   size_t dwr_part;     // float[DWR_SPLIT * d * E]
   size_t xp;           // bf16[rows_max * d]
   size_t hg, hu, act;  // bf16[rows_max * f]
-  size_t o;            // bf16[rows_max * d]   o in forward, overwritten by d_o in backward
+  size_t o;            // bf16[rows_max * d]   gate-scaled o in forward, the gathered dy rows in backward
   size_t dhg, dhu;     // bf16[rows_max * f]
   size_t dxp;          // bf16[rows_max * d]
   size_t dxr;          // bf16[T * d]  router term of dx (dl W_r^T)
@@ -85,11 +87,14 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
 // ---- launchers (combine.cu)
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
                     uint16_t* y, cudaStream_t st);
-void launch_combine_bwd(const Shape& s, int64_t T, const uint16_t* dy, uint16_t* o_to_do, const float* gates,
-                        const int32_t* inv, float* dg, cudaStream_t st);
+// rows[r,:] = src[row_token[r],:] (zero for pad rows) for every padded row: xp from x, and the dy rows of backward
+void launch_gather_rows(const Shape& s, const WsLayout& L, const char* ws, const uint16_t* src, uint16_t* rows,
+                        cudaStream_t st);
+// dg[t,j] = sum over column tiles of dg_part[tile][inv[t,j]], then dl (fp32 and the two-term bf16 split)
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
-                       const float* dg, const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi,
-                       uint16_t* dl_lo, cudaStream_t st);
+                       const float* dg_part, int dg_tiles, int64_t rows_max, const int32_t* inv, float* dg,
+                       const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi, uint16_t* dl_lo,
+                       cudaStream_t st);
 // SIMT dW_r (any E) and the shared partial reduction / db_r
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
                 float* db_r, bool partials_ready, cudaStream_t st);

@@ -417,6 +417,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.N_total = f;
       p.out0 = hg; p.out1 = hu; p.out2 = act;
       p.ld_out = f;
+      p.row_gate = reinterpret_cast<const float*>(ws + L.row_gate);
       if (!ok) return MOE_ERR_CUDA;
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_F3>(ctx, p, st);
     case GEMM_F4:
@@ -438,6 +439,9 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.in0 = hg; p.in1 = hu;
       p.out0 = dhg; p.out1 = dhu;
       p.ld_out = f;
+      p.row_gate = reinterpret_cast<const float*>(ws + L.row_gate);
+      p.outf = reinterpret_cast<float*>(ws + L.dg_part);
+      p.rows_max = L.rows_max;
       if (!ok) return MOE_ERR_CUDA;
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B2>(ctx, p, st);
     case GEMM_B4:

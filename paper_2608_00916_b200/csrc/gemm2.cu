@@ -217,14 +217,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
               umma_bf16_pair(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
             }
             // the stage is free in both CTAs once these MMAs have read it
-            umma_commit_pair(mapa_shared(empty_bar(s), 0));
-            umma_commit_pair(mapa_shared(empty_bar(s), 1));
+            umma_commit_pair_both(empty_bar(s));
           }
           __syncwarp();
         }
         if (ok && lane == 0) {
-          umma_commit_pair(mapa_shared(tfull_bar(acc), 0));
-          umma_commit_pair(mapa_shared(tfull_bar(acc), 1));
+          umma_commit_pair_both(tfull_bar(acc));
         }
         __syncwarp();
       }

@@ -57,7 +57,9 @@ struct GemmParams {
   float* gates;
   float* gates_out;
   float* psum_part;     // RT: [4 * tiles, E] per-warp column sums of p
-  float* outf;          // DWR: [slices, d, E] fp32 partials
+  float* outf;          // DWR: [slices, d, E] fp32 partials; B2: [column tiles, rows_max] partial sums of dg
+  const float* row_gate;  // F3, B2: gate of every padded row (0 for pad rows)
+  int64_t rows_max;     // B2: stride of the dg partial slices
 };
 
 template <int KIND>
@@ -251,6 +253,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       const int col = n0 + c * 32;
       if (write && col < p.N_total) {
         float t[32];
+        const float gate = p.row_gate[row];  // the combine weight is folded into the saved activation
 #pragma unroll
         for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(rg[i]);
         stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
@@ -260,7 +263,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const float hg = __uint_as_float(rg[i]);
-          t[i] = hg * fast_sigmoid(hg) * __uint_as_float(ru[i]);
+          t[i] = gate * hg * fast_sigmoid(hg) * __uint_as_float(ru[i]);
         }
         stage_store32(es, p.out2 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
       }
@@ -268,6 +271,8 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
   } else if (KIND == GEMM_B2) {
     // hg, hu of the thread's row are read straight from global memory, one 32-column chunk ahead of their use
     uint4 nh[4], nu[4];
+    const float gate = write ? p.row_gate[row] : 0.f;
+    float dgp = 0.f;  // this row's share of dg = <dy, o> = <da, silu(hg) hu> over the tile's columns
     const bool rd0 = write && n0 < p.N_total;
     if (rd0) {
       const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + n0);
@@ -315,13 +320,17 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const float sg = fast_sigmoid(hg[i]);
-          hu[i] = __uint_as_float(rd[i]) * hu[i] * sg * (1.f + hg[i] * (1.f - sg));  // dhg
-          t[i] = __uint_as_float(rd[i]) * hg[i] * sg;                                 // dhu
+          const float da = __uint_as_float(rd[i]);  // dy W_down^T without the gate
+          dgp = fmaf(da, hg[i] * sg * hu[i], dgp);
+          const float dag = gate * da;
+          hu[i] = dag * hu[i] * sg * (1.f + hg[i] * (1.f - sg));  // dhg
+          t[i] = dag * hg[i] * sg;                                 // dhu
         }
         stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, hu, lane);
         stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
       }
     }
+    if (write) p.outf[static_cast<int64_t>(n0 / 256) * p.rows_max + row] = dgp;
   } else {
     // plain bf16 store: F4, B4, DX (row GEMMs), B3, B5 (weight gradients)
 #pragma unroll 1

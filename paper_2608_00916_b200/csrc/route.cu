@@ -312,7 +312,9 @@ __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int
                                                            const int32_t* __restrict__ tile_base,
                                                            const int32_t* __restrict__ offsets,
                                                            const int32_t* __restrict__ pad_offsets,
+                                                           const float* __restrict__ gates,
                                                            int32_t* __restrict__ inv, int32_t* __restrict__ row_token,
+                                                           float* __restrict__ row_gate,
                                                            int32_t* __restrict__ perm_out) {
   extern __shared__ uint32_t sc_masks[];
   const int64_t tile_t0 = static_cast<int64_t>(blockIdx.x) * TOK_TILE;
@@ -328,27 +330,44 @@ __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int
     const int r = pad_offsets[e] + rank;
     inv[t * k + j] = r;
     row_token[r] = static_cast<int32_t>(t);
+    row_gate[r] = gates[t * k + j];
     if (perm_out) perm_out[offsets[e] + rank] = static_cast<int32_t>(t * k + j);
   }
 }
 
-// xp[r,:] = x[row_token[r],:], zero for pad rows.  One warp per row, 16-byte accesses.
-__global__ void __launch_bounds__(256) gather_rows_kernel(int d, const uint16_t* __restrict__ x,
+// rows[r,:] = src[row_token[r],:], zero for pad rows.  One warp per row; a lane keeps four 16-byte loads in
+// flight before it stores.
+__global__ void __launch_bounds__(256) gather_rows_kernel(int d, const uint16_t* __restrict__ src,
                                                           const int32_t* __restrict__ row_token,
                                                           const int32_t* __restrict__ sched,
-                                                          uint16_t* __restrict__ xp) {
+                                                          uint16_t* __restrict__ rows) {
   const int lane = threadIdx.x & 31;
   const int64_t r = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (r >= sched[1]) return;
   const int t = row_token[r];
-  uint4* dst = reinterpret_cast<uint4*>(xp + r * d);
+  uint4* dst = reinterpret_cast<uint4*>(rows + r * d);
   const int n16 = d / 8;
   if (t < 0) {
     for (int i = lane; i < n16; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
   } else {
-    const uint4* src = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(t) * d);
-    for (int i = lane; i < n16; i += 32) dst[i] = __ldg(src + i);
+    const uint4* s4 = reinterpret_cast<const uint4*>(src + static_cast<int64_t>(t) * d);
+    int i = lane;
+    for (; i + 96 < n16; i += 128) {
+      const uint4 a = __ldg(s4 + i), b = __ldg(s4 + i + 32), c = __ldg(s4 + i + 64), e = __ldg(s4 + i + 96);
+      dst[i] = a;
+      dst[i + 32] = b;
+      dst[i + 64] = c;
+      dst[i + 96] = e;
+    }
+    for (; i < n16; i += 32) dst[i] = __ldg(s4 + i);
   }
+}
+
+void launch_gather_rows(const Shape& s, const WsLayout& L, const char* ws, const uint16_t* src, uint16_t* rows,
+                        cudaStream_t st) {
+  const int gblocks = static_cast<int>((L.rows_max + 7) / 8);
+  gather_rows_kernel<<<gblocks, 256, 0, st>>>(s.d, src, reinterpret_cast<const int32_t*>(ws + L.row_token),
+                                              reinterpret_cast<const int32_t*>(ws + L.sched), rows);
 }
 
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
@@ -359,6 +378,7 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
   const int tiles = static_cast<int>(L.tok_tiles);
   const size_t msm = sizeof(uint32_t) * 8 * s.E;
   cudaMemsetAsync(row_token, 0xFF, sizeof(int32_t) * L.rows_max, st);
+  cudaMemsetAsync(ws + L.row_gate, 0, sizeof(float) * L.rows_max, st);
   if (tiles > 0) hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
   scan_kernel<<<1, SCAN_THREADS, 0, st>>>(T, s.E, s.k, tiles, psum_rows, tile_counts,
                                  reinterpret_cast<int32_t*>(ws + L.counts), reinterpret_cast<int32_t*>(ws + L.offsets),
@@ -372,11 +392,9 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
   if (tiles > 0) {
     scatter_kernel<<<tiles, TOK_TILE, msm, st>>>(
         T, s.E, s.k, idx, tile_counts, reinterpret_cast<const int32_t*>(ws + L.offsets),
-        reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<int32_t*>(ws + L.inv), row_token,
-        perm_out);
-    const int gblocks = static_cast<int>((L.rows_max + 7) / 8);
-    gather_rows_kernel<<<gblocks, 256, 0, st>>>(s.d, x, row_token, reinterpret_cast<const int32_t*>(ws + L.sched),
-                                                reinterpret_cast<uint16_t*>(ws + L.xp));
+        reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const float*>(ws + L.gates),
+        reinterpret_cast<int32_t*>(ws + L.inv), row_token, reinterpret_cast<float*>(ws + L.row_gate), perm_out);
+    launch_gather_rows(s, L, ws, x, reinterpret_cast<uint16_t*>(ws + L.xp), st);
   }
 }
 

@@ -30,19 +30,24 @@ def check_all(r: Run, ofw, obw, d_aux, stages=True):
     fw = r.forward()
     check_routing(fw, ofw)
     d, f, k, E = r.d, r.f, r.k, r.E
+    # the library folds the gate of a routed row into its saved activation: act and o are stored gate-scaled
+    g_row = ofw["gates"].reshape(-1)[ofw["perm"]][:, None]
     if stages:
         for nm, w in (("xp", d), ("hg", f), ("hu", f), ("act", f), ("o", d)):
             got, pad = r.rows(nm, w)
-            assert rel_fro(got, ofw[nm]) <= (0.0 if nm == "xp" else TOL), nm
+            ref = ofw[nm] * g_row if nm in ("act", "o") else ofw[nm]
+            assert rel_fro(got, ref) <= (0.0 if nm == "xp" else TOL), nm
             assert not pad.any(), f"pad rows of {nm} are not zero"
     assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
     bw = r.backward(d_aux)
     if stages:
         assert rel_fro(r.layer.buffer("dg", torch.float32).cpu().numpy().reshape(-1, k), obw["dg"]) <= TOL
-        for nm, w, on in (("o", d, "d_o"), ("dhg", f, "dhg"), ("dhu", f, "dhu"), ("dxp", d, "dxp")):
+        # in backward the o buffer holds the gathered dy rows (d_o without its gate)
+        dy_rows = synth.bf16_bits_to_f64(r.inp["dy"])[ofw["perm"] // k]
+        for nm, w, ref in (("o", d, dy_rows), ("dhg", f, obw["dhg"]), ("dhu", f, obw["dhu"]), ("dxp", d, obw["dxp"])):
             got, pad = r.rows(nm, w)
-            assert rel_fro(got, obw[on]) <= TOL, on
-            assert not pad.any(), f"pad rows of {on} are not zero"
+            assert rel_fro(got, ref) <= (0.0 if nm == "o" else TOL), nm
+            assert not pad.any(), f"pad rows of {nm} (backward) are not zero"
         assert rel_fro(r.layer.buffer("dl", torch.float32).cpu().numpy().reshape(-1, E), obw["dl"]) <= TOL
     for nm in ("dx", "dW_gate", "dW_up", "dW_down"):
         assert rel_fro(from_dev_bf16(bw[nm]), obw[nm]) <= TOL, nm
