@@ -354,6 +354,23 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
   }
 }
 
+// Called by an epilogue thread before it starts waiting for the tile's accumulator: the SwiGLU-backward epilogue
+// reads hg and hu of its row from global memory, and those rows come straight from DRAM.  Pulling their lines
+// into L2 while the tile's main loop still runs keeps the epilogue from stalling on each 32-column chunk (it was
+// the slower side of this kernel: accumulators waited for it).
+template <int KIND>
+__device__ __forceinline__ void epilogue_prefetch(const GemmParams& p, int64_t row, int n0, bool write) {
+  if (KIND == GEMM_B2 && write) {
+    const int cols = min(256, p.N_total - n0);
+    const uint16_t* h = p.in0 + row * p.ld_out + n0;
+    const uint16_t* u = p.in1 + row * p.ld_out + n0;
+    for (int c = 0; c < cols; c += 64) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(h + c));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(u + c));
+    }
+  }
+}
+
 // Weight gradient of an expert without tokens: the thread's row of the output tile is zero.
 template <int KIND>
 __device__ __forceinline__ void wgrad_zero_fill(const GemmParams& p, int e, int m, int n0) {
