@@ -28,6 +28,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.counts = take(sizeof(int32_t) * s.E);
   L.offsets = take(sizeof(int32_t) * (s.E + 1));
   L.pad_offsets = take(sizeof(int32_t) * (s.E + 1));
+  L.expert_order = take(sizeof(int32_t) * s.E);
   L.sched = take(sizeof(int32_t) * 4);
   L.tile_expert = take(sizeof(int32_t) * L.max_m_tiles);
   L.pair_tab = take(sizeof(int32_t) * 4 * L.max_m_tiles);

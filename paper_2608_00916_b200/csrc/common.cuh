@@ -32,6 +32,7 @@ struct WsLayout {
   size_t counts;       // int32[E]    rows per expert
   size_t offsets;      // int32[E+1]  exclusive scan of counts (canonical, unpadded)
   size_t pad_offsets;  // int32[E+1]  exclusive scan of counts rounded up to ROW_PAD
+  size_t expert_order; // int32[E]    experts sorted by row count, largest first
   size_t sched;        // int32[4]    [0] number of 128-row tiles, [1] padded row total, [2] number of block pairs
   size_t tile_expert;  // int32[max_m_tiles] expert of every 128-row tile
   size_t pair_tab;     // int32[4 * max_m_tiles] pairs of 128-row blocks of one expert: {expert, first row, blocks, 0}

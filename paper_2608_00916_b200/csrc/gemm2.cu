@@ -41,8 +41,9 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
   Tile2 tl;
   if (Traits<KIND>::WGRAD) {
     const int per = p.m_tiles * p.n_tiles;
-    tl.e = t / per;
-    const int rem = t - tl.e * per;
+    const int slot = t / per;
+    tl.e = p.expert_order[slot];  // longest K loops first
+    const int rem = t - slot * per;
     tl.m0 = (rem / p.n_tiles) * 2 * BM + rank * BM;
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
     tl.row0 = p.pad_offsets[tl.e];

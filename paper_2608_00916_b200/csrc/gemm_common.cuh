@@ -27,6 +27,7 @@ struct GemmParams {
   const int32_t* sched;        // [0] number of 128-row tiles
   const int32_t* tile_expert;  // expert of each 128-row tile
   const int32_t* pad_offsets;  // padded segment starts, E + 1 entries
+  const int32_t* expert_order; // weight gradients: experts by row count, largest first
   const int32_t* pair_tab;     // CTA-pair kernels: per pair of row blocks {expert, first row, blocks (1|2), 0}
   int32_t* status;
   unsigned long long* timers;  // null, or 8 counters of this kind: summed over CTAs (see gemm.cu)
@@ -93,6 +94,7 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     const int rem = t - tl.e * per;
     tl.m0 = (rem / p.n_tiles) * BM;
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
+    if (KIND != GEMM_DWR) tl.e = p.expert_order[tl.e];  // longest K loops first
     if (KIND == GEMM_DWR) {  // "expert" = token slice
       tl.row0 = tl.e * p.split_rows;
       tl.nkb = max(0, min(p.split_rows, p.rows_total - tl.row0)) / BK;

@@ -235,6 +235,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
                                                             int32_t* __restrict__ pad_offsets,
                                                             int32_t* __restrict__ sched, int32_t* __restrict__ tile_expert,
                                                             int32_t* __restrict__ pair_tab,
+                                                            int32_t* __restrict__ expert_order,
                                                             const float* __restrict__ psum_part,
                                                             float* __restrict__ psum, int32_t* __restrict__ counts_out,
                                                             float* __restrict__ aux_out, int32_t* __restrict__ status) {
@@ -257,14 +258,29 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
     s_ps[tid] = ps;
   }
   __syncthreads();
-  for (int e = tid; e < E; e += SCAN_THREADS) {
-    int run = 0;
-    for (int tl = 0; tl < tok_tiles; ++tl) {
-      int c = tile_counts[static_cast<int64_t>(tl) * E + e];
-      tile_counts[static_cast<int64_t>(tl) * E + e] = run;
-      run += c;
+  // exclusive prefix of every expert's column of tile_counts along the tiles: one warp per expert, 32 tiles per step
+  {
+    const int lane = tid & 31, wid = tid >> 5;
+    for (int e = wid; e < E; e += SCAN_THREADS / 32) {
+      int run = 0;
+      for (int t0 = 0; t0 < tok_tiles; t0 += 32) {
+        const int tl = t0 + lane;
+        const int c = tl < tok_tiles ? tile_counts[static_cast<int64_t>(tl) * E + e] : 0;
+        int inc = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+          if (lane >= off) inc += v;
+        }
+        if (tl < tok_tiles) tile_counts[static_cast<int64_t>(tl) * E + e] = run + inc - c;
+        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+      }
+      if (lane == 0) s_cnt[e] = run;
     }
-    s_cnt[e] = run;
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += SCAN_THREADS) {
+    const int run = s_cnt[e];
     counts[e] = run;
     counts_out[e] = run;
     float ps = 0.f;
@@ -272,6 +288,11 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
     psum[e] = ps;
     // aux term: (c_e / (T k)) * (Psum_e / T)
     s_term[e] = (T > 0) ? (static_cast<float>(run) / static_cast<float>(T * k)) * (ps / static_cast<float>(T)) : 0.f;
+    // position of e in the order "most rows first" (ties by index): the weight-gradient kernels start with the
+    // experts whose K loops are longest so that a skewed load does not leave a long tail
+    int rank = 0;
+    for (int o = 0; o < E; ++o) rank += (s_cnt[o] > run || (s_cnt[o] == run && o < e)) ? 1 : 0;
+    expert_order[rank] = e;
   }
   __syncthreads();
   if (tid == 0) {
@@ -386,6 +407,7 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
                                  reinterpret_cast<int32_t*>(ws + L.sched),
                                  reinterpret_cast<int32_t*>(ws + L.tile_expert),
                                  reinterpret_cast<int32_t*>(ws + L.pair_tab),
+                                 reinterpret_cast<int32_t*>(ws + L.expert_order),
                                  reinterpret_cast<const float*>(ws + L.psum_part),
                                  reinterpret_cast<float*>(ws + L.psum), counts_out, aux_out,
                                  reinterpret_cast<int32_t*>(ws + L.status));
