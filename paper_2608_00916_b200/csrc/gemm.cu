@@ -72,7 +72,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     uint32_t it = 0;
     bool ok = true;
     long long t_wait = 0, t_begin = clock64();
-    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+    for (int rd = 0; rd * static_cast<int>(gridDim.x) < ntiles && ok; ++rd) {
+      const int t = tile_of_round<KIND>(rd, blockIdx.x, gridDim.x);
+      if (t >= ntiles) continue;
       const Tile tl = get_tile<KIND>(p, t);
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
         const int s = it % STAGES;
@@ -107,7 +109,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     uint32_t it = 0, tc = 0;
     bool ok = true;
     long long t_acc = 0, t_full = 0, t_begin = clock64();
-    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+    for (int rd = 0; rd * static_cast<int>(gridDim.x) < ntiles && ok; ++rd) {
+      const int t = tile_of_round<KIND>(rd, blockIdx.x, gridDim.x);
+      if (t >= ntiles) continue;
       const Tile tl = get_tile<KIND>(p, t);
       if (tl.nkb == 0) continue;
       const int acc = tc & 1;
@@ -163,7 +167,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     uint32_t tc = 0;
     bool ok = true;
     long long t_idle = 0, t_begin = clock64();
-    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+    for (int rd = 0; rd * static_cast<int>(gridDim.x) < ntiles && ok; ++rd) {
+      const int t = tile_of_round<KIND>(rd, blockIdx.x, gridDim.x);
+      if (t >= ntiles) continue;
       const Tile tl = get_tile<KIND>(p, t);
       const int rin = ew * 32 + lane;  // row inside the tile
       if (tl.nkb == 0) {

@@ -148,7 +148,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
     uint32_t it = 0;
     bool ok = true;
     long long t_wait = 0, t_begin = clock64();
-    for (int t = cid; t < ntiles && ok; t += nclusters) {
+    for (int rd = 0; rd * nclusters < ntiles && ok; ++rd) {
+      const int t = tile_of_round<KIND>(rd, cid, nclusters);
+      if (t >= ntiles) continue;
       const Tile2 tl = get_tile2<KIND>(p, t, rank);
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
         const int s = it % STAGES2;
@@ -184,7 +186,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       uint32_t it = 0, tc = 0;
       bool ok = true;
       long long t_acc = 0, t_full = 0, t_begin = clock64();
-      for (int t = cid; t < ntiles && ok; t += nclusters) {
+      for (int rd = 0; rd * nclusters < ntiles && ok; ++rd) {
+      const int t = tile_of_round<KIND>(rd, cid, nclusters);
+      if (t >= ntiles) continue;
         const Tile2 tl = get_tile2<KIND>(p, t, rank);
         if (tl.nkb == 0) continue;
         const int acc = tc & 1;
@@ -244,7 +248,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
     uint32_t tc = 0;
     bool ok = true;
     long long t_idle = 0, t_begin = clock64();
-    for (int t = cid; t < ntiles && ok; t += nclusters) {
+    for (int rd = 0; rd * nclusters < ntiles && ok; ++rd) {
+      const int t = tile_of_round<KIND>(rd, cid, nclusters);
+      if (t >= ntiles) continue;
       const Tile2 tl = get_tile2<KIND>(p, t, rank);
       const int rin = ew * 32 + lane;
       if (tl.nkb == 0) {

@@ -78,6 +78,14 @@ struct Tile {
   int e, row0, m0, n0, nkb;
 };
 
+// Static tile assignment of the persistent kernels: worker `w` of `nw` takes one tile per round.  Weight-gradient
+// tiles are ordered longest first, so odd rounds run through the workers backwards (a snake): the worker that got the
+// longest tile of one round gets the shortest of the next, which evens out skewed expert loads.
+template <int KIND>
+__device__ __forceinline__ int tile_of_round(int round, int w, int nw) {
+  return round * nw + ((Traits<KIND>::WGRAD && (round & 1)) ? nw - 1 - w : w);
+}
+
 template <int KIND>
 __device__ __forceinline__ int total_tiles(const GemmParams& p) {
   if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;

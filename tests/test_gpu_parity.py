@@ -79,6 +79,7 @@ def test_tiny_config_stage_by_stage():
     (300, 128, 1, 1, 256, 16),    # E = 1, k = 1: dense SwiGLU MLP
     (2049, 256, 32, 8, 128, 17),  # more than 8 token tiles, k = 8
     (520, 320, 256, 6, 64, 18),   # the largest expert count
+    (200, 128, 64, 32, 128, 19),  # the largest top_k
 ])
 def test_odd_shapes(T, d, E, k, f, seed):
     shape = synth.MoEShape(T, d, E, k, f)
@@ -225,6 +226,6 @@ def test_full_coarse_config_sampled():
     sampled_parity("coarse", n_tokens=8)
 
 
-@pytest.mark.parametrize("name", ["sweep_T1000", "sweep_T8191"])
+@pytest.mark.parametrize("name", ["sweep_T1000", "sweep_T4096", "sweep_T8191", "sweep_T32768", "sweep_T65536"])
 def test_sweep_sampled(name):
     sampled_parity(name, n_tokens=24)
