@@ -82,7 +82,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -142,7 +142,7 @@ def host_cores():
 
 def run_reference(args, shape, inp, workload):
     """--impl reference: the oracle is the timed arm (bounded sample per step)."""
-    sample_T = min(shape.T, 256)
+    sample_T = min(shape.T, 2048)
     for _ in range(min(args.warmup, 1)):
         oracle_sample_tokens_per_s(inp, shape, sample_T)
     times = []
