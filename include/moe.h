@@ -96,6 +96,13 @@ MOE_API const char* moe_status_string(moe_status s);
 /* Synchronises the stream and returns the device-side status word of the workspace. */
 MOE_API moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_stream);
 
+/* Exercises the device-side failure path without faulting anything: launches one tiny kernel whose bounded wait
+ * (on a barrier nothing signals) runs out after a few thousand polls; the kernel records the timeout in the
+ * workspace's status word and returns.  A following moe_poll_status reports MOE_ERR_DEVICE_TIMEOUT; the context
+ * stays usable and the next moe_forward clears the word.  The layer's kernels bound every wait the same way
+ * (about a second); nothing in the library makes a GPU fault, trap or hang on purpose. */
+MOE_API moe_status moe_selftest_timeout(moe_ctx* ctx, void* workspace, void* cuda_stream);
+
 /* Per-stage timing.  With enable != 0, moe_forward / moe_backward record CUDA events between their
  * kernels on the caller's stream, one event set per forward+backward pair, in a ring of MOE_PROF_RING sets.
  * moe_stage_times waits for the recorded events, ADDS to ms[s] (host array of MOE_NUM_STAGES floats) the

@@ -15,7 +15,7 @@ STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine"
                "unpermute_bwd"]
 EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
-           "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static"]
+           "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout"]
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -63,6 +63,8 @@ def load_library() -> C.CDLL:
     lib.moe_e2e_device_bytes.restype = sz
     lib.moe_step_host.argtypes = [vp, i64, C.c_int] + [vp] * 6 + [C.c_float] + [vp] * 7 + [vp, sz, vp]
     lib.moe_step_host.restype = C.c_int
+    lib.moe_selftest_timeout.argtypes = [vp, vp, vp]
+    lib.moe_selftest_timeout.restype = C.c_int
     lib.moe_router_wgrad_static.argtypes = [i64, C.c_int32, C.c_int32, vp, vp, vp, vp]
     lib.moe_router_wgrad_static.restype = C.c_int
     _lib = lib
@@ -207,6 +209,10 @@ class MoELayer:
     def poll(self) -> None:
         """Synchronises and raises if a device-side bounded wait ran out."""
         _check(self.lib, self.lib.moe_poll_status(self.h, _ptr(self.ws), self._stream()), "device status")
+
+    def selftest_timeout(self) -> None:
+        """Launches the kernel whose bounded wait runs out (see moe_selftest_timeout); poll() then raises."""
+        _check(self.lib, self.lib.moe_selftest_timeout(self.h, _ptr(self.ws), self._stream()), "moe_selftest_timeout")
 
     def set_profiling(self, on: bool) -> None:
         _check(self.lib, self.lib.moe_set_profiling(self.h, 1 if on else 0), "moe_set_profiling")

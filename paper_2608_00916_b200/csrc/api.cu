@@ -200,6 +200,41 @@ moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_strea
   return st[0] == DEV_OK ? MOE_OK : MOE_ERR_DEVICE_TIMEOUT;
 }
 
+// One CTA waits, with the library's bounded-wait helper cut down to a few thousand polls, on an mbarrier that
+// nothing ever signals; the wait gives up, records DEV_TIMEOUT in the status word and the kernel returns normally.
+__global__ void selftest_timeout_kernel(int32_t* status) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = static_cast<uint32_t>(__cvta_generic_to_shared(&bar));
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
+    bool done = false;
+    for (int i = 0; i < 4096 && !done; ++i) {
+      uint32_t ok;
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t"
+          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(ok)
+          : "r"(b), "r"(0u)
+          : "memory");
+      done = ok != 0;
+    }
+    if (!done) {
+      atomicExch(status, DEV_TIMEOUT);
+      status[1] = 9000;
+    }
+  }
+}
+
+moe_status moe_selftest_timeout(moe_ctx* ctx, void* workspace, void* cuda_stream) {
+  if (!ctx || !workspace) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  const WsLayout L = make_layout(c->s, 0);
+  selftest_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + L.status));
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
 moe_status moe_set_profiling(moe_ctx* ctx, int enable) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);

@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
         }
         t_wait += clock64() - w0;
         if (lane == 0) {
-          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          mbar_expect_tx(full_bar(s), p.stage_tx);
           const uint32_t sA = smem_base + s * STAGE_BYTES;
           issue_loads<KIND>(p, tl, kb, sA, sA + A_BYTES, full_bar(s));
         }
@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc = umma_idesc(BM, BN, TR::A_MN, TR::B_MN);
+    const uint32_t idesc = umma_idesc(BM, KIND == GEMM_RT ? p.mma_n : BN, TR::A_MN, TR::B_MN);
     constexpr uint32_t A_LBO = TR::A_MN ? CHUNK_BYTES : 0, B_LBO = TR::B_MN ? CHUNK_BYTES : 0;
     constexpr uint32_t A_KSTEP = TR::A_MN ? 2048 : 32, B_KSTEP = TR::B_MN ? 2048 : 32;  // bytes per K = 16
     uint32_t it = 0, tc = 0;
@@ -203,99 +203,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
                               TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
                               es, lane);
       } else if (KIND == GEMM_RT) {
-        // Routing epilogue: one thread per token; the row of E logits is re-read from tensor memory in every
-        // pass.  Pass j picks the largest logit that comes after pick j-1 in the order (value descending,
-        // index ascending), which is the rule "largest not taken yet, lowest index among equals".
-        const int64_t tok = row;
-        const bool valid = tok < p.T;
-        const int E = p.N_total, k = p.top_k;
-        const int nch = (E + 31) >> 5;
-        float selv[MAX_K];
-        int seli[MAX_K];
-        float pv = INFINITY;
-        int pi = -1;
-        for (int j = 0; j < k; ++j) {
-          float bv = -INFINITY;
-          int bi = 0x7FFFFFFF;
-          for (int c = 0; c < nch; ++c) {
-            uint32_t r[32];
-            tmem_ld32(taddr + c * 32, r);
-            tmem_ld_wait();
-            float val[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) val[i] = __uint_as_float(r[i]) + s_bias[c * 32 + i];
-            if (j == 0 && valid) {
-#pragma unroll
-              for (int i = 0; i < 32; i += 4) {
-                if (c * 32 + i < E) {
-                  const float4 w = make_float4(val[i], val[i + 1], val[i + 2], val[i + 3]);
-                  *reinterpret_cast<float4*>(p.logits + tok * E + c * 32 + i) = w;
-                  if (p.logits_out) *reinterpret_cast<float4*>(p.logits_out + tok * E + c * 32 + i) = w;
-                }
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int e = c * 32 + i;
-              const bool after = (val[i] < pv) || (val[i] == pv && e > pi);
-              if (e < E && after && val[i] > bv) {
-                bv = val[i];
-                bi = e;
-              }
-            }
-          }
-          selv[j] = bv;
-          seli[j] = bi;
-          pv = bv;
-          pi = bi;
-        }
-        const float vmax = selv[0];
-        float z = 0.f;
-        for (int c = 0; c < nch; ++c) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c * 32, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c * 32 + i < E) z += expf(__uint_as_float(r[i]) + s_bias[c * 32 + i] - vmax);
-        }
-        const float rz = valid ? 1.f / z : 0.f;
-        for (int c = 0; c < nch; ++c) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c * 32, r);
-          tmem_ld_wait();
-          float pc[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            pc[i] = (c * 32 + i < E) ? expf(__uint_as_float(r[i]) + s_bias[c * 32 + i] - vmax) * rz : 0.f;
-          // column sums over the 32 tokens of this warp: butterfly transpose-reduce, lane L ends with column L
-#pragma unroll
-          for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              if (i < cnt) {
-                const bool up = (lane & off) != 0;
-                const float send = up ? pc[i] : pc[i + cnt];
-                const float keep = up ? pc[i + cnt] : pc[i];
-                pc[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
-              }
-            }
-          }
-          if (c * 32 + lane < E)
-            p.psum_part[(static_cast<int64_t>(tl.row0 / BM) * 4 + ew) * E + c * 32 + lane] = pc[0];
-        }
-        if (valid) {
-          float zs = 0.f;
-          for (int j = 0; j < k; ++j) zs += expf(selv[j] - vmax);
-          const float rzs = 1.f / zs;
-          for (int j = 0; j < k; ++j) {
-            const float g = expf(selv[j] - vmax) * rzs;
-            p.idx[tok * k + j] = seli[j];
-            p.gates[tok * k + j] = g;
-            p.idx_out[tok * k + j] = seli[j];
-            p.gates_out[tok * k + j] = g;
-          }
-        }
+        if (p.N_total <= 128)
+          routing_epilogue_regs(p, s_bias, row, tl.row0 / BM, ew, taddr, lane);
+        else
+          routing_epilogue_tmem(p, s_bias, row, tl.row0 / BM, ew, taddr, lane);
       } else if (KIND == GEMM_DWR) {
         // fp32 partial of dW_r for this token slice: hi and lo halves of dl share one accumulator pair
         const int m = tl.m0 + rin;
@@ -414,6 +325,9 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   const bool pair = !ctx->single_cta;  // expert GEMMs on CTA pairs (256 x 256 tiles)
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
+  p.b_chunks = 4;
+  p.mma_n = BN;
+  p.stage_tx = STAGE_BYTES;
   bool ok = true;
   switch (kind) {
     case GEMM_F3:
@@ -496,6 +410,9 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.n_tiles = 1;
       p.k_blocks = d / BK;
       p.N_total = E;
+      p.b_chunks = (E + 63) / 64;
+      p.mma_n = (E + 15) / 16 * 16;
+      p.stage_tx = A_BYTES + p.b_chunks * CHUNK_BYTES;
       p.T = T;
       p.top_k = s.k;
       p.bias = io.b_r;

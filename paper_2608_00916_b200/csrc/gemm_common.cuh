@@ -45,6 +45,9 @@ struct GemmParams {
   int64_t ld_out;
   int64_t expert_stride;
   // router kinds
+  int b_chunks;         // RT: 64-column chunks of W_r actually loaded (ceil(E / 64))
+  int mma_n;            // RT: N of the MMA (E rounded up to 16)
+  uint32_t stage_tx;    // bytes one stage's loads deliver (RT loads fewer B chunks)
   int static_m_tiles;   // RT, DX: number of 128-token tiles
   int split_rows;       // DWR: tokens per slice (multiple of 64)
   int rows_total;       // DWR: tokens rounded up to 64
@@ -148,7 +151,9 @@ __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl,
     if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
     if (DO_B) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+      for (int c = 0; c < 4; ++c)
+        if (KIND != GEMM_RT || c < p.b_chunks)
+          tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
     }
   } else if (KIND == GEMM_B2) {
     if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
@@ -396,6 +401,202 @@ __device__ __forceinline__ void wgrad_zero_fill(const GemmParams& p, int e, int 
       col = n0 + (c & 3) * 32;
     }
     if (col < p.N_total) store_bf16x32(base + e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, z);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- routing epilogues
+// One thread per token (TMEM lane).  Pass j picks the largest logit that comes after pick j-1 in the order (value
+// descending, index ascending), which is the rule "largest not taken yet, lowest index among equals" without a
+// "taken" mask.  Gates are the softmax over the picked logits; the softmax over all E logits is summed per
+// column with a butterfly transpose-reduce (lane L ends with column L), one partial row per warp, fixed order.
+//
+// Generic version (any E <= 256): the row of logits is re-read from tensor memory in every pass.
+__device__ __forceinline__ void routing_epilogue_tmem(const GemmParams& p, const float* s_bias, int64_t row, int tile,
+                                                      int ew, uint32_t taddr, int lane) {
+        const int64_t tok = row;
+        const bool valid = tok < p.T;
+        const int E = p.N_total, k = p.top_k;
+        const int nch = (E + 31) >> 5;
+        float selv[MAX_K];
+        int seli[MAX_K];
+        float pv = INFINITY;
+        int pi = -1;
+        for (int j = 0; j < k; ++j) {
+          float bv = -INFINITY;
+          int bi = 0x7FFFFFFF;
+          for (int c = 0; c < nch; ++c) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_ld_wait();
+            float val[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) val[i] = __uint_as_float(r[i]) + s_bias[c * 32 + i];
+            if (j == 0 && valid) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4) {
+                if (c * 32 + i < E) {
+                  const float4 w = make_float4(val[i], val[i + 1], val[i + 2], val[i + 3]);
+                  *reinterpret_cast<float4*>(p.logits + tok * E + c * 32 + i) = w;
+                  if (p.logits_out) *reinterpret_cast<float4*>(p.logits_out + tok * E + c * 32 + i) = w;
+                }
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int e = c * 32 + i;
+              const bool after = (val[i] < pv) || (val[i] == pv && e > pi);
+              if (e < E && after && val[i] > bv) {
+                bv = val[i];
+                bi = e;
+              }
+            }
+          }
+          selv[j] = bv;
+          seli[j] = bi;
+          pv = bv;
+          pi = bi;
+        }
+        const float vmax = selv[0];
+        float z = 0.f;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i < E) z += expf(__uint_as_float(r[i]) + s_bias[c * 32 + i] - vmax);
+        }
+        const float rz = valid ? 1.f / z : 0.f;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+          float pc[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            pc[i] = (c * 32 + i < E) ? expf(__uint_as_float(r[i]) + s_bias[c * 32 + i] - vmax) * rz : 0.f;
+          // column sums over the 32 tokens of this warp: butterfly transpose-reduce, lane L ends with column L
+#pragma unroll
+          for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              if (i < cnt) {
+                const bool up = (lane & off) != 0;
+                const float send = up ? pc[i] : pc[i + cnt];
+                const float keep = up ? pc[i + cnt] : pc[i];
+                pc[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
+              }
+            }
+          }
+          if (c * 32 + lane < E)
+            p.psum_part[(static_cast<int64_t>(tile) * 4 + ew) * E + c * 32 + lane] = pc[0];
+        }
+        if (valid) {
+          float zs = 0.f;
+          for (int j = 0; j < k; ++j) zs += expf(selv[j] - vmax);
+          const float rzs = 1.f / zs;
+          for (int j = 0; j < k; ++j) {
+            const float g = expf(selv[j] - vmax) * rzs;
+            p.idx[tok * k + j] = seli[j];
+            p.gates[tok * k + j] = g;
+            p.idx_out[tok * k + j] = seli[j];
+            p.gates_out[tok * k + j] = g;
+          }
+        }
+}
+
+// E <= 128: the whole row of logits stays in registers (one TMEM read), exponentials use the fast intrinsic.
+__device__ __forceinline__ void routing_epilogue_regs(const GemmParams& p, const float* s_bias, int64_t row, int tile,
+                                                      int ew, uint32_t taddr, int lane) {
+  const int64_t tok = row;
+  const bool valid = tok < p.T;
+  const int E = p.N_total, k = p.top_k;
+  float v[128];
+  {
+    uint32_t r0[32], r1[32], r2[32], r3[32];
+    tmem_ld32(taddr, r0);
+    tmem_ld32(taddr + 32, r1);
+    tmem_ld32(taddr + 64, r2);
+    tmem_ld32(taddr + 96, r3);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      v[i] = __uint_as_float(r0[i]) + s_bias[i];
+      v[32 + i] = __uint_as_float(r1[i]) + s_bias[32 + i];
+      v[64 + i] = __uint_as_float(r2[i]) + s_bias[64 + i];
+      v[96 + i] = __uint_as_float(r3[i]) + s_bias[96 + i];
+    }
+  }
+  if (valid) {
+#pragma unroll
+    for (int i = 0; i < 128; i += 4) {
+      if (i < E) {
+        const float4 w = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        *reinterpret_cast<float4*>(p.logits + tok * E + i) = w;
+        if (p.logits_out) *reinterpret_cast<float4*>(p.logits_out + tok * E + i) = w;
+      }
+    }
+  }
+  float selv[MAX_K];
+  int seli[MAX_K];
+  float pv = INFINITY;
+  int pi = -1;
+  for (int j = 0; j < k; ++j) {
+    float bv = -INFINITY;
+    int bi = 0x7FFFFFFF;
+#pragma unroll
+    for (int i = 0; i < 128; ++i) {
+      const bool after = (v[i] < pv) || (v[i] == pv && i > pi);
+      if (i < E && after && v[i] > bv) {
+        bv = v[i];
+        bi = i;
+      }
+    }
+    selv[j] = bv;
+    seli[j] = bi;
+    pv = bv;
+    pi = bi;
+  }
+  const float vmax = selv[0];
+  float z = 0.f;
+#pragma unroll
+  for (int i = 0; i < 128; ++i) {
+    v[i] = (i < E) ? __expf(v[i] - vmax) : 0.f;
+    z += v[i];
+  }
+  const float rz = valid ? 1.f / z : 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    if (c * 32 < E) {
+      float pc[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) pc[i] = v[c * 32 + i] * rz;
+#pragma unroll
+      for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          if (i < cnt) {
+            const bool up = (lane & off) != 0;
+            const float send = up ? pc[i] : pc[i + cnt];
+            const float keep = up ? pc[i + cnt] : pc[i];
+            pc[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
+          }
+        }
+      }
+      if (c * 32 + lane < E) p.psum_part[(static_cast<int64_t>(tile) * 4 + ew) * E + c * 32 + lane] = pc[0];
+    }
+  }
+  if (valid) {
+    float zs = 0.f;
+    for (int j = 0; j < k; ++j) zs += __expf(selv[j] - vmax);
+    const float rzs = 1.f / zs;
+    for (int j = 0; j < k; ++j) {
+      const float g = __expf(selv[j] - vmax) * rzs;
+      p.idx[tok * k + j] = seli[j];
+      p.gates[tok * k + j] = g;
+      p.idx_out[tok * k + j] = seli[j];
+      p.gates_out[tok * k + j] = g;
+    }
   }
 }
 

@@ -159,6 +159,49 @@ def test_repeated_calls_are_bitwise_reproducible():
         assert torch.equal(ga[n], gb[n]), n
 
 
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A device-side wait that can never complete gives up, the status word says so, and the same context and
+    workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
+    from paper_2608_00916_b200.binding import MoEError
+    inp = synth.make_inputs(synth.MoEShape(300, 128, 8, 2, 128), 25)
+    ofw, obw = oracle_run(inp, 2, 0.0)
+    r = Run(inp, 2)
+    r.forward()  # allocates the workspace, status ok
+    r.layer.selftest_timeout()
+    with pytest.raises(MoEError, match="bounded device-side wait"):
+        r.layer.poll()
+    fw = r.forward()  # clears the status word and runs normally
+    check_routing(fw, ofw)
+    assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+
+
+def test_forward_backward_replay_from_a_cuda_graph():
+    """Neither call synchronises, allocates or reads anything back, so a forward + backward pair can be captured
+    into a CUDA graph (after one eager call has set the kernels' attributes) and replayed: same bits as eager."""
+    inp = synth.make_inputs(synth.MoEShape(512, 256, 16, 4, 256), 26)
+    r = Run(inp, 4)
+    v = r.dev
+    eager_fw = r.layer.forward(v["x"], v["W_r"], v["W_gate"], v["W_up"], v["W_down"])
+    eager_bw = r.layer.backward(v["dy"], 0.03)
+    torch.cuda.synchronize()
+    keep = {n: eager_fw[n].clone() for n in ("y", "idx", "gates", "aux")} | {n: eager_bw[n].clone() for n in ("dx", "dW_r", "dW_gate")}
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            gfw = r.layer.forward(v["x"], v["W_r"], v["W_gate"], v["W_up"], v["W_down"])
+            gbw = r.layer.backward(v["dy"], 0.03)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    r.layer.poll()
+    for n in ("y", "idx", "gates", "aux"):
+        assert torch.equal(gfw[n], keep[n]), n
+    for n in ("dx", "dW_r", "dW_gate"):
+        assert torch.equal(gbw[n], keep[n]), n
+
+
 def test_midsize_qwen_shape_full_oracle():
     """The Qwen3-30B-A3B expert shape with fewer tokens, full oracle in float32 mode."""
     shape = synth.MoEShape(2048, 2048, 128, 8, 768)
