@@ -51,14 +51,15 @@ typedef struct {
   int32_t E;      /* experts,      1 <= E <= 256                                   */
   int32_t f;      /* expert width, multiple of 64                                  */
   int32_t top_k;  /* experts per token, 1 <= top_k <= E and top_k <= 32            */
-  int32_t flags;  /* 0, or MOE_FLAG_CTA_PAIR_TILES                                 */
+  int32_t flags;  /* 0, or one of the MOE_FLAG_* tile flags                        */
 } moe_config;
 
-/* Runs the expert GEMMs on CTA pairs (256 x 256 tiles, tcgen05 cta_group::2, each CTA staging half of B) instead
- * of the default one-CTA 128 x 256 tiles.  Same results.  On the Qwen3-30B-A3B shape the pairs are not faster
- * (their dummy half-tiles for experts with an odd number of 128-row blocks cost what the halved B traffic saves),
- * so they are an option, not the default. */
+/* Tile shape of the expert GEMMs.  By default the library chooses per GEMM: weight gradients run on CTA pairs
+ * (256 x 256 tiles, tcgen05 cta_group::2, each CTA staging half of B), row GEMMs run on pairs when few experts share
+ * many rows (the dummy half-tile of an expert with an odd number of 128-row blocks then costs < 3 %) and on one-CTA
+ * 128 x 256 tiles otherwise.  The flags force one shape everywhere (same results; for comparison measurements). */
 #define MOE_FLAG_CTA_PAIR_TILES 1
+#define MOE_FLAG_SINGLE_CTA_TILES 2
 
 typedef struct moe_ctx moe_ctx; /* opaque, lives in host memory */
 

@@ -9,7 +9,8 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
 NUM_STAGES = 16
-FLAG_CTA_PAIR_TILES = 1  # MOE_FLAG_CTA_PAIR_TILES of include/moe.h
+FLAG_CTA_PAIR_TILES = 1    # MOE_FLAG_CTA_PAIR_TILES of include/moe.h
+FLAG_SINGLE_CTA_TILES = 2  # MOE_FLAG_SINGLE_CTA_TILES
 STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine", "combine_bwd",
                "dgrad_down_swiglu_bwd", "wgrad_down", "dgrad_gateup", "wgrad_gateup", "router_bwd", "dW_r",
                "unpermute_bwd"]

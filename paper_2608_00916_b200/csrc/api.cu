@@ -112,7 +112,7 @@ moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
   if (!c) return MOE_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
   c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
-  c->single_cta = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 0 : 1;
+  c->tile_mode = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 1 : ((cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 2 : 0);
   *out = reinterpret_cast<moe_ctx*>(c);
   return MOE_OK;
 }

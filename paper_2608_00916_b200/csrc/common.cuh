@@ -70,7 +70,7 @@ struct moe_ctx_impl {
   int sm_count;
   int device;
   void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
-  int single_cta;   // 1: expert GEMMs on one-CTA tiles (128 x 256) instead of CTA pairs (256 x 256)
+  int tile_mode;    // 0: choose per GEMM (see use_pair_tiles), 1: always CTA pairs, 2: always one-CTA tiles
   int profiling;
   cudaEvent_t ev[MOE_PROF_RING][MOE_NUM_STAGES][2];
   unsigned char ev_used[MOE_PROF_RING][MOE_NUM_STAGES];

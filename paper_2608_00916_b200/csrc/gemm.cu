@@ -322,7 +322,14 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
   p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
   p.timers = getenv("MOE_GEMM_TIMERS") ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
-  const bool pair = !ctx->single_cta;  // expert GEMMs on CTA pairs (256 x 256 tiles)
+  // CTA pairs (256 x 256 tiles, half of B per SM) or one-CTA tiles (128 x 256)?  Pairs move a third less operand
+  // data per flop, which under the power cap is worth ~12 % on long-K shapes; their cost is the dummy half-tile of
+  // every expert with an odd number of 128-row blocks (row GEMMs only).  Weight gradients pair along the weight
+  // dimension and have no such waste, so they always pair; row GEMMs pair when the expected waste (64 rows per
+  // expert) stays under 3 % of the routed rows.
+  const bool wgrad_kind = kind == GEMM_B3 || kind == GEMM_B5;
+  const bool pair = ctx->tile_mode == 1 ||
+                    (ctx->tile_mode == 0 && (wgrad_kind || 64.0 * E < 0.03 * static_cast<double>(T) * s.k));
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
   p.b_chunks = 4;

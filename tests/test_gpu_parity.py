@@ -88,14 +88,15 @@ def test_odd_shapes(T, d, E, k, f, seed):
     check_all(Run(inp, k), ofw, obw, 0.05)
 
 
+@pytest.mark.parametrize("flag", [1, 2])
 @pytest.mark.parametrize("T,d,E,k,f,seed", [(1000, 512, 16, 4, 384, 14), (333, 192, 5, 5, 320, 15), (2049, 256, 32, 8, 128, 17)])
-def test_cta_pair_tiles_option(T, d, E, k, f, seed):
-    """The cta_group::2 variant of the expert GEMMs (pairs of CTAs on 256-row tiles) gives the same results."""
-    from paper_2608_00916_b200.binding import FLAG_CTA_PAIR_TILES
+def test_forced_tile_shapes(T, d, E, k, f, seed, flag):
+    """Forcing CTA pairs (cta_group::2, 256-row tiles; flag 1) or one-CTA tiles (flag 2) for every expert GEMM gives
+    the same results as the default per-GEMM choice."""
     shape = synth.MoEShape(T, d, E, k, f)
     inp = synth.make_inputs(shape, seed, x_std=1.0)
     ofw, obw = oracle_run(inp, k, 0.05)
-    check_all(Run(inp, k, flags=FLAG_CTA_PAIR_TILES), ofw, obw, 0.05)
+    check_all(Run(inp, k, flags=flag), ofw, obw, 0.05)
 
 
 def test_skewed_small_with_bias_and_empty_experts():
