@@ -84,7 +84,7 @@ MOE_API void moe_destroy(moe_ctx* ctx);
 MOE_API size_t moe_workspace_bytes(const moe_ctx* ctx, int64_t T);
 
 /* Byte offset and size of a named internal buffer inside the workspace, for stage-by-stage tests.
- * Names: "counts" "offsets" "pad_offsets" "logits" "idx" "gates" "inv" "row_token" "xp" "hg" "hu" "act"
+ * Names: "counts" "offsets" "pad_offsets" "logits" "idx" "gates" "inv" "row_gate" "xp" "hg" "hu" "act"
  * "o" "dhg" "dhu" "dxp" "dg" "dl".  Internal row buffers (xp, hg, hu, act, o, dhg, dhu, dxp) are laid out
  * expert-major with every expert's segment padded to a multiple of 128 rows ("pad_offsets"); pad rows
  * are zero.  "act" and "o" are stored already multiplied by the row's gate (so the combine is a plain sum); after

@@ -39,7 +39,6 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.idx = take(sizeof(int32_t) * R);
   L.gates = take(sizeof(float) * R);
   L.inv = take(sizeof(int32_t) * R);
-  L.row_token = take(sizeof(int32_t) * L.rows_max);
   L.row_gate = take(sizeof(float) * L.rows_max);
   L.dg_part = take(sizeof(float) * ((s.f + 255) / 256) * L.rows_max);
   L.dg = take(sizeof(float) * R);
@@ -152,7 +151,7 @@ moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char* name, s
              {"idx", L.idx, sizeof(int32_t) * R},
              {"gates", L.gates, sizeof(float) * R},
              {"inv", L.inv, sizeof(int32_t) * R},
-             {"row_token", L.row_token, sizeof(int32_t) * L.rows_max},
+             {"row_gate", L.row_gate, sizeof(float) * L.rows_max},
              {"xp", L.xp, rows_d},
              {"hg", L.hg, rows_f},
              {"hu", L.hu, rows_f},
@@ -362,7 +361,7 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   const bool tc_router = router_on_tensor_cores(s);
   if (T > 0) {
     StageTimer tm(c, st, 5);
-    launch_gather_rows(s, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st);
+    launch_gather_rows(s, T, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st);
   }
   if (T > 0) {
     StageTimer tm(c, st, 6);

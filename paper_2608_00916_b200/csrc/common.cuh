@@ -43,7 +43,6 @@ struct WsLayout {
   size_t idx;          // int32[T*k]
   size_t gates;        // float[T*k]
   size_t inv;          // int32[T*k]  padded row of pair (t, j)
-  size_t row_token;    // int32[rows_max] token of a padded row, -1 for pad rows
   size_t row_gate;     // float[rows_max] gate of a padded row, 0 for pad rows
   size_t dg_part;      // float[ceil(f/256) * rows_max] per-row partial sums of dg, one slice per dgrad-down column tile
   size_t dg;           // float[T*k]
@@ -88,9 +87,9 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
 // ---- launchers (combine.cu)
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
                     uint16_t* y, cudaStream_t st);
-// rows[r,:] = src[row_token[r],:] (zero for pad rows) for every padded row: xp from x, and the dy rows of backward
-void launch_gather_rows(const Shape& s, const WsLayout& L, const char* ws, const uint16_t* src, uint16_t* rows,
-                        cudaStream_t st);
+// rows[inv[t,j],:] = src[t,:] for every (token, slot), pad rows zeroed: xp from x, and the dy rows of backward
+void launch_gather_rows(const Shape& s, int64_t T, const WsLayout& L, const char* ws, const uint16_t* src,
+                        uint16_t* rows, cudaStream_t st);
 // dg[t,j] = sum over column tiles of dg_part[tile][inv[t,j]], then dl (fp32 and the two-term bf16 split)
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
                        const float* dg_part, int dg_tiles, int64_t rows_max, const int32_t* inv, float* dg,

@@ -253,9 +253,15 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
   const int G = SCAN_THREADS / E;
   if (tid < G * E) {
     const int g = tid / E, e = tid - g * E;
-    float ps = 0.f;
-    for (int b = g; b < psum_rows; b += G) ps += psum_part[static_cast<int64_t>(b) * E + e];
-    s_ps[tid] = ps;
+    // eight loads in flight per thread; the partial sums are combined in a fixed order
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    int b = g;
+    for (; b + 7 * G < psum_rows; b += 8 * G) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc[u] += psum_part[static_cast<int64_t>(b + u * G) * E + e];
+    }
+    for (; b < psum_rows; b += G) acc[0] += psum_part[static_cast<int64_t>(b) * E + e];
+    s_ps[tid] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
   }
   __syncthreads();
   // exclusive prefix of every expert's column of tile_counts along the tiles: one warp per expert, 32 tiles per step
@@ -334,7 +340,7 @@ __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int
                                                            const int32_t* __restrict__ offsets,
                                                            const int32_t* __restrict__ pad_offsets,
                                                            const float* __restrict__ gates,
-                                                           int32_t* __restrict__ inv, int32_t* __restrict__ row_token,
+                                                           int32_t* __restrict__ inv,
                                                            float* __restrict__ row_gate,
                                                            int32_t* __restrict__ perm_out) {
   extern __shared__ uint32_t sc_masks[];
@@ -350,55 +356,63 @@ __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int
     rank += __popc(sc_masks[warp * E + e] & ((1u << lane) - 1u));
     const int r = pad_offsets[e] + rank;
     inv[t * k + j] = r;
-    row_token[r] = static_cast<int32_t>(t);
     row_gate[r] = gates[t * k + j];
     if (perm_out) perm_out[offsets[e] + rank] = static_cast<int32_t>(t * k + j);
   }
 }
 
-// rows[r,:] = src[row_token[r],:], zero for pad rows.  One warp per row; a lane keeps four 16-byte loads in
-// flight before it stores.
-__global__ void __launch_bounds__(256) gather_rows_kernel(int d, const uint16_t* __restrict__ src,
-                                                          const int32_t* __restrict__ row_token,
-                                                          const int32_t* __restrict__ sched,
-                                                          uint16_t* __restrict__ rows) {
-  const int lane = threadIdx.x & 31;
-  const int64_t r = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
-  if (r >= sched[1]) return;
-  const int t = row_token[r];
-  uint4* dst = reinterpret_cast<uint4*>(rows + r * d);
+// rows[inv[t,j],:] = src[t,:] for every (token, slot), and zero for the pad rows of every expert segment.
+// One warp per token: the token's row is read ONCE into registers and written to its k destination rows (a
+// gather by destination row re-reads each source row k times at far-apart moments; with the 0.5 GB output stream
+// flowing through L2 in between, those re-reads came from DRAM: 328 MB read instead of 67 MB at the Qwen shape).
+// Blocks past the token range zero the pad rows, one expert per block.
+__global__ void __launch_bounds__(256) scatter_rows_kernel(int64_t T, int d, int k, int E, int tok_blocks,
+                                                           const uint16_t* __restrict__ src,
+                                                           const int32_t* __restrict__ inv,
+                                                           const int32_t* __restrict__ counts,
+                                                           const int32_t* __restrict__ pad_offsets,
+                                                           uint16_t* __restrict__ rows) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n16 = d / 8;
-  if (t < 0) {
-    for (int i = lane; i < n16; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
-  } else {
-    const uint4* s4 = reinterpret_cast<const uint4*>(src + static_cast<int64_t>(t) * d);
-    int i = lane;
-    for (; i + 96 < n16; i += 128) {
-      const uint4 a = __ldg(s4 + i), b = __ldg(s4 + i + 32), c = __ldg(s4 + i + 64), e = __ldg(s4 + i + 96);
-      dst[i] = a;
-      dst[i + 32] = b;
-      dst[i + 64] = c;
-      dst[i + 96] = e;
+  if (static_cast<int>(blockIdx.x) >= tok_blocks) {
+    const int e = blockIdx.x - tok_blocks;
+    const int64_t r0 = static_cast<int64_t>(pad_offsets[e]) + counts[e], r1 = pad_offsets[e + 1];
+    uint4* dst = reinterpret_cast<uint4*>(rows + r0 * d);
+    const int64_t n = (r1 - r0) * n16;
+    for (int64_t i = threadIdx.x; i < n; i += 256) dst[i] = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * 8 + warp;
+  if (t >= T) return;
+  const uint4* s4 = reinterpret_cast<const uint4*>(src + t * d);
+  for (int c0 = 0; c0 < n16; c0 += 256) {  // 256 x 16 B = 4 KB of the row per pass, 8 pieces per lane
+    uint4 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (c0 + lane + 32 * i < n16) v[i] = __ldg(s4 + c0 + lane + 32 * i);
+    for (int j = 0; j < k; ++j) {
+      uint4* dst = reinterpret_cast<uint4*>(rows + static_cast<int64_t>(inv[t * k + j]) * d);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (c0 + lane + 32 * i < n16) dst[c0 + lane + 32 * i] = v[i];
     }
-    for (; i < n16; i += 32) dst[i] = __ldg(s4 + i);
   }
 }
 
-void launch_gather_rows(const Shape& s, const WsLayout& L, const char* ws, const uint16_t* src, uint16_t* rows,
-                        cudaStream_t st) {
-  const int gblocks = static_cast<int>((L.rows_max + 7) / 8);
-  gather_rows_kernel<<<gblocks, 256, 0, st>>>(s.d, src, reinterpret_cast<const int32_t*>(ws + L.row_token),
-                                              reinterpret_cast<const int32_t*>(ws + L.sched), rows);
+void launch_gather_rows(const Shape& s, int64_t T, const WsLayout& L, const char* ws, const uint16_t* src,
+                        uint16_t* rows, cudaStream_t st) {
+  const int tok_blocks = static_cast<int>((T + 7) / 8);
+  scatter_rows_kernel<<<tok_blocks + s.E, 256, 0, st>>>(
+      T, s.d, s.k, s.E, tok_blocks, src, reinterpret_cast<const int32_t*>(ws + L.inv),
+      reinterpret_cast<const int32_t*>(ws + L.counts), reinterpret_cast<const int32_t*>(ws + L.pad_offsets), rows);
 }
 
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
                     int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st) {
   int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
   int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
-  int32_t* row_token = reinterpret_cast<int32_t*>(ws + L.row_token);
   const int tiles = static_cast<int>(L.tok_tiles);
   const size_t msm = sizeof(uint32_t) * 8 * s.E;
-  cudaMemsetAsync(row_token, 0xFF, sizeof(int32_t) * L.rows_max, st);
   cudaMemsetAsync(ws + L.row_gate, 0, sizeof(float) * L.rows_max, st);
   if (tiles > 0) hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
   scan_kernel<<<1, SCAN_THREADS, 0, st>>>(T, s.E, s.k, tiles, psum_rows, tile_counts,
@@ -415,8 +429,8 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
     scatter_kernel<<<tiles, TOK_TILE, msm, st>>>(
         T, s.E, s.k, idx, tile_counts, reinterpret_cast<const int32_t*>(ws + L.offsets),
         reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const float*>(ws + L.gates),
-        reinterpret_cast<int32_t*>(ws + L.inv), row_token, reinterpret_cast<float*>(ws + L.row_gate), perm_out);
-    launch_gather_rows(s, L, ws, x, reinterpret_cast<uint16_t*>(ws + L.xp), st);
+        reinterpret_cast<int32_t*>(ws + L.inv), reinterpret_cast<float*>(ws + L.row_gate), perm_out);
+    launch_gather_rows(s, T, L, ws, x, reinterpret_cast<uint16_t*>(ws + L.xp), st);
   }
 }
 

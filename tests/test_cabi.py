@@ -59,7 +59,7 @@ def test_workspace_arithmetic(lib):
         layer.find(T, "nonsense")
     # regions do not overlap
     spans = sorted(layer.find(T, nm) for nm in ("counts", "offsets", "pad_offsets", "logits", "idx", "gates", "inv",
-                                                 "row_token", "xp", "hg", "hu", "act", "o", "dhg", "dhu", "dxp", "dg",
+                                                 "row_gate", "xp", "hg", "hu", "act", "o", "dhg", "dhu", "dxp", "dg",
                                                  "dl"))
     for (o1, n1), (o2, _) in zip(spans, spans[1:]):
         assert o1 + n1 <= o2
