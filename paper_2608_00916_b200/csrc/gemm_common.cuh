@@ -537,25 +537,44 @@ __device__ __forceinline__ void routing_epilogue_regs(const GemmParams& p, const
       }
     }
   }
+  // Top-k by k rounds of (max value, lowest index attaining it, remove it).  Only one warp per scheduler runs this
+  // code, so it is written for instruction-level parallelism: the value maximum and the index minimum are
+  // FMNMX / IMNMX chains split four ways, everything else is independent per column; no predicate feeds a
+  // loop-carried dependency (a compare-and-select chain took 56 cycles per column here).
+#pragma unroll
+  for (int i = 0; i < 128; ++i)
+    if (i >= E) v[i] = -INFINITY;  // columns beyond E can never be picked
   float selv[MAX_K];
   int seli[MAX_K];
-  float pv = INFINITY;
-  int pi = -1;
   for (int j = 0; j < k; ++j) {
-    float bv = -INFINITY;
-    int bi = 0x7FFFFFFF;
+    float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int i = 0; i < 128; ++i) {
-      const bool after = (v[i] < pv) || (v[i] == pv && i > pi);
-      if (i < E && after && v[i] > bv) {
-        bv = v[i];
-        bi = i;
-      }
-    }
-    selv[j] = bv;
+    for (int i = 0; i < 128; ++i) m[i & 3] = fmaxf(m[i & 3], v[i]);
+    const float best = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+    int q[4] = {0x7FFFFFFF, 0x7FFFFFFF, 0x7FFFFFFF, 0x7FFFFFFF};
+#pragma unroll
+    for (int i = 0; i < 128; ++i) q[i & 3] = min(q[i & 3], v[i] == best ? i : 0x7FFFFFFF);
+    const int bi = min(min(q[0], q[1]), min(q[2], q[3]));
+#pragma unroll
+    for (int i = 0; i < 128; ++i) v[i] = (i == bi) ? -INFINITY : v[i];
+    selv[j] = best;
     seli[j] = bi;
-    pv = bv;
-    pi = bi;
+  }
+  // the picks were removed from the register copy: read the row again for the softmax statistics
+  {
+    uint32_t r0[32], r1[32], r2[32], r3[32];
+    tmem_ld32(taddr, r0);
+    tmem_ld32(taddr + 32, r1);
+    tmem_ld32(taddr + 64, r2);
+    tmem_ld32(taddr + 96, r3);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      v[i] = __uint_as_float(r0[i]) + s_bias[i];
+      v[32 + i] = __uint_as_float(r1[i]) + s_bias[32 + i];
+      v[64 + i] = __uint_as_float(r2[i]) + s_bias[64 + i];
+      v[96 + i] = __uint_as_float(r3[i]) + s_bias[96 + i];
+    }
   }
   const float vmax = selv[0];
   float z = 0.f;
