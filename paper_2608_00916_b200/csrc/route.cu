@@ -269,17 +269,27 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
     const int lane = tid & 31, wid = tid >> 5;
     for (int e = wid; e < E; e += SCAN_THREADS / 32) {
       int run = 0;
-      for (int t0 = 0; t0 < tok_tiles; t0 += 32) {
-        const int tl = t0 + lane;
-        const int c = tl < tok_tiles ? tile_counts[static_cast<int64_t>(tl) * E + e] : 0;
-        int inc = c;
+      for (int tb = 0; tb < tok_tiles; tb += 256) {  // up to 8 steps of 32 tiles with all their loads in flight
+        int c[8];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const int v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
-          if (lane >= off) inc += v;
+        for (int u = 0; u < 8; ++u) {
+          const int tl = tb + 32 * u + lane;
+          c[u] = tl < tok_tiles ? tile_counts[static_cast<int64_t>(tl) * E + e] : 0;
         }
-        if (tl < tok_tiles) tile_counts[static_cast<int64_t>(tl) * E + e] = run + inc - c;
-        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int tl = tb + 32 * u + lane;
+          if (tb + 32 * u < tok_tiles) {
+            int inc = c[u];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+              const int v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+              if (lane >= off) inc += v;
+            }
+            if (tl < tok_tiles) tile_counts[static_cast<int64_t>(tl) * E + e] = run + inc - c[u];
+            run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+          }
+        }
       }
       if (lane == 0) s_cnt[e] = run;
     }
@@ -301,28 +311,59 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
     expert_order[rank] = e;
   }
   __syncthreads();
-  if (tid == 0) {
-    int off = 0, poff = 0, npair = 0;
-    float aux = 0.f;
-    for (int e = 0; e < E; ++e) {
-      offsets[e] = off;
-      pad_offsets[e] = poff;
-      s_pad[e] = poff;
-      s_pair[e] = npair;
-      const int blocks = (s_cnt[e] + ROW_PAD - 1) / ROW_PAD;
-      off += s_cnt[e];
-      poff += blocks * ROW_PAD;
-      npair += (blocks + 1) / 2;
-      aux += s_term[e];
+  if (tid < 32) {
+    // exclusive scans of counts, padded counts and block pairs over the experts: lane L owns experts 8L .. 8L+7
+    const int lane = tid;
+    int cn[8], pd[8], pr[8];
+    int scn = 0, spd = 0, spr = 0;
+    float sterm = 0.f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = lane * 8 + u;
+      const int cnt = e < E ? s_cnt[e] : 0;
+      const int blocks = (cnt + ROW_PAD - 1) / ROW_PAD;
+      cn[u] = scn;
+      pd[u] = spd;
+      pr[u] = spr;
+      scn += cnt;
+      spd += blocks * ROW_PAD;
+      spr += (blocks + 1) / 2;
+      sterm += e < E ? s_term[e] : 0.f;
     }
-    offsets[E] = off;
-    pad_offsets[E] = poff;
-    s_pad[E] = poff;
-    s_pair[E] = npair;
-    sched[0] = poff / ROW_PAD;
-    sched[1] = poff;
-    sched[2] = npair;
-    aux_out[0] = aux * static_cast<float>(E);
+    int icn = scn, ipd = spd, ipr = spr;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int a = __shfl_up_sync(0xFFFFFFFFu, icn, off), b = __shfl_up_sync(0xFFFFFFFFu, ipd, off),
+                c = __shfl_up_sync(0xFFFFFFFFu, ipr, off);
+      if (lane >= off) {
+        icn += a;
+        ipd += b;
+        ipr += c;
+      }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sterm += __shfl_xor_sync(0xFFFFFFFFu, sterm, off);  // fixed tree
+    const int bcn = icn - scn, bpd = ipd - spd, bpr = ipr - spr;  // exclusive bases of this lane
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int e = lane * 8 + u;
+      if (e < E) {
+        offsets[e] = bcn + cn[u];
+        pad_offsets[e] = bpd + pd[u];
+        s_pad[e] = bpd + pd[u];
+        s_pair[e] = bpr + pr[u];
+      }
+    }
+    if (lane == 31) {
+      offsets[E] = icn;
+      pad_offsets[E] = ipd;
+      s_pad[E] = ipd;
+      s_pair[E] = ipr;
+      sched[0] = ipd / ROW_PAD;
+      sched[1] = ipd;
+      sched[2] = ipr;
+      aux_out[0] = sterm * static_cast<float>(E);
+    }
   }
   __syncthreads();
   for (int e = tid; e < E; e += SCAN_THREADS) {
