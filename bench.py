@@ -171,6 +171,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="qwen", choices=list(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="train", choices=["train", "inference"],
+                    help="train: forward + backward (the headline metric); inference: forward-only entry point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -213,6 +215,37 @@ def main():
     grads = {"dx": torch.empty_like(tens["x"]), "dW_r": torch.empty(shape.d, shape.E, dtype=torch.float32, device="cuda"),
              "dW_gate": torch.empty_like(tens["W_gate"]), "dW_up": torch.empty_like(tens["W_up"]),
              "dW_down": torch.empty_like(tens["W_down"])}
+
+    if args.mode == "inference":
+        # forward-only scoring pass (a "next" row beyond the training step): own metric, device-resident timing only
+        def fstep():
+            layer.forward(tens["x"], tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], b_r=b_r, want_perm=False,
+                          inference=True)
+        for _ in range(args.warmup):
+            fstep()
+        layer.poll()
+        pdist.barrier()
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(args.steps):
+            fstep()
+        f1.record()
+        torch.cuda.synchronize()
+        pdist.barrier()
+        ms = pdist.max_over_ranks(f0.elapsed_time(f1)) / args.steps
+        if rank == 0:
+            fl = 6 * T * shape.k * shape.d * shape.f
+            print(json.dumps({"metric": "moe_layer_fwd_tokens_per_s", "value": world * T / (ms / 1e3), "unit": "tokens/s",
+                              "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                              "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                              "data": "synthetic", "config": {"workload": args.workload, "mode": "inference",
+                                                              "T_per_gpu": T, "d": shape.d, "E": shape.E,
+                                                              "top_k": shape.k, "f": shape.f},
+                              "grouped_gemm_useful_tflops_over_whole_pass": fl / (ms * 1e-3) / 1e12,
+                              "gpu_launches": 9 * args.steps}))
+        pdist.finish()
+        return
 
     def step():
         layer.forward(tens["x"], tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], b_r=b_r, want_perm=False)

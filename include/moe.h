@@ -140,6 +140,18 @@ MOE_API moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const
                        int32_t* expert_counts, int32_t* perm, float* aux_loss, float* logits_out,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Forward pass for inference / scoring (the paper's serving use, Section "Evaluation and serving": rerankers score
+ * query-passage pairs with forward passes only).  Same arguments and results as moe_forward, but the gate/up GEMM
+ * does not store its pre-activations, so 2 * T * top_k * f * 2 bytes less are written, the workspace only needs
+ * moe_inference_workspace_bytes(ctx, T) bytes (routing tables, xp, act, o) and it cannot feed moe_backward. */
+MOE_API size_t moe_inference_workspace_bytes(const moe_ctx* ctx, int64_t T);
+MOE_API moe_status moe_forward_inference(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r,
+                                         const float* b_r, const float* logits_in, const uint16_t* W_gate,
+                                         const uint16_t* W_up, const uint16_t* W_down, uint16_t* y,
+                                         int32_t* topk_idx, float* topk_w, int32_t* expert_counts, int32_t* perm,
+                                         float* aux_loss, float* logits_out, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream);
+
 /* Backward pass of the forward call that filled `workspace`.
  *   dy    [T,d] bf16 upstream gradient of y;  d_aux: host scalar, dLoss/d(aux_loss)
  *   x, W_r, W_gate, W_up, W_down: the forward inputs

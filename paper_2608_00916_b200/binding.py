@@ -16,7 +16,8 @@ STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine"
                "unpermute_bwd"]
 EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
-           "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout"]
+           "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout",
+           "moe_forward_inference", "moe_inference_workspace_bytes"]
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -58,6 +59,10 @@ def load_library() -> C.CDLL:
     lib.moe_stage_times.restype = C.c_int
     lib.moe_forward.argtypes = [vp, i64] + [vp] * 14 + [vp, sz, vp]
     lib.moe_forward.restype = C.c_int
+    lib.moe_forward_inference.argtypes = lib.moe_forward.argtypes
+    lib.moe_forward_inference.restype = C.c_int
+    lib.moe_inference_workspace_bytes.argtypes = [vp, i64]
+    lib.moe_inference_workspace_bytes.restype = sz
     lib.moe_backward.argtypes = [vp, i64, vp, C.c_float] + [vp] * 11 + [vp, sz, vp]
     lib.moe_backward.restype = C.c_int
     lib.moe_e2e_device_bytes.argtypes = [vp, i64]
@@ -129,6 +134,9 @@ class MoELayer:
     def workspace_bytes(self, T: int) -> int:
         return int(self.lib.moe_workspace_bytes(self.h, T))
 
+    def inference_workspace_bytes(self, T: int) -> int:
+        return int(self.lib.moe_inference_workspace_bytes(self.h, T))
+
     def find(self, T: int, name: str):
         off, n = C.c_size_t(), C.c_size_t()
         _check(self.lib, self.lib.moe_workspace_find(self.h, T, name.encode(), C.byref(off), C.byref(n)),
@@ -140,9 +148,9 @@ class MoELayer:
         off, n = self.find(self.T, name)
         return self.ws[off:off + n].view(dtype)
 
-    def _ensure_ws(self, T: int):
+    def _ensure_ws(self, T: int, inference: bool = False):
         import torch
-        need = self.workspace_bytes(T)
+        need = self.inference_workspace_bytes(T) if inference else self.workspace_bytes(T)
         if self.ws is None or self.ws.numel() < need:
             self.ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
         self.T = T
@@ -152,7 +160,9 @@ class MoELayer:
         return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
     # ---- calls
-    def forward(self, x, W_r, W_gate, W_up, W_down, b_r=None, logits_in=None, want_logits=False, want_perm=True):
+    def forward(self, x, W_r, W_gate, W_up, W_down, b_r=None, logits_in=None, want_logits=False, want_perm=True,
+                inference=False):
+        """inference=True runs moe_forward_inference: no pre-activations are saved and backward() is not possible."""
         import torch
         T = x.shape[0]
         d, E, f, k = self.d, self.E, self.f, self.k
@@ -160,7 +170,7 @@ class MoELayer:
         assert tuple(W_r.shape) == (d, E) and W_r.dtype == torch.bfloat16 and W_r.is_contiguous()
         for w, shp in ((W_gate, (E, d, f)), (W_up, (E, d, f)), (W_down, (E, f, d))):
             assert tuple(w.shape) == shp and w.dtype == torch.bfloat16 and w.is_contiguous()
-        self._ensure_ws(T)
+        self._ensure_ws(T, inference)
         dev = x.device
         out = {
             "y": torch.empty(T, d, dtype=torch.bfloat16, device=dev),
@@ -175,17 +185,20 @@ class MoELayer:
             assert b_r.dtype == torch.float32 and b_r.numel() == E
         if logits_in is not None:
             assert logits_in.dtype == torch.float32 and tuple(logits_in.shape) == (T, E) and logits_in.is_contiguous()
-        rc = self.lib.moe_forward(self.h, T, _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(logits_in), _ptr(W_gate), _ptr(W_up),
+        fn = self.lib.moe_forward_inference if inference else self.lib.moe_forward
+        rc = fn(self.h, T, _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(logits_in), _ptr(W_gate), _ptr(W_up),
                                   _ptr(W_down), _ptr(out["y"]), _ptr(out["idx"]), _ptr(out["gates"]),
                                   _ptr(out["counts"]), _ptr(out["perm"]), _ptr(out["aux"]), _ptr(out["logits"]),
                                   _ptr(self.ws), self.ws.numel(), self._stream())
         _check(self.lib, rc, "moe_forward")
-        self._saved = (x, W_r, W_gate, W_up, W_down)
+        self._saved = None if inference else (x, W_r, W_gate, W_up, W_down)
         return out
 
     def backward(self, dy, d_aux: float, want_db: bool = False, grads=None):
         """Gradients for the last forward().  `grads` may carry preallocated output tensors."""
         import torch
+        if self._saved is None:
+            raise MoEError("backward() needs a preceding training forward()")
         x, W_r, W_gate, W_up, W_down = self._saved
         T = x.shape[0]
         d, E, f = self.d, self.E, self.f

@@ -40,18 +40,19 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.gates = take(sizeof(float) * R);
   L.inv = take(sizeof(int32_t) * R);
   L.row_gate = take(sizeof(float) * L.rows_max);
+  const size_t rows_d = sizeof(uint16_t) * L.rows_max * s.d, rows_f = sizeof(uint16_t) * L.rows_max * s.f;
+  L.xp = take(rows_d);
+  L.act = take(rows_f);
+  L.o = take(rows_d);
+  L.infer_total = off;  // everything above is all a forward-only call touches
+  L.hg = take(rows_f);
+  L.hu = take(rows_f);
   L.dg_part = take(sizeof(float) * ((s.f + 255) / 256) * L.rows_max);
   L.dg = take(sizeof(float) * R);
   L.dl = take(sizeof(float) * T * s.E);
   L.dl_hi = take(sizeof(uint16_t) * (T * s.E + 64));
   L.dl_lo = take(sizeof(uint16_t) * (T * s.E + 64));
   L.dwr_part = take(sizeof(float) * DWR_SPLIT * s.d * s.E);
-  const size_t rows_d = sizeof(uint16_t) * L.rows_max * s.d, rows_f = sizeof(uint16_t) * L.rows_max * s.f;
-  L.xp = take(rows_d);
-  L.hg = take(rows_f);
-  L.hu = take(rows_f);
-  L.act = take(rows_f);
-  L.o = take(rows_d);
   L.dhg = take(rows_f);
   L.dhu = take(rows_f);
   L.dxp = take(rows_d);
@@ -271,11 +272,11 @@ moe_status moe_stage_times(moe_ctx* ctx, float* ms, int32_t* steps) {
   return MOE_OK;
 }
 
-moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
-                       const float* logits_in, const uint16_t* W_gate, const uint16_t* W_up,
-                       const uint16_t* W_down, uint16_t* y, int32_t* topk_idx, float* topk_w,
-                       int32_t* expert_counts, int32_t* perm, float* aux_loss, float* logits_out,
-                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r,
+                               const float* b_r, const float* logits_in, const uint16_t* W_gate,
+                               const uint16_t* W_up, const uint16_t* W_down, uint16_t* y, int32_t* topk_idx,
+                               float* topk_w, int32_t* expert_counts, int32_t* perm, float* aux_loss,
+                               float* logits_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   const Shape& s = c->s;
@@ -286,12 +287,13 @@ moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_
     return MOE_ERR_INVALID_ARG;
   if (T * s.k > (int64_t(1) << 30)) return MOE_ERR_UNSUPPORTED;
   const WsLayout L = make_layout(s, T);
-  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE;
+  if (workspace_bytes < (training ? L.total : L.infer_total)) return MOE_ERR_WORKSPACE;
   moe_status rc = ensure_device(c);
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* ws = static_cast<char*>(workspace);
   GemmIO io;
+  io.save_preactivations = training;
   io.x = x; io.W_r = W_r; io.b_r = b_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
   io.idx_out = topk_idx; io.gates_out = topk_w; io.logits_out = logits_out;
   const bool tc_router = router_on_tensor_cores(s) && logits_in == nullptr;
@@ -329,6 +331,29 @@ moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_
     }
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                       const float* logits_in, const uint16_t* W_gate, const uint16_t* W_up,
+                       const uint16_t* W_down, uint16_t* y, int32_t* topk_idx, float* topk_w,
+                       int32_t* expert_counts, int32_t* perm, float* aux_loss, float* logits_out,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return forward_impl(true, ctx, T, x, W_r, b_r, logits_in, W_gate, W_up, W_down, y, topk_idx, topk_w, expert_counts,
+                      perm, aux_loss, logits_out, workspace, workspace_bytes, cuda_stream);
+}
+
+moe_status moe_forward_inference(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                                 const float* logits_in, const uint16_t* W_gate, const uint16_t* W_up,
+                                 const uint16_t* W_down, uint16_t* y, int32_t* topk_idx, float* topk_w,
+                                 int32_t* expert_counts, int32_t* perm, float* aux_loss, float* logits_out,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return forward_impl(false, ctx, T, x, W_r, b_r, logits_in, W_gate, W_up, W_down, y, topk_idx, topk_w, expert_counts,
+                      perm, aux_loss, logits_out, workspace, workspace_bytes, cuda_stream);
+}
+
+size_t moe_inference_workspace_bytes(const moe_ctx* ctx, int64_t T) {
+  if (!ctx || T < 0) return 0;
+  return make_layout(reinterpret_cast<const moe_ctx_impl*>(ctx)->s, T).infer_total;
 }
 
 moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,

@@ -55,6 +55,7 @@ struct WsLayout {
   size_t dhg, dhu;     // bf16[rows_max * f]
   size_t dxp;          // bf16[rows_max * d]
   size_t dxr;          // bf16[T * d]  router term of dx (dl W_r^T)
+  size_t infer_total;  // bytes a forward-only call needs (tables, xp, act, o)
   size_t total;
   int64_t rows_max;    // upper bound of the padded row total for T tokens
   int64_t max_m_tiles;
@@ -107,6 +108,7 @@ void launch_unpermute_sum(const Shape& s, int64_t T, const uint16_t* dxp, const 
 enum GemmKind { GEMM_F3 = 0, GEMM_F4, GEMM_B2, GEMM_B3, GEMM_B4, GEMM_B5, GEMM_RT, GEMM_DX, GEMM_DWR, GEMM_KINDS };
 // Caller tensors a grouped-GEMM launch may need besides the workspace.
 struct GemmIO {
+  bool save_preactivations = true;  // forward: also write hg, hu (needed by backward only)
   const uint16_t* x = nullptr;
   const uint16_t* W_r = nullptr;
   const float* b_r = nullptr;

@@ -347,6 +347,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.out0 = hg; p.out1 = hu; p.out2 = act;
       p.ld_out = f;
       p.row_gate = reinterpret_cast<const float*>(ws + L.row_gate);
+      p.save_pre = io.save_preactivations ? 1 : 0;
       if (!ok) return MOE_ERR_CUDA;
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_F3>(ctx, p, st);
     case GEMM_F4:

@@ -63,6 +63,7 @@ struct GemmParams {
   float* psum_part;     // RT: [4 * tiles, E] per-warp column sums of p
   float* outf;          // DWR: [slices, d, E] fp32 partials; B2: [column tiles, rows_max] partial sums of dg
   const float* row_gate;  // F3, B2: gate of every padded row (0 for pad rows)
+  int save_pre;         // F3: 1 = also store hg, hu (training), 0 = only the activation (forward-only calls)
   int64_t rows_max;     // B2: stride of the dg partial slices
 };
 
@@ -269,12 +270,14 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       if (write && col < p.N_total) {
         float t[32];
         const float gate = p.row_gate[row];  // the combine weight is folded into the saved activation
+        if (p.save_pre) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(rg[i]);
-        stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
+          for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(rg[i]);
+          stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(ru[i]);
-        stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
+          for (int i = 0; i < 32; ++i) t[i] = __uint_as_float(ru[i]);
+          stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
+        }
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const float hg = __uint_as_float(rg[i]);

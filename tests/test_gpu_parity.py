@@ -160,6 +160,28 @@ def test_repeated_calls_are_bitwise_reproducible():
         assert torch.equal(ga[n], gb[n]), n
 
 
+@pytest.mark.parametrize("T,d,E,k,f,seed", [(1000, 512, 16, 4, 384, 14), (777, 256, 64, 8, 192, 27)])
+def test_forward_inference_entry(T, d, E, k, f, seed):
+    """moe_forward_inference: same y and routing as the training forward, from a workspace of only the inference size
+    (no pre-activation buffers), and no backward afterwards."""
+    from paper_2608_00916_b200.binding import MoEError
+    shape = synth.MoEShape(T, d, E, k, f)
+    inp = synth.make_inputs(shape, seed, x_std=1.0)
+    ofw, _ = oracle_run(inp, k, 0.0)
+    r = Run(inp, k)
+    v = r.dev
+    assert r.layer.inference_workspace_bytes(T) < r.layer.workspace_bytes(T)
+    fw = r.layer.forward(v["x"], v["W_r"], v["W_gate"], v["W_up"], v["W_down"], want_logits=True, inference=True)
+    r.layer.poll()
+    assert r.layer.ws.numel() == max(r.layer.inference_workspace_bytes(T), 256)  # the small workspace sufficed
+    check_routing(fw, ofw)
+    assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+    with pytest.raises(MoEError):
+        r.layer.backward(v["dy"], 0.0)
+    train = Run(inp, k).forward()
+    assert torch.equal(train["y"], fw["y"])  # bitwise the same outputs as the training forward
+
+
 def test_bounded_wait_reports_timeout_and_context_survives():
     """A device-side wait that can never complete gives up, the status word says so, and the same context and
     workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
