@@ -171,8 +171,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="qwen", choices=list(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--mode", default="train", choices=["train", "inference"],
-                    help="train: forward + backward (the headline metric); inference: forward-only entry point")
+    ap.add_argument("--mode", default="train", choices=["train", "inference", "accumulate"],
+                    help="train: forward + backward (the headline metric); inference: forward-only entry point; "
+                         "accumulate: forward + backward that adds weight gradients into fp32 buffers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -247,9 +248,19 @@ def main():
         pdist.finish()
         return
 
+    acc = None
+    if args.mode == "accumulate":
+        acc = {"dW_r": torch.zeros(shape.d, shape.E, device="cuda"),
+               "dW_gate": torch.zeros(shape.E, shape.d, shape.f, device="cuda"),
+               "dW_up": torch.zeros(shape.E, shape.d, shape.f, device="cuda"),
+               "dW_down": torch.zeros(shape.E, shape.f, shape.d, device="cuda")}
+
     def step():
         layer.forward(tens["x"], tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], b_r=b_r, want_perm=False)
-        layer.backward(tens["dy"], inp["d_aux"], grads=grads)
+        if acc is not None:
+            layer.backward_accumulate(tens["dy"], inp["d_aux"], acc)
+        else:
+            layer.backward(tens["dy"], inp["d_aux"], grads=grads)
 
     for _ in range(args.warmup):
         step()
@@ -351,7 +362,7 @@ def main():
     line = {"metric": "moe_layer_fwd_bwd_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "T_per_gpu": T, "d": shape.d, "E": shape.E, "top_k": shape.k,
+            "config": {"workload": args.workload, "mode": args.mode, "T_per_gpu": T, "d": shape.d, "E": shape.E, "top_k": shape.k,
                        "f": shape.f, "parallelism": f"dp{world} over tokens, experts replicated (EP=1), no collective",
                        "l2": "inputs larger than L2 (1.2 GB of expert weights streamed per pass); no explicit flush",
                        "redrawn_tokens": inp["meta"]["redrawn"]},

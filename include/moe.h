@@ -164,6 +164,19 @@ MOE_API moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
                         uint16_t* dW_up, uint16_t* dW_down, void* workspace, size_t workspace_bytes,
                         void* cuda_stream);
 
+/* Backward pass that ADDS the weight gradients to fp32 buffers instead of overwriting bf16 ones: the gradient
+ * accumulation of a training step that is split into micro-batches (the paper's Megatron backend keeps fp32
+ * gradient buffers that the distributed optimizer consumes, Section "Megatron backend").
+ *   dW_gate, dW_up [E,d,f] fp32, dW_down [E,f,d] fp32, dW_r [d,E] fp32, db_r [E] fp32 or NULL: each is read, the
+ *   micro-batch's gradient is added in fp32 (no bf16 rounding of the gradient), and written back.  The caller
+ *   zeroes them at the start of an accumulation window.  Slabs of experts without tokens are left untouched.
+ *   dx [T,d] bf16 is overwritten as in moe_backward.  All other arguments as in moe_backward. */
+MOE_API moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux,
+                                           const uint16_t* x, const uint16_t* W_r, const uint16_t* W_gate,
+                                           const uint16_t* W_up, const uint16_t* W_down, uint16_t* dx, float* dW_r,
+                                           float* db_r, float* dW_gate, float* dW_up, float* dW_down,
+                                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Host-buffer convenience used for end-to-end timing: every tensor argument is a HOST pointer (pinned
  * memory recommended); the call copies inputs to the device buffers of `dev` (a device scratch of
  * moe_e2e_device_bytes(ctx, T) bytes owned by the caller), runs forward and backward, copies y, dx, aux and

@@ -17,7 +17,7 @@ STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine"
 EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
            "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout",
-           "moe_forward_inference", "moe_inference_workspace_bytes"]
+           "moe_forward_inference", "moe_inference_workspace_bytes", "moe_backward_accumulate"]
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -65,6 +65,8 @@ def load_library() -> C.CDLL:
     lib.moe_inference_workspace_bytes.restype = sz
     lib.moe_backward.argtypes = [vp, i64, vp, C.c_float] + [vp] * 11 + [vp, sz, vp]
     lib.moe_backward.restype = C.c_int
+    lib.moe_backward_accumulate.argtypes = lib.moe_backward.argtypes
+    lib.moe_backward_accumulate.restype = C.c_int
     lib.moe_e2e_device_bytes.argtypes = [vp, i64]
     lib.moe_e2e_device_bytes.restype = sz
     lib.moe_step_host.argtypes = [vp, i64, C.c_int] + [vp] * 6 + [C.c_float] + [vp] * 7 + [vp, sz, vp]
@@ -219,6 +221,25 @@ class MoELayer:
                                    self.ws.numel(), self._stream())
         _check(self.lib, rc, "moe_backward")
         return out
+
+    def backward_accumulate(self, dy, d_aux: float, acc):
+        """Backward of the last forward() that adds the weight gradients into the fp32 tensors of `acc`
+        (keys dW_r [d,E], dW_gate, dW_up [E,d,f], dW_down [E,f,d], optional db_r [E]); returns dx."""
+        import torch
+        if self._saved is None:
+            raise MoEError("backward_accumulate() needs a preceding training forward()")
+        x, W_r, W_gate, W_up, W_down = self._saved
+        T = x.shape[0]
+        for n, shp in (("dW_r", (self.d, self.E)), ("dW_gate", (self.E, self.d, self.f)), ("dW_up", (self.E, self.d, self.f)),
+                       ("dW_down", (self.E, self.f, self.d))):
+            assert acc[n].dtype == torch.float32 and tuple(acc[n].shape) == shp and acc[n].is_contiguous(), n
+        dx = torch.empty(T, self.d, dtype=torch.bfloat16, device=x.device)
+        rc = self.lib.moe_backward_accumulate(self.h, T, _ptr(dy), C.c_float(d_aux), _ptr(x), _ptr(W_r), _ptr(W_gate),
+                                              _ptr(W_up), _ptr(W_down), _ptr(dx), _ptr(acc["dW_r"]), _ptr(acc.get("db_r")),
+                                              _ptr(acc["dW_gate"]), _ptr(acc["dW_up"]), _ptr(acc["dW_down"]),
+                                              _ptr(self.ws), self.ws.numel(), self._stream())
+        _check(self.lib, rc, "moe_backward_accumulate")
+        return dx
 
     def poll(self) -> None:
         """Synchronises and raises if a device-side bounded wait ran out."""

@@ -356,16 +356,19 @@ size_t moe_inference_workspace_bytes(const moe_ctx* ctx, int64_t T) {
   return make_layout(reinterpret_cast<const moe_ctx_impl*>(ctx)->s, T).infer_total;
 }
 
-moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
-                        const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
-                        const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
-                        uint16_t* dW_up, uint16_t* dW_down, void* workspace, size_t workspace_bytes,
-                        void* cuda_stream) {
+// acc_* non-null: accumulate mode (fp32 weight-gradient buffers are added to; dW_r / db_r are added to as well)
+static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
+                                const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                                const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
+                                uint16_t* dW_up, uint16_t* dW_down, float* acc_gate, float* acc_up, float* acc_down,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  const bool accumulate = acc_gate != nullptr;
   if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   const Shape& s = c->s;
-  if (!W_r || !W_gate || !W_up || !W_down || !dW_r || !dW_gate || !dW_up || !dW_down || !workspace)
-    return MOE_ERR_INVALID_ARG;
+  if (!W_r || !W_gate || !W_up || !W_down || !dW_r || !workspace) return MOE_ERR_INVALID_ARG;
+  if (accumulate ? (!acc_up || !acc_down) : (!dW_gate || !dW_up || !dW_down)) return MOE_ERR_INVALID_ARG;
+  if (accumulate && (!aligned16(acc_gate) || !aligned16(acc_up) || !aligned16(acc_down))) return MOE_ERR_INVALID_ARG;
   if (T > 0 && (!dy || !x || !dx)) return MOE_ERR_INVALID_ARG;
   if (!aligned16(dy) || !aligned16(x) || !aligned16(W_r) || !aligned16(W_gate) || !aligned16(W_up) ||
       !aligned16(W_down) || !aligned16(dx) || !aligned16(dW_gate) || !aligned16(dW_up) || !aligned16(dW_down) ||
@@ -383,6 +386,7 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   GemmIO io;
   io.x = x; io.W_r = W_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
   io.dW_gate = dW_gate; io.dW_up = dW_up; io.dW_down = dW_down; io.dx = dx;
+  io.dW_gate_acc = acc_gate; io.dW_up_acc = acc_up; io.dW_down_acc = acc_down;
   const bool tc_router = router_on_tensor_cores(s);
   if (T > 0) {
     StageTimer tm(c, st, 5);
@@ -421,7 +425,7 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
       rc = launch_grouped_gemm(c, GEMM_DWR, T, L, ws, io, st);
       if (rc != MOE_OK) return rc;
     }
-    launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, tc_router && T > 0, st);
+    launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, tc_router && T > 0, st, accumulate);
   }
   {
     StageTimer tm(c, st, 12);
@@ -436,6 +440,25 @@ moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux
   }
   if (c->profiling) c->prof_step++;
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
+                        const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                        const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
+                        uint16_t* dW_up, uint16_t* dW_down, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+  return backward_impl(ctx, T, dy, d_aux, x, W_r, W_gate, W_up, W_down, dx, dW_r, db_r, dW_gate, dW_up, dW_down, nullptr,
+                       nullptr, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
+                                   const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                                   const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, float* dW_gate,
+                                   float* dW_up, float* dW_down, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream) {
+  if (!dW_gate || !dW_up || !dW_down) return MOE_ERR_INVALID_ARG;
+  return backward_impl(ctx, T, dy, d_aux, x, W_r, W_gate, W_up, W_down, dx, dW_r, db_r, nullptr, nullptr, nullptr, dW_gate,
+                       dW_up, dW_down, workspace, workspace_bytes, cuda_stream);
 }
 
 // ------------------------------------------------------------------------------------------ host-buffer step

@@ -206,18 +206,19 @@ __global__ void __launch_bounds__(256) dwr_partial_kernel(int64_t T, int d, int 
     }
 }
 
-__global__ void dwr_reduce_kernel(int64_t n, const float* __restrict__ part, float* __restrict__ dW_r) {
+__global__ void dwr_reduce_kernel(int64_t n, const float* __restrict__ part, float* __restrict__ dW_r,
+                                  int accumulate) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n) return;
   float s = 0.f;
 #pragma unroll
   for (int sl = 0; sl < DWR_SPLIT; ++sl) s += part[sl * n + i];
-  dW_r[i] = s;
+  dW_r[i] = accumulate ? dW_r[i] + s : s;
 }
 
 // db_r[e] = sum_t dl[t,e]: one block per 32 experts, 8 warps stride over the tokens, fixed-order final sum.
 __global__ void __launch_bounds__(256) dbr_kernel(int64_t T, int E, const float* __restrict__ dl,
-                                                  float* __restrict__ db_r) {
+                                                  float* __restrict__ db_r, int accumulate) {
   __shared__ float part[8][32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int e = blockIdx.x * 32 + lane;
@@ -230,19 +231,19 @@ __global__ void __launch_bounds__(256) dbr_kernel(int64_t T, int E, const float*
     float a = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) a += part[w][lane];
-    db_r[e] = a;
+    db_r[e] = accumulate ? db_r[e] + a : a;
   }
 }
 
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
-                float* db_r, bool partials_ready, cudaStream_t st) {
+                float* db_r, bool partials_ready, cudaStream_t st, bool accumulate) {
   const int64_t n = static_cast<int64_t>(s.d) * s.E;
   if (!partials_ready) {
     dim3 grid(s.d / DW_BM, DWR_SPLIT);
     dwr_partial_kernel<<<grid, 256, sizeof(float) * DW_BK * s.E, st>>>(T, s.d, s.E, x, dl, part);
   }
-  dwr_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(n, part, dW_r);
-  if (db_r) dbr_kernel<<<(s.E + 31) / 32, 256, 0, st>>>(T, s.E, dl, db_r);
+  dwr_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(n, part, dW_r, accumulate ? 1 : 0);
+  if (db_r) dbr_kernel<<<(s.E + 31) / 32, 256, 0, st>>>(T, s.E, dl, db_r, accumulate ? 1 : 0);
 }
 
 // ------------------------------------------------------------------------------------------ unpermute backward

@@ -98,7 +98,7 @@ void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int
                        cudaStream_t st);
 // SIMT dW_r (any E) and the shared partial reduction / db_r
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
-                float* db_r, bool partials_ready, cudaStream_t st);
+                float* db_r, bool partials_ready, cudaStream_t st, bool accumulate = false);
 void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const float* dl,
                           const uint16_t* W_r, uint16_t* dx, cudaStream_t st);
 // dx[t,:] = dxr[t,:] + sum_j dxp[inv[t,j],:]  (router term already contracted on the tensor cores)
@@ -119,6 +119,9 @@ struct GemmIO {
   uint16_t* dW_up = nullptr;
   uint16_t* dW_down = nullptr;
   uint16_t* dx = nullptr;
+  float* dW_gate_acc = nullptr;  // accumulate mode: fp32 buffers the weight gradients are added to
+  float* dW_up_acc = nullptr;
+  float* dW_down_acc = nullptr;
   int32_t* idx_out = nullptr;
   float* gates_out = nullptr;
   float* logits_out = nullptr;

@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
-      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, true);
+      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, true, tl.e, tl.m0 + rin);
       const long long w0 = clock64();
       if (!mbar_wait(tfull_bar(acc), aph)) {
         ok = false;
@@ -393,6 +393,8 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.M_total = f;
       p.N_total = d;
       p.out0 = dW_down;
+      p.accf0 = io.dW_down_acc;
+      p.acc_fp32 = io.dW_down_acc != nullptr;
       p.ld_out = d;
       p.expert_stride = static_cast<int64_t>(f) * d;
       if (!ok) return MOE_ERR_CUDA;
@@ -406,6 +408,8 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
       p.M_total = d;
       p.N_total = f;
       p.out0 = dW_gate; p.out1 = dW_up;
+      p.accf0 = io.dW_gate_acc; p.accf1 = io.dW_up_acc;
+      p.acc_fp32 = io.dW_gate_acc != nullptr;
       p.ld_out = f;
       p.expert_stride = static_cast<int64_t>(d) * f;
       if (!ok) return MOE_ERR_CUDA;

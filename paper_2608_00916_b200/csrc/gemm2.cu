@@ -260,7 +260,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
-      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, tl.write);
+      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, tl.write, tl.e, tl.m0 + rin);
       const long long w0 = clock64();
       if (!mbar_wait(tfull_bar(acc), aph)) {
         ok = false;

@@ -62,6 +62,9 @@ struct GemmParams {
   float* gates_out;
   float* psum_part;     // RT: [4 * tiles, E] per-warp column sums of p
   float* outf;          // DWR: [slices, d, E] fp32 partials; B2: [column tiles, rows_max] partial sums of dg
+  float* accf0;         // B3, B5 in accumulate mode: fp32 weight-gradient buffers that the tile is ADDED to
+  float* accf1;
+  int acc_fp32;
   const float* row_gate;  // F3, B2: gate of every padded row (0 for pad rows)
   int save_pre;         // F3: 1 = also store hg, hu (training), 0 = only the activation (forward-only calls)
   int64_t rows_max;     // B2: stride of the dg partial slices
@@ -252,6 +255,45 @@ __device__ __forceinline__ void stage_store32(EpiStage& es, uint16_t* out, int64
   }
 }
 
+// fp32 accumulate variant for the weight gradients: out[r, 0..31] += v for the 32 rows of the slab.  The 32 x 32 fp32
+// unit (4 KB = both staging units of the warp) is written one row per lane and read back with eight lanes per
+// 128-byte row segment, so the global read-modify-write is coalesced.  The old values are loaded by the caller one
+// chunk ahead (accum_load) so that their latency overlaps the previous chunk's work.
+__device__ __forceinline__ void accum_load(const float* out, int64_t ld, int rows_valid, int lane, float4 (&g)[8]) {
+  const int ch = lane & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = (lane >> 3) + 4 * i;
+    if (r < rows_valid) g[i] = *reinterpret_cast<const float4*>(out + r * ld + ch * 4);
+  }
+}
+__device__ __forceinline__ void stage_accum32(EpiStage& es, float* out, int64_t ld, int rows_valid,
+                                              const float (&v)[32], const float4 (&g)[8], int lane) {
+  const uint32_t unit = es.base;
+  __syncwarp();  // reads of the previous use are done
+  const uint32_t rowaddr = unit + lane * 128;
+  const uint32_t sw = lane & 7;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    st_shared_v4(rowaddr + ((j ^ sw) << 4), __float_as_uint(v[4 * j + 0]), __float_as_uint(v[4 * j + 1]),
+                 __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
+  __syncwarp();
+  const int ch = lane & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = (lane >> 3) + 4 * i;
+    const uint4 w = ld_shared_v4(unit + r * 128 + ((ch ^ (r & 7)) << 4));
+    if (r < rows_valid) {
+      float4 a = g[i];
+      a.x += __uint_as_float(w.x);
+      a.y += __uint_as_float(w.y);
+      a.z += __uint_as_float(w.z);
+      a.w += __uint_as_float(w.w);
+      *reinterpret_cast<float4*>(out + r * ld + ch * 4) = a;
+    }
+  }
+}
+
 // `slab` is the first output row of the warp's 32-row slab (row of the padded row buffers for row GEMMs, row of
 // the expert's weight-gradient slab for weight gradients); `row` is the thread's own row (only the SwiGLU-backward
 // epilogue reads through it).  `write` (warp-uniform) is false for a tile half whose rows do not exist; `rows_valid`
@@ -349,6 +391,32 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       }
     }
     if (write) p.outf[static_cast<int64_t>(n0 / 256) * p.rows_max + row] = dgp;
+  } else if (Traits<KIND>::WGRAD && KIND != GEMM_DWR && p.acc_fp32) {
+    // accumulate mode of the weight gradients: fp32 read-modify-write, old values fetched one chunk ahead
+    auto dst_of = [&](int c) -> float* {
+      float* fb = (KIND == GEMM_B5 && c >= 4) ? p.accf1 : p.accf0;
+      const int col = (KIND == GEMM_B5) ? n0 + (c & 3) * 32 : n0 + c * 32;
+      return (write && col < p.N_total) ? fb + e * p.expert_stride + static_cast<int64_t>(slab) * p.ld_out + col : nullptr;
+    };
+    float4 gn[8];
+    float* dn = dst_of(0);
+    if (dn) accum_load(dn, p.ld_out, rows_valid, lane, gn);
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+      float4 g[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) g[i] = gn[i];
+      float* dc = dn;
+      dn = c + 1 < 8 ? dst_of(c + 1) : nullptr;
+      if (dn) accum_load(dn, p.ld_out, rows_valid, lane, gn);
+      uint32_t rd[32];
+      tmem_ld32(taddr + c * 32, rd);
+      tmem_ld_wait();
+      float v[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rd[i]);
+      if (dc) stage_accum32(es, dc, p.ld_out, rows_valid, v, g, lane);
+    }
   } else {
     // plain bf16 store: F4, B4, DX (row GEMMs), B3, B5 (weight gradients)
 #pragma unroll 1
@@ -365,9 +433,14 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
         base = (c >= 4) ? p.out1 : p.out0;
         col = n0 + (c & 3) * 32;
       }
-      if (write && col < p.N_total)
-        stage_store32(es, base + e * p.expert_stride + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, v,
-                      lane);
+      if (Traits<KIND>::WGRAD) {
+        if (write && col < p.N_total)
+          stage_store32(es, base + e * p.expert_stride + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid,
+                        v, lane);
+      } else {
+        if (write && col < p.N_total)
+          stage_store32(es, base + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, v, lane);
+      }
     }
   }
 }
@@ -377,7 +450,19 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
 // into L2 while the tile's main loop still runs keeps the epilogue from stalling on each 32-column chunk (it was
 // the slower side of this kernel: accumulators waited for it).
 template <int KIND>
-__device__ __forceinline__ void epilogue_prefetch(const GemmParams& p, int64_t row, int n0, bool write) {
+__device__ __forceinline__ void epilogue_prefetch(const GemmParams& p, int64_t row, int n0, bool write, int e = 0,
+                                                  int m = 0) {
+  if ((KIND == GEMM_B3 || KIND == GEMM_B5) && p.acc_fp32 && write && m < p.M_total) {
+    // accumulate mode: this thread's row of the fp32 gradient tile (1 KB) will be read by the epilogue
+    const int span = KIND == GEMM_B5 ? 128 : 256;
+    const int cols = min(span, p.N_total - n0);
+    const float* a0 = p.accf0 + e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + n0;
+    for (int c = 0; c < cols; c += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(a0 + c));
+    if (KIND == GEMM_B5) {
+      const float* a1 = p.accf1 + e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + n0;
+      for (int c = 0; c < cols; c += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(a1 + c));
+    }
+  }
   if (KIND == GEMM_B2 && write) {
     const int cols = min(256, p.N_total - n0);
     const uint16_t* h = p.in0 + row * p.ld_out + n0;
@@ -392,7 +477,7 @@ __device__ __forceinline__ void epilogue_prefetch(const GemmParams& p, int64_t r
 // Weight gradient of an expert without tokens: the thread's row of the output tile is zero.
 template <int KIND>
 __device__ __forceinline__ void wgrad_zero_fill(const GemmParams& p, int e, int m, int n0) {
-  if (m >= p.M_total) return;
+  if (m >= p.M_total || p.acc_fp32) return;  // accumulate mode: an expert without tokens adds nothing
   float z[32];
 #pragma unroll
   for (int i = 0; i < 32; ++i) z[i] = 0.f;

@@ -182,6 +182,38 @@ def test_forward_inference_entry(T, d, E, k, f, seed):
     assert torch.equal(train["y"], fw["y"])  # bitwise the same outputs as the training forward
 
 
+@pytest.mark.parametrize("flag", [0, 1, 2])
+def test_backward_accumulate_over_micro_batches(flag):
+    """moe_backward_accumulate adds the weight gradients of successive micro-batches into fp32 buffers: after
+    three micro-batches (one of them leaving experts empty) the buffers hold the sum of the oracle's gradients."""
+    d, E, k, f = 256, 16, 4, 320
+    base = synth.make_inputs(synth.MoEShape(400, d, E, k, f), 51)
+    acc = {"dW_r": torch.zeros(d, E, device="cuda"), "db_r": torch.zeros(E, device="cuda"),
+           "dW_gate": torch.zeros(E, d, f, device="cuda"), "dW_up": torch.zeros(E, d, f, device="cuda"),
+           "dW_down": torch.zeros(E, f, d, device="cuda")}
+    ref = {n: 0.0 for n in ("dW_r", "db_r", "dW_gate", "dW_up", "dW_down")}
+    for i, T in enumerate((400, 37, 513)):
+        mb = synth.make_inputs(synth.MoEShape(T, d, E, k, f), 60 + i)
+        inp = dict(base)
+        inp["x"], inp["dy"] = mb["x"], mb["dy"]
+        # re-guard the router gaps for these tokens against the shared W_r
+        l = synth._guard_logits(inp["x"], inp["W_r"], None)
+        keep = ~synth._gap_violations(l, k)
+        inp["x"], inp["dy"] = inp["x"][keep], inp["dy"][keep]
+        ofw, obw = oracle_run(inp, k, 0.02)
+        r = Run(inp, k, flags=flag)
+        r.forward()
+        dx = r.layer.backward_accumulate(r.dev["dy"], 0.02, acc)
+        r.layer.poll()
+        assert rel_fro(from_dev_bf16(dx), obw["dx"]) <= TOL
+        for n in ref:
+            ref[n] = ref[n] + obw[n]
+    for n in ref:
+        assert rel_fro(acc[n].cpu().numpy(), ref[n]) <= TOL, n
+    # fp32 accumulation keeps more of the gradient than the bf16 outputs of moe_backward do
+    assert rel_fro(acc["dW_down"].cpu().numpy(), ref["dW_down"]) <= 3e-3
+
+
 def test_bounded_wait_reports_timeout_and_context_survives():
     """A device-side wait that can never complete gives up, the status word says so, and the same context and
     workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
