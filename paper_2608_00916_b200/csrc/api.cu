@@ -33,7 +33,8 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.tile_expert = take(sizeof(int32_t) * L.max_m_tiles);
   L.pair_tab = take(sizeof(int32_t) * 4 * L.max_m_tiles);
   L.tile_counts = take(sizeof(int32_t) * (L.tok_tiles + 1) * s.E);
-  L.psum_part = take(sizeof(float) * (L.router_blocks + 1) * s.E);
+  // rows: one per SIMT router block, or four (one per epilogue warp) per 128-token tile of the tensor-core router
+  L.psum_part = take(sizeof(float) * (L.router_blocks + 4 * ((T + 127) / 128) + 1) * s.E);
   L.psum = take(sizeof(float) * s.E);
   L.logits = take(sizeof(float) * T * s.E);
   L.idx = take(sizeof(int32_t) * R);

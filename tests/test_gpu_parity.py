@@ -99,6 +99,36 @@ def test_forced_tile_shapes(T, d, E, k, f, seed, flag):
     check_all(Run(inp, k, flags=flag), ofw, obw, 0.05)
 
 
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        E = int(rng.choice([1, 2, 3, 8, 12, 16, 24, 40, 64, 96, 128, 200, 256]))
+        k = int(rng.integers(1, min(E, 9) + 1))
+        d = 64 * int(rng.integers(1, 9))
+        f = 64 * int(rng.integers(1, 9))
+        T = int(rng.choice([1, 2, 31, 33, 127, 129, 500, 1023, 1500, 2600]))
+        out.append((T, d, E, k, f, 1000 + i))
+    return out
+
+
+@pytest.mark.parametrize("T,d,E,k,f,seed", _random_shapes(24, 2024))
+def test_random_shapes(T, d, E, k, f, seed):
+    """A seeded sweep over odd combinations of sizes (every width a multiple of 64, expert counts with and without
+    the tensor-core router path, token counts around tile boundaries): full stage-by-stage parity each time."""
+    shape = synth.MoEShape(T, d, E, k, f)
+    inp = synth.make_inputs(shape, seed, x_std=1.0)
+    if seed % 3 == 0:
+        inp["b_r"] = (0.2 * np.random.default_rng(seed).standard_normal(E)).astype(np.float32)
+        l = synth._guard_logits(inp["x"], inp["W_r"], inp["b_r"])
+        keep = ~synth._gap_violations(l, k)
+        if not keep.any():
+            pytest.skip("no guarded token in this draw")
+        inp["x"], inp["dy"] = inp["x"][keep], inp["dy"][keep]
+    ofw, obw = oracle_run(inp, k, 0.03)
+    check_all(Run(inp, k, flags=seed % 3), ofw, obw, 0.03)
+
+
 def test_skewed_small_with_bias_and_empty_experts():
     shape = synth.MoEShape(2048, 256, 32, 4, 256)
     inp = synth.make_inputs(shape, 7, x_std=1.0, skew=True)
