@@ -129,6 +129,55 @@ def test_random_shapes(T, d, E, k, f, seed):
     check_all(Run(inp, k, flags=seed % 3), ofw, obw, 0.03)
 
 
+@pytest.mark.parametrize("T,d,E,k,f", [(1, 64, 8, 2, 64), (47, 128, 256, 3, 64), (300, 192, 24, 4, 320), (1029, 256, 16, 8, 128)])
+def test_no_write_outside_the_declared_buffers(T, d, E, k, f):
+    """Canaries: the bytes after the workspace, the alignment gaps between its internal buffers and the bytes after
+    every caller output keep their fill pattern through a forward + backward."""
+    import ctypes as C
+    from paper_2608_00916_b200.binding import MoELayer, _ptr, _check
+    shape = synth.MoEShape(T, d, E, k, f)
+    inp = synth.make_inputs(shape, 77)
+    dev = {n: torch.from_numpy(inp[n].view(np.int16)).cuda().view(torch.bfloat16)
+           for n in ("x", "W_r", "W_gate", "W_up", "W_down", "dy")}
+    layer = MoELayer(d, E, f, k)
+    need = layer.workspace_bytes(T)
+    PAD = 4096
+    ws = torch.full((need + PAD,), 0xA5, dtype=torch.uint8, device="cuda")
+    names = ["counts", "offsets", "pad_offsets", "logits", "idx", "gates", "inv", "row_gate", "xp", "hg", "hu", "act", "o",
+             "dhg", "dhu", "dxp", "dxr", "dg", "dl", "status", "timers"]
+    spans = sorted(layer.find(T, n) for n in names)
+
+    def guarded(shape_, dtype):
+        n = int(np.prod(shape_)) if len(shape_) else 1
+        buf = torch.full((n * torch.empty((), dtype=dtype).element_size() + 256,), 0x5A, dtype=torch.uint8, device="cuda")
+        return buf, buf[: buf.numel() - 256].view(dtype).view(*shape_) if n else buf[:0].view(dtype).view(*shape_)
+
+    outs = {n: guarded(shp, dt) for n, shp, dt in (
+        ("y", (T, d), torch.bfloat16), ("idx", (T, k), torch.int32), ("gates", (T, k), torch.float32),
+        ("counts", (E,), torch.int32), ("perm", (T * k,), torch.int32), ("aux", (1,), torch.float32),
+        ("dx", (T, d), torch.bfloat16), ("dW_r", (d, E), torch.float32), ("db_r", (E,), torch.float32),
+        ("dW_gate", (E, d, f), torch.bfloat16), ("dW_up", (E, d, f), torch.bfloat16), ("dW_down", (E, f, d), torch.bfloat16))}
+    o = {n: v[1] for n, v in outs.items()}
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    lib = layer.lib
+    _check(lib, lib.moe_forward(layer.h, T, _ptr(dev["x"]), _ptr(dev["W_r"]), None, None, _ptr(dev["W_gate"]),
+                                _ptr(dev["W_up"]), _ptr(dev["W_down"]), _ptr(o["y"]), _ptr(o["idx"]), _ptr(o["gates"]),
+                                _ptr(o["counts"]), _ptr(o["perm"]), _ptr(o["aux"]), None, _ptr(ws), need, st), "fwd")
+    _check(lib, lib.moe_backward(layer.h, T, _ptr(dev["dy"]), C.c_float(0.01), _ptr(dev["x"]), _ptr(dev["W_r"]),
+                                 _ptr(dev["W_gate"]), _ptr(dev["W_up"]), _ptr(dev["W_down"]), _ptr(o["dx"]), _ptr(o["dW_r"]),
+                                 _ptr(o["db_r"]), _ptr(o["dW_gate"]), _ptr(o["dW_up"]), _ptr(o["dW_down"]), _ptr(ws), need,
+                                 st), "bwd")
+    torch.cuda.synchronize()
+    assert bool((ws[need:] == 0xA5).all()), "wrote past the workspace"
+    for (off, n), (noff, _) in zip(spans, spans[1:]):
+        gap = ws[off + n: noff]
+        # only gaps that are pure alignment padding (< 256 bytes) are guaranteed to be nobody's buffer
+        if 0 < gap.numel() < 256:
+            assert bool((gap == 0xA5).all()), f"wrote into the padding after offset {off}+{n}"
+    for n, (buf, _) in outs.items():
+        assert bool((buf[-256:] == 0x5A).all()), f"wrote past {n}"
+
+
 def test_skewed_small_with_bias_and_empty_experts():
     shape = synth.MoEShape(2048, 256, 32, 4, 256)
     inp = synth.make_inputs(shape, 7, x_std=1.0, skew=True)
