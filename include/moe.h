@@ -181,7 +181,8 @@ MOE_API moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16
  * memory recommended); the call copies inputs to the device buffers of `dev` (a device scratch of
  * moe_e2e_device_bytes(ctx, T) bytes owned by the caller), runs forward and backward, copies y, dx, aux and
  * the weight gradients back and synchronises the stream.  copy_weights != 0 also uploads the weights and
- * downloads their gradients; with 0 the weights must already be resident from an earlier call. */
+ * downloads their gradients; with 0 the weights must already be resident from an earlier call.  The copies run on
+ * two streams of the context so that dy arrives while forward runs and y leaves while backward runs. */
 MOE_API size_t moe_e2e_device_bytes(const moe_ctx* ctx, int64_t T);
 MOE_API moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16_t* x, const uint16_t* W_r,
                          const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,

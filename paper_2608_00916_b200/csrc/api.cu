@@ -127,6 +127,11 @@ void moe_destroy(moe_ctx* ctx) {
         cudaEventDestroy(c->ev[r][i][0]);
         cudaEventDestroy(c->ev[r][i][1]);
       }
+  if (c->e2e_created) {
+    cudaStreamDestroy(c->s_in);
+    cudaStreamDestroy(c->s_out);
+    for (int i = 0; i < 6; ++i) cudaEventDestroy(c->e2e_ev[i]);
+  }
   delete c;
 }
 
@@ -509,42 +514,64 @@ moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* D = static_cast<char*>(dev);
   const size_t td = sizeof(uint16_t) * T * s.d, w = sizeof(uint16_t) * s.E * s.d * s.f;
+  // Copies run on two private streams so that they overlap the compute stream: dy arrives while forward runs,
+  // y leaves while backward runs; only the copy of x before forward and of dx after backward are exposed.
+  if (!c->e2e_created) {
+    if (cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    for (int i = 0; i < 6; ++i)
+      if (cudaEventCreateWithFlags(&c->e2e_ev[i], cudaEventDisableTiming) != cudaSuccess) return MOE_ERR_CUDA;
+    c->e2e_created = 1;
+  }
+  cudaEvent_t ev_start = c->e2e_ev[0], ev_x = c->e2e_ev[1], ev_dy = c->e2e_ev[2], ev_fwd = c->e2e_ev[3],
+              ev_bwd = c->e2e_ev[4], ev_out = c->e2e_ev[5];
   bool ok = true;
   auto h2d = [&](size_t off, const void* src, size_t n) {
-    ok = ok && cudaMemcpyAsync(D + off, src, n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(D + off, src, n, cudaMemcpyHostToDevice, c->s_in) == cudaSuccess;
   };
   auto d2h = [&](void* dst, size_t off, size_t n) {
-    ok = ok && cudaMemcpyAsync(dst, D + off, n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(dst, D + off, n, cudaMemcpyDeviceToHost, c->s_out) == cudaSuccess;
   };
-  h2d(L.x, x, td);
-  h2d(L.dy, dy, td);
+  // everything already queued on the caller's stream comes first
+  ok = ok && cudaEventRecord(ev_start, st) == cudaSuccess && cudaStreamWaitEvent(c->s_in, ev_start, 0) == cudaSuccess;
   if (copy_weights) {
     h2d(L.W_r, W_r, sizeof(uint16_t) * s.d * s.E);
     h2d(L.Wg, W_gate, w);
     h2d(L.Wu, W_up, w);
     h2d(L.Wd, W_down, w);
   }
+  h2d(L.x, x, td);
+  ok = ok && cudaEventRecord(ev_x, c->s_in) == cudaSuccess;
+  h2d(L.dy, dy, td);
+  ok = ok && cudaEventRecord(ev_dy, c->s_in) == cudaSuccess;
   if (!ok) return MOE_ERR_CUDA;
   const size_t wsb = make_layout(s, T).total;
   auto U = [&](size_t off) { return reinterpret_cast<uint16_t*>(D + off); };
+  if (cudaStreamWaitEvent(st, ev_x, 0) != cudaSuccess) return MOE_ERR_CUDA;
   moe_status rc = moe_forward(ctx, T, U(L.x), U(L.W_r), nullptr, nullptr, U(L.Wg), U(L.Wu), U(L.Wd), U(L.y),
                               reinterpret_cast<int32_t*>(D + L.idx), reinterpret_cast<float*>(D + L.gates),
                               reinterpret_cast<int32_t*>(D + L.counts), nullptr, reinterpret_cast<float*>(D + L.aux),
                               nullptr, D + L.ws, wsb, cuda_stream);
   if (rc != MOE_OK) return rc;
+  ok = ok && cudaEventRecord(ev_fwd, st) == cudaSuccess && cudaStreamWaitEvent(c->s_out, ev_fwd, 0) == cudaSuccess;
+  d2h(y, L.y, td);
+  d2h(aux_loss, L.aux, sizeof(float));
+  if (!ok || cudaStreamWaitEvent(st, ev_dy, 0) != cudaSuccess) return MOE_ERR_CUDA;
   rc = moe_backward(ctx, T, U(L.dy), d_aux, U(L.x), U(L.W_r), U(L.Wg), U(L.Wu), U(L.Wd), U(L.dx),
                     reinterpret_cast<float*>(D + L.dWr), nullptr, U(L.dWg), U(L.dWu), U(L.dWd), D + L.ws, wsb,
                     cuda_stream);
   if (rc != MOE_OK) return rc;
-  d2h(y, L.y, td);
+  ok = ok && cudaEventRecord(ev_bwd, st) == cudaSuccess && cudaStreamWaitEvent(c->s_out, ev_bwd, 0) == cudaSuccess;
   d2h(dx, L.dx, td);
-  d2h(aux_loss, L.aux, sizeof(float));
   if (copy_weights) {
     d2h(dW_r, L.dWr, sizeof(float) * s.d * s.E);
     d2h(dW_gate, L.dWg, w);
     d2h(dW_up, L.dWu, w);
     d2h(dW_down, L.dWd, w);
   }
+  // the caller's stream continues only after the results have left
+  ok = ok && cudaEventRecord(ev_out, c->s_out) == cudaSuccess && cudaStreamWaitEvent(st, ev_out, 0) == cudaSuccess;
   if (!ok) return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
   return moe_poll_status(ctx, D + L.ws, cuda_stream);

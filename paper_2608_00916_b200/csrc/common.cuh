@@ -76,6 +76,10 @@ struct moe_ctx_impl {
   unsigned char ev_used[MOE_PROF_RING][MOE_NUM_STAGES];
   int ev_created;
   int64_t prof_step;   // forward+backward pairs recorded so far
+  // moe_step_host: copy-in / copy-out streams and the events that order them against the compute stream
+  cudaStream_t s_in, s_out;
+  cudaEvent_t e2e_ev[6];
+  int e2e_created;
   int64_t prof_read;   // pairs already reported by moe_stage_times
 };
 

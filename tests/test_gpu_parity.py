@@ -293,6 +293,35 @@ def test_backward_accumulate_over_micro_batches(flag):
     assert rel_fro(acc["dW_down"].cpu().numpy(), ref["dW_down"]) <= 3e-3
 
 
+def test_step_host_matches_the_device_path():
+    """moe_step_host (host buffers in, host buffers out, copies overlapped with compute on the context's own streams)
+    returns the same bits as forward + backward on device tensors; a second call with resident weights too."""
+    shape = synth.MoEShape(900, 256, 16, 4, 192)
+    inp = synth.make_inputs(shape, 88)
+    r = Run(inp, 4)
+    fw = r.forward()
+    bw = r.backward(inp["d_aux"], want_db=False)
+    T, d, E, f = shape.T, shape.d, shape.E, shape.f
+    host = {n: torch.from_numpy(inp[n].view(np.int16)).pin_memory() for n in ("x", "dy", "W_r", "W_gate", "W_up", "W_down")}
+    host.update(y=torch.zeros(T, d, dtype=torch.int16).pin_memory(), dx=torch.zeros(T, d, dtype=torch.int16).pin_memory(),
+                aux=torch.zeros(1).pin_memory(), dW_r=torch.zeros(d, E).pin_memory(),
+                dW_gate=torch.zeros(E, d, f, dtype=torch.int16).pin_memory(),
+                dW_up=torch.zeros(E, d, f, dtype=torch.int16).pin_memory(),
+                dW_down=torch.zeros(E, f, d, dtype=torch.int16).pin_memory())
+    layer = r.layer
+    dev_buf = torch.empty(layer.e2e_device_bytes(T), dtype=torch.uint8, device="cuda")
+    for copy_weights in (True, False):
+        for n in ("y", "dx"):
+            host[n].zero_()
+        layer.step_host(T, dev_buf, host, inp["d_aux"], copy_weights=copy_weights)
+        assert torch.equal(host["y"], fw["y"].view(torch.int16).cpu())
+        assert torch.equal(host["dx"], bw["dx"].view(torch.int16).cpu())
+        assert float(host["aux"][0]) == float(fw["aux"].cpu()[0])
+    assert torch.equal(host["dW_r"], bw["dW_r"].cpu())
+    for n in ("dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(host[n], bw[n].view(torch.int16).cpu()), n
+
+
 def test_bounded_wait_reports_timeout_and_context_survives():
     """A device-side wait that can never complete gives up, the status word says so, and the same context and
     workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
