@@ -32,8 +32,8 @@ LAUNCHES_PER_STEP = 19  # router, hist, scan, scatter, gather, 2 GEMMs, combine;
 # dram bytes per launch of the dominant kernel taken from the committed ncu capture (profiles/), by stage name;
 # None where no capture has been taken for the workload.
 NCU_TRAFFIC = {  # profiles/grouped_gemms_qwen_dram_traffic.md
-    ("qwen", "gemm_gateup_swiglu"): 1.997e9, ("qwen", "gemm_down"): 1.153e9, ("qwen", "dgrad_down_swiglu_bwd"): 1.861e9,
-    ("qwen", "wgrad_down"): 1.164e9, ("qwen", "dgrad_gateup"): 1.784e9, ("qwen", "wgrad_gateup"): 1.771e9,
+    ("qwen", "gemm_gateup_swiglu"): 1.995e9, ("qwen", "gemm_down"): 1.151e9, ("qwen", "dgrad_down_swiglu_bwd"): 1.881e9,
+    ("qwen", "wgrad_down"): 1.163e9, ("qwen", "dgrad_gateup"): 1.784e9, ("qwen", "wgrad_gateup"): 1.823e9,
 }
 
 
