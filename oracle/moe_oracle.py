@@ -120,12 +120,16 @@ def expert_ffn(xr: np.ndarray, Wg: np.ndarray, Wu: np.ndarray, Wd: np.ndarray):
 
 # --------------------------------------------------------------------------------------------- forward
 def forward(x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, k: int, b_r=None, logits_in=None,
-            dtype=np.float64, keep: bool = True) -> dict:
+            dtype=np.float64, keep: bool = True, expert_weights=None) -> dict:
     """Whole layer.  Arguments are bf16 bit tensors x[T,d], W_r[d,E], W_gate/W_up[E,d,f], W_down[E,f,d].
 
     ``logits_in`` (float array [T,E]) replaces the router contraction when given, so that ties can be
     constructed by hand.  With ``keep`` the per-row intermediates (in permuted row order) are returned
-    for the backward pass and for stage-by-stage comparison."""
+    for the backward pass and for stage-by-stage comparison.  ``expert_weights(e)`` may supply expert e's
+    (W_gate, W_up, W_down) as float arrays instead of the bf16 tensors (used by the low-rank adapter variant)."""
+    if expert_weights is None:
+        def expert_weights(e):
+            return widen_bf16(Wg_bits[e], dtype), widen_bf16(Wu_bits[e], dtype), widen_bf16(Wd_bits[e], dtype)
     x = widen_bf16(x_bits, dtype)
     T, d = x.shape
     E = Wg_bits.shape[0]
@@ -152,8 +156,7 @@ def forward(x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, k: int, b_r=None, logits
         if r1 == r0:
             continue
         te = tok[r0:r1]
-        hg, hu, a, o = expert_ffn(x[te], widen_bf16(Wg_bits[e], dtype), widen_bf16(Wu_bits[e], dtype),
-                                  widen_bf16(Wd_bits[e], dtype))
+        hg, hu, a, o = expert_ffn(x[te], *expert_weights(e))
         # tokens within one expert are distinct, so this indexed add has no repeated index
         y[te] += g[te, slot[r0:r1]][:, None] * o
         if keep:
@@ -167,11 +170,14 @@ def forward(x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, k: int, b_r=None, logits
 
 # --------------------------------------------------------------------------------------------- backward
 def backward(fw: dict, dy_bits, d_aux: float, x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits,
-             dtype=np.float64, has_bias: bool = False) -> dict:
+             dtype=np.float64, has_bias: bool = False, expert_weights=None) -> dict:
     """Gradients of  L = <y, dy> + d_aux * aux  with the routing choice (idx, counts) held fixed.
 
     Returns dx[T,d], dW_r[d,E], db_r[E], dW_gate/dW_up[E,d,f], dW_down[E,f,d], plus the intermediates
     dg[T,k], dl[T,E] and the per-row d_o, dhg, dhu, dxp in permuted order."""
+    if expert_weights is None:
+        def expert_weights(e):
+            return widen_bf16(Wg_bits[e], dtype), widen_bf16(Wu_bits[e], dtype), widen_bf16(Wd_bits[e], dtype)
     k = fw["k"]
     x = widen_bf16(x_bits, dtype)
     dy = widen_bf16(dy_bits, dtype)
@@ -196,7 +202,7 @@ def backward(fw: dict, dy_bits, d_aux: float, x_bits, Wr_bits, Wg_bits, Wu_bits,
         if r1 == r0:
             continue
         te, se = tok[r0:r1], slot[r0:r1]
-        Wg, Wu, Wd = widen_bf16(Wg_bits[e], dtype), widen_bf16(Wu_bits[e], dtype), widen_bf16(Wd_bits[e], dtype)
+        Wg, Wu, Wd = expert_weights(e)
         hg, hu, a, o = fw["hg"][r0:r1], fw["hu"][r0:r1], fw["act"][r0:r1], fw["o"][r0:r1]
         # combine: y[t] = sum_j g[t,j] o[t,j]
         dg[te, se] = (dy[te] * o).sum(axis=1)
@@ -281,3 +287,43 @@ def expert_grads(e: int, fw_route: dict, dy_bits, x_bits, Wg_bits, Wu_bits, Wd_b
     dhg = da * hu * sig * (1.0 + hg * (1.0 - sig))
     dhu = da * hg * sig
     return x.T @ dhg, x.T @ dhu, a.T @ d_o
+
+
+# --------------------------------------------------------------------------------------------- expert LoRA
+# Low-rank adapters on the experts' fc1 (gate | up, one shared down-projection A1) and fc2, base weights frozen
+# (the paper's "moe_experts" LoRA target group: experts.*.linear_fc1, experts.*.linear_fc2).  By definition the
+# adapted layer is the plain layer evaluated with the effective weights
+#     W_gate' = W_gate + s A1 B1_gate,   W_up' = W_up + s A1 B1_up,   W_down' = W_down + s A2 B2,
+# and the adapter gradients follow from the gradient with respect to the effective weights by the chain rule:
+#     dA1 = s (dW_gate' B1_gate^T + dW_up' B1_up^T),  dB1_gate = s A1^T dW_gate',  dB1_up = s A1^T dW_up',
+#     dA2 = s dW_down' B2^T,  dB2 = s A2^T dW_down'.
+def lora_expert_weights(Wg_bits, Wu_bits, Wd_bits, A1_bits, B1g_bits, B1u_bits, A2_bits, B2_bits, scale, dtype=np.float64):
+    def get(e):
+        A1 = widen_bf16(A1_bits[e], dtype)
+        A2 = widen_bf16(A2_bits[e], dtype)
+        return (widen_bf16(Wg_bits[e], dtype) + scale * A1 @ widen_bf16(B1g_bits[e], dtype),
+                widen_bf16(Wu_bits[e], dtype) + scale * A1 @ widen_bf16(B1u_bits[e], dtype),
+                widen_bf16(Wd_bits[e], dtype) + scale * A2 @ widen_bf16(B2_bits[e], dtype))
+    return get
+
+
+def lora_forward(x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, A1_bits, B1g_bits, B1u_bits, A2_bits, B2_bits, scale,
+                 k: int, b_r=None, dtype=np.float64) -> dict:
+    ew = lora_expert_weights(Wg_bits, Wu_bits, Wd_bits, A1_bits, B1g_bits, B1u_bits, A2_bits, B2_bits, scale, dtype)
+    return forward(x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, k, b_r=b_r, dtype=dtype, expert_weights=ew)
+
+
+def lora_backward(fw: dict, dy_bits, d_aux, x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, A1_bits, B1g_bits, B1u_bits,
+                  A2_bits, B2_bits, scale, dtype=np.float64) -> dict:
+    ew = lora_expert_weights(Wg_bits, Wu_bits, Wd_bits, A1_bits, B1g_bits, B1u_bits, A2_bits, B2_bits, scale, dtype)
+    bw = backward(fw, dy_bits, d_aux, x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits, dtype=dtype, expert_weights=ew)
+    E = Wg_bits.shape[0]
+    A1, A2 = widen_bf16(A1_bits, dtype), widen_bf16(A2_bits, dtype)
+    B1g, B1u, B2 = widen_bf16(B1g_bits, dtype), widen_bf16(B1u_bits, dtype), widen_bf16(B2_bits, dtype)
+    out = {"dx": bw["dx"], "dW_r": bw["dW_r"], "db_r": bw["db_r"]}
+    out["dA1"] = scale * np.stack([bw["dW_gate"][e] @ B1g[e].T + bw["dW_up"][e] @ B1u[e].T for e in range(E)])
+    out["dB1_gate"] = scale * np.stack([A1[e].T @ bw["dW_gate"][e] for e in range(E)])
+    out["dB1_up"] = scale * np.stack([A1[e].T @ bw["dW_up"][e] for e in range(E)])
+    out["dA2"] = scale * np.stack([bw["dW_down"][e] @ B2[e].T for e in range(E)])
+    out["dB2"] = scale * np.stack([A2[e].T @ bw["dW_down"][e] for e in range(E)])
+    return out

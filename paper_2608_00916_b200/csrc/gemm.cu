@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    const uint32_t idesc = umma_idesc(BM, KIND == GEMM_RT ? p.mma_n : BN, TR::A_MN, TR::B_MN);
+    const uint32_t idesc = umma_idesc(BM, p.mma_n, TR::A_MN, TR::B_MN);
     constexpr uint32_t A_LBO = TR::A_MN ? CHUNK_BYTES : 0, B_LBO = TR::B_MN ? CHUNK_BYTES : 0;
     constexpr uint32_t A_KSTEP = TR::A_MN ? 2048 : 32, B_KSTEP = TR::B_MN ? 2048 : 32;  // bytes per K = 16
     uint32_t it = 0, tc = 0;
@@ -335,6 +335,9 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.b_chunks = 4;
   p.mma_n = BN;
   p.stage_tx = STAGE_BYTES;
+  p.nseg = (kind == GEMM_B4 || kind == GEMM_DX) ? 2 : 1;
+  p.k_blocks1 = 0;
+  p.out_scale = 1.f;
   bool ok = true;
   switch (kind) {
     case GEMM_F3:

@@ -57,7 +57,7 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
     tl.write = rank < info.z;
     tl.m0 = 0;
     tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
-    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
+    tl.nkb = p.k_blocks * p.nseg;
   }
   return tl;
 }

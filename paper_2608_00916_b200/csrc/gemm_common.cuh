@@ -24,6 +24,7 @@ constexpr size_t GEMM_SMEM = static_cast<size_t>(STAGES) * STAGE_BYTES + EPI_BYT
 
 struct GemmParams {
   CUtensorMap mapA0, mapA1, mapB0, mapB1;
+  CUtensorMap mapA2, mapB2, mapB3;  // operands of the optional extra K segment (low-rank adapter path)
   const int32_t* sched;        // [0] number of 128-row tiles
   const int32_t* tile_expert;  // expert of each 128-row tile
   const int32_t* pad_offsets;  // padded segment starts, E + 1 entries
@@ -35,6 +36,9 @@ struct GemmParams {
   int m_tiles;   // weight gradients: output tiles along M per expert
   int E;
   int k_blocks;  // row GEMMs: K blocks per segment
+  int nseg;      // row GEMMs: K segments of k_blocks blocks (B4, DX: up to 2)
+  int k_blocks1; // row GEMMs: K blocks of the extra segment that follows them (0: none)
+  float out_scale;  // plain epilogues multiply the accumulator by this
   int M_total;   // weight gradients: rows of one expert's output
   int N_total;   // columns of the output
   uint16_t* out0;
@@ -45,9 +49,9 @@ struct GemmParams {
   int64_t ld_out;
   int64_t expert_stride;
   // router kinds
-  int b_chunks;         // RT: 64-column chunks of W_r actually loaded (ceil(E / 64))
-  int mma_n;            // RT: N of the MMA (E rounded up to 16)
-  uint32_t stage_tx;    // bytes one stage's loads deliver (RT loads fewer B chunks)
+  int b_chunks;         // 64-column chunks of an MN-major B tile actually loaded (4 = the whole 256-wide tile)
+  int mma_n;            // N of the MMA (256 unless the B tile is narrower)
+  uint32_t stage_tx;    // bytes one stage's loads deliver
   int static_m_tiles;   // RT, DX: number of 128-token tiles
   int split_rows;       // DWR: tokens per slice (multiple of 64)
   int rows_total;       // DWR: tokens rounded up to 64
@@ -123,14 +127,14 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     tl.row0 = mt * BM;
     tl.m0 = 0;
     tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
-    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
+    tl.nkb = p.k_blocks * p.nseg + p.k_blocks1;
   } else {
     const int mt = t / p.n_tiles;
     tl.e = p.tile_expert[mt];
     tl.row0 = mt * BM;
     tl.m0 = 0;
     tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
-    tl.nkb = p.k_blocks * Traits<KIND>::NSEG;
+    tl.nkb = p.k_blocks * p.nseg + p.k_blocks1;
   }
   return tl;
 }
@@ -141,50 +145,58 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
 template <int KIND>
 __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl, int kb, uint32_t sA, uint32_t sB,
                                             uint32_t bar) {
-  constexpr bool DO_A = true, DO_B = true;
-  if (KIND == GEMM_F3) {
-    if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-    if (DO_B) {
+  if (!Traits<KIND>::WGRAD && kb >= p.k_blocks * p.nseg) {
+    // extra K segment of a row GEMM: A = a 64-wide row buffer (x A1, act A2, ... of the low-rank adapters),
+    // B = the matching adapter matrix of expert e
+    const int kk = kb - p.k_blocks * p.nseg;
+    tma_load_2d(sA, &p.mapA2, bar, kk * BK, tl.row0);
+    if (KIND == GEMM_F3) {
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
-        tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
+        tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB2, bar, tl.n0 + c * 64, kk * BK, tl.e);
+        tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB3, bar, tl.n0 + c * 64, kk * BK, tl.e);
       }
+    } else if (KIND == GEMM_F4) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB2, bar, tl.n0 + c * 64, kk * BK, tl.e);
+    } else {  // B2, B4: K-major adapter matrix, one box
+      tma_load_3d(sB, &p.mapB2, bar, kk * BK, tl.n0, tl.e);
+    }
+    return;
+  }
+  if (KIND == GEMM_F3) {
+    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
+      tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
     }
   } else if (KIND == GEMM_F4 || KIND == GEMM_RT) {
-    if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-    if (DO_B) {
+    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
-        if (KIND != GEMM_RT || c < p.b_chunks)
-          tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
-    }
+    for (int c = 0; c < 4; ++c)
+      if (c < p.b_chunks) tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
   } else if (KIND == GEMM_B2) {
-    if (DO_A) tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
-    if (DO_B) tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
+    tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
   } else if (KIND == GEMM_B4 || KIND == GEMM_DX) {
     const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
-    if (DO_A) tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
-    if (DO_B) tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
+    tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
+    tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
   } else if (KIND == GEMM_B3) {
     const int row = tl.row0 + kb * BK;
-    if (DO_A) {
 #pragma unroll
-      for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
-    }
-    if (DO_B) {
+    for (int c = 0; c < 2; ++c) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
-    }
+    for (int c = 0; c < 4; ++c)
+      if (c < p.b_chunks) tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
   } else {  // GEMM_B5, GEMM_DWR
     const int row = tl.row0 + kb * BK;
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      if (DO_A) tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
-      if (DO_B) {
-        tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
-        tma_load_2d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, row);
-      }
+      tma_load_2d(sA + c * CHUNK_BYTES, &p.mapA0, bar, tl.m0 + c * 64, row);
+      tma_load_2d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, row);
+      tma_load_2d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, row);
     }
   }
 }
@@ -236,7 +248,7 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
 
 // out points at (first row of the slab, first of the 32 columns); rows_valid = rows of the slab inside the tensor.
 __device__ __forceinline__ void stage_store32(EpiStage& es, uint16_t* out, int64_t ld, int rows_valid,
-                                              const float (&v)[32], int lane) {
+                                              const float (&v)[32], int lane, int cols_valid = 32) {
   const uint32_t unit = es.base + (es.n & 1u) * EPI_UNIT_BYTES;
   ++es.n;
   const uint32_t rowaddr = unit + lane * 64;
@@ -251,7 +263,7 @@ __device__ __forceinline__ void stage_store32(EpiStage& es, uint16_t* out, int64
   for (int i = 0; i < 4; ++i) {
     const int r = (lane >> 2) + 8 * i;
     const uint4 w = ld_shared_v4(unit + r * 64 + ((ch ^ ((r >> 1) & 3)) << 4));
-    if (r < rows_valid) *reinterpret_cast<uint4*>(out + r * ld + ch * 8) = w;
+    if (r < rows_valid && ch * 8 < cols_valid) *reinterpret_cast<uint4*>(out + r * ld + ch * 8) = w;
   }
 }
 
@@ -426,7 +438,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       tmem_ld_wait();
       float v[32];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rd[i]);
+      for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(rd[i]) * p.out_scale;
       uint16_t* base = p.out0;
       int col = n0 + c * 32;
       if (KIND == GEMM_B5) {
@@ -436,10 +448,11 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       if (Traits<KIND>::WGRAD) {
         if (write && col < p.N_total)
           stage_store32(es, base + e * p.expert_stride + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid,
-                        v, lane);
+                        v, lane, p.N_total - col);
       } else {
         if (write && col < p.N_total)
-          stage_store32(es, base + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, v, lane);
+          stage_store32(es, base + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, v, lane,
+                        p.N_total - col);
       }
     }
   }

@@ -28,7 +28,8 @@ import numpy as np
 GAP = 1e-4  # minimum distance between neighbouring logits among the k+1 largest of a token
 
 # tensor ids of the Philox keys
-_TID = {"x": 1, "W_r": 2, "W_gate": 3, "W_up": 4, "W_down": 5, "dy": 6, "x_redraw": 7, "pi": 8}
+_TID = {"x": 1, "W_r": 2, "W_gate": 3, "W_up": 4, "W_down": 5, "dy": 6, "x_redraw": 7, "pi": 8,
+        "A1": 9, "B1_gate": 10, "B1_up": 11, "A2": 12, "B2": 13}
 
 
 @dataclasses.dataclass(frozen=True)
@@ -196,3 +197,14 @@ def make_inputs(shape: MoEShape, seed: int, x_std: float = 1.0, skew: bool = Fal
 def make_config(name: str, **overrides) -> dict:
     shape, seed, x_std, skew = CONFIGS[name]
     return make_inputs(shape, seed, x_std=x_std, skew=skew, **overrides)
+
+
+def make_lora(shape: MoEShape, seed: int, rank: int = 16, std: float = 0.05, threads: int = 8) -> dict:
+    """Rank-`rank` adapters for the experts' fc1 (A1 [E,d,r], B1_gate / B1_up [E,r,f]) and fc2 (A2 [E,f,r],
+    B2 [E,r,d]), all N(0, std) in bf16 (a trained state: in a fresh adapter the B matrices would be zero)."""
+    E, d, f = shape.E, shape.d, shape.f
+    return {"A1": normal_bf16(seed, "A1", (E, d, rank), std, threads),
+            "B1_gate": normal_bf16(seed, "B1_gate", (E, rank, f), std, threads),
+            "B1_up": normal_bf16(seed, "B1_up", (E, rank, f), std, threads),
+            "A2": normal_bf16(seed, "A2", (E, f, rank), std, threads),
+            "B2": normal_bf16(seed, "B2", (E, rank, d), std, threads), "rank": rank}

@@ -321,3 +321,61 @@ def test_fp32_mode_close_to_fp64():
     assert np.array_equal(f64["idx"], f32["idx"]) and np.array_equal(f64["perm"], f32["perm"])
     rel = np.linalg.norm(f32["y"] - f64["y"]) / np.linalg.norm(f64["y"])
     assert rel < 1e-5
+
+
+# ---------------------------------------------------------------------------------- expert LoRA pins
+def _lora_problem():
+    inp = small_problem(T=10, d=8, E=4, k=2, f=6)
+    lo = synth.make_lora(synth.MoEShape(10, 8, 4, 2, 6), 9, rank=3, std=0.4, threads=1)
+    return inp, lo, 0.7
+
+
+def _lora_run(inp, lo, s, k=2):
+    args = (inp["W_gate"], inp["W_up"], inp["W_down"], lo["A1"], lo["B1_gate"], lo["B1_up"], lo["A2"], lo["B2"], s)
+    fw = orc.lora_forward(inp["x"], inp["W_r"], *args, k, b_r=inp["b_r"])
+    bw = orc.lora_backward(fw, inp["dy"], 0.2, inp["x"], inp["W_r"], *args)
+    return fw, bw
+
+
+def test_lora_with_zero_adapters_is_the_base_layer():
+    inp, lo, s = _lora_problem()
+    lo0 = dict(lo)
+    lo0["B1_gate"], lo0["B1_up"], lo0["B2"] = (np.zeros_like(lo[n]) for n in ("B1_gate", "B1_up", "B2"))
+    fw, bw = _lora_run(inp, lo0, s)
+    base = run_fw(inp, 2)
+    np.testing.assert_array_equal(fw["y"], base["y"])
+    np.testing.assert_array_equal(bw["dx"], run_bw(base, inp, 0.2)["dx"])
+    assert not bw["dA1"].any() and not bw["dA2"].any()  # dA = s dW B^T vanishes with B = 0
+
+
+def test_lora_gradients_against_torch_autograd():
+    """The adapted layer written with torch ops on the adapter parameters themselves (low-rank path computed as
+    (x A) B, never forming W + s A B) and differentiated by autograd."""
+    inp, lo, s = _lora_problem()
+    fw, bw = _lora_run(inp, lo, s)
+    k = 2
+    x = _t64(inp["x"]).requires_grad_(True)
+    Wr = _t64(inp["W_r"]); b = torch.from_numpy(inp["b_r"]).double()
+    Wg, Wu, Wd = _t64(inp["W_gate"]), _t64(inp["W_up"]), _t64(inp["W_down"])
+    P = {n: _t64(lo[n]).requires_grad_(True) for n in ("A1", "B1_gate", "B1_up", "A2", "B2")}
+    T, E = x.shape[0], Wr.shape[1]
+    l = x @ Wr + b
+    mask = torch.zeros(T, E, dtype=torch.float64)
+    mask.scatter_(1, torch.from_numpy(fw["idx"].astype(np.int64)), 1.0)
+    p = torch.softmax(l, dim=1)
+    gate = p * mask / (p * mask).sum(1, keepdim=True)
+    y = torch.zeros_like(x)
+    for e in range(E):
+        u = x @ P["A1"][e]
+        hg = x @ Wg[e] + s * (u @ P["B1_gate"][e])
+        hu = x @ Wu[e] + s * (u @ P["B1_up"][e])
+        a = F.silu(hg) * hu
+        o = a @ Wd[e] + s * ((a @ P["A2"][e]) @ P["B2"][e])
+        y = y + gate[:, e:e + 1] * o
+    np.testing.assert_allclose(fw["y"], y.detach().numpy(), rtol=1e-10, atol=1e-13)
+    aux = E * ((mask.sum(0) / (T * k)) * p.mean(0)).sum()
+    ((y * _t64(inp["dy"])).sum() + 0.2 * aux).backward()
+    np.testing.assert_allclose(bw["dx"], x.grad.numpy(), rtol=1e-9, atol=1e-12)
+    for n, key in (("A1", "dA1"), ("B1_gate", "dB1_gate"), ("B1_up", "dB1_up"), ("A2", "dA2"), ("B2", "dB2")):
+        want = P[n].grad.numpy()
+        np.testing.assert_allclose(bw[key], want, rtol=1e-9, atol=1e-12 * max(1.0, np.abs(want).max()), err_msg=key)
