@@ -177,6 +177,32 @@ MOE_API moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16
                                            float* db_r, float* dW_gate, float* dW_up, float* dW_down,
                                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Expert LoRA: the same layer with frozen expert weights and trainable rank-r adapters on the experts' fc1 (gate | up)
+ * and fc2 (down) - the paper's "moe_experts" LoRA target group (experts.*.linear_fc1, experts.*.linear_fc2; Section
+ * "LoRA target groups for MoE").  Effective weights:
+ *     W_gate' = W_gate + scale * A1 B1_gate,   W_up' = W_up + scale * A1 B1_up,   W_down' = W_down + scale * A2 B2
+ * with A1 [E,d,r], B1_gate, B1_up [E,r,f], A2 [E,f,r], B2 [E,r,d], all bf16; r = rank, a multiple of 8 in [8, 64].
+ * The effective weights are never formed: the low-rank products (x A1, act A2, ...) are 64-wide row buffers that
+ * enter the expert GEMMs as one extra K segment, and the adapter gradients are skinny GEMMs; no gradient of the
+ * frozen W_gate / W_up / W_down is computed.  Everything else (routing, outputs, dx, dW_r) is as in moe_forward /
+ * moe_backward.  The workspace needs moe_lora_workspace_bytes(ctx, T) bytes.  Gradients dA1, dB1_gate, dB1_up, dA2,
+ * dB2 have the adapters' shapes, are bf16 and are overwritten (zero slabs for experts without tokens). */
+MOE_API size_t moe_lora_workspace_bytes(const moe_ctx* ctx, int64_t T);
+MOE_API moe_status moe_lora_forward(moe_ctx* ctx, int64_t T, int32_t rank, float scale, const uint16_t* x,
+                                    const uint16_t* W_r, const float* b_r, const uint16_t* W_gate,
+                                    const uint16_t* W_up, const uint16_t* W_down, const uint16_t* A1,
+                                    const uint16_t* B1_gate, const uint16_t* B1_up, const uint16_t* A2,
+                                    const uint16_t* B2, uint16_t* y, int32_t* topk_idx, float* topk_w,
+                                    int32_t* expert_counts, float* aux_loss, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream);
+MOE_API moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, float scale, const uint16_t* dy,
+                                     float d_aux, const uint16_t* x, const uint16_t* W_r, const uint16_t* W_gate,
+                                     const uint16_t* W_up, const uint16_t* W_down, const uint16_t* A1,
+                                     const uint16_t* B1_gate, const uint16_t* B1_up, const uint16_t* A2,
+                                     const uint16_t* B2, uint16_t* dx, float* dW_r, uint16_t* dA1, uint16_t* dB1_gate,
+                                     uint16_t* dB1_up, uint16_t* dA2, uint16_t* dB2, void* workspace,
+                                     size_t workspace_bytes, void* cuda_stream);
+
 /* Host-buffer convenience used for end-to-end timing: every tensor argument is a HOST pointer (pinned
  * memory recommended); the call copies inputs to the device buffers of `dev` (a device scratch of
  * moe_e2e_device_bytes(ctx, T) bytes owned by the caller), runs forward and backward, copies y, dx, aux and

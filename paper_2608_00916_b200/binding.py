@@ -17,7 +17,8 @@ STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine"
 EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
            "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout",
-           "moe_forward_inference", "moe_inference_workspace_bytes", "moe_backward_accumulate"]
+           "moe_forward_inference", "moe_inference_workspace_bytes", "moe_backward_accumulate",
+           "moe_lora_workspace_bytes", "moe_lora_forward", "moe_lora_backward"]
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -67,6 +68,12 @@ def load_library() -> C.CDLL:
     lib.moe_backward.restype = C.c_int
     lib.moe_backward_accumulate.argtypes = lib.moe_backward.argtypes
     lib.moe_backward_accumulate.restype = C.c_int
+    lib.moe_lora_workspace_bytes.argtypes = [vp, i64]
+    lib.moe_lora_workspace_bytes.restype = sz
+    lib.moe_lora_forward.argtypes = [vp, i64, C.c_int32, C.c_float] + [vp] * 16 + [vp, sz, vp]
+    lib.moe_lora_forward.restype = C.c_int
+    lib.moe_lora_backward.argtypes = [vp, i64, C.c_int32, C.c_float, vp, C.c_float] + [vp] * 17 + [vp, sz, vp]
+    lib.moe_lora_backward.restype = C.c_int
     lib.moe_e2e_device_bytes.argtypes = [vp, i64]
     lib.moe_e2e_device_bytes.restype = sz
     lib.moe_step_host.argtypes = [vp, i64, C.c_int] + [vp] * 6 + [C.c_float] + [vp] * 7 + [vp, sz, vp]
@@ -240,6 +247,54 @@ class MoELayer:
                                               _ptr(self.ws), self.ws.numel(), self._stream())
         _check(self.lib, rc, "moe_backward_accumulate")
         return dx
+
+    # ---- expert LoRA (frozen expert weights, rank-r adapters on fc1 and fc2)
+    def lora_forward(self, x, W_r, W_gate, W_up, W_down, lora: dict, scale: float, b_r=None):
+        """lora: dict of bf16 CUDA tensors A1 [E,d,r], B1_gate, B1_up [E,r,f], A2 [E,f,r], B2 [E,r,d]."""
+        import torch
+        T = x.shape[0]
+        d, E, f, k = self.d, self.E, self.f, self.k
+        r = lora["A1"].shape[2]
+        for n, shp in (("A1", (E, d, r)), ("B1_gate", (E, r, f)), ("B1_up", (E, r, f)), ("A2", (E, f, r)), ("B2", (E, r, d))):
+            assert tuple(lora[n].shape) == shp and lora[n].dtype == torch.bfloat16 and lora[n].is_contiguous(), n
+        need = int(self.lib.moe_lora_workspace_bytes(self.h, T))
+        if self.ws is None or self.ws.numel() < need:
+            self.ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+        self.T = T
+        dev = x.device
+        out = {"y": torch.empty(T, d, dtype=torch.bfloat16, device=dev),
+               "idx": torch.empty(T, k, dtype=torch.int32, device=dev),
+               "gates": torch.empty(T, k, dtype=torch.float32, device=dev),
+               "counts": torch.empty(E, dtype=torch.int32, device=dev),
+               "aux": torch.empty(1, dtype=torch.float32, device=dev)}
+        rc = self.lib.moe_lora_forward(self.h, T, r, C.c_float(scale), _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(W_gate),
+                                       _ptr(W_up), _ptr(W_down), _ptr(lora["A1"]), _ptr(lora["B1_gate"]),
+                                       _ptr(lora["B1_up"]), _ptr(lora["A2"]), _ptr(lora["B2"]), _ptr(out["y"]),
+                                       _ptr(out["idx"]), _ptr(out["gates"]), _ptr(out["counts"]), _ptr(out["aux"]),
+                                       _ptr(self.ws), self.ws.numel(), self._stream())
+        _check(self.lib, rc, "moe_lora_forward")
+        self._saved = None
+        self._lora_saved = (x, W_r, W_gate, W_up, W_down, lora, scale)
+        return out
+
+    def lora_backward(self, dy, d_aux: float):
+        import torch
+        x, W_r, W_gate, W_up, W_down, lora, scale = self._lora_saved
+        T = x.shape[0]
+        r = lora["A1"].shape[2]
+        dev = x.device
+        out = {"dx": torch.empty(T, self.d, dtype=torch.bfloat16, device=dev),
+               "dW_r": torch.empty(self.d, self.E, dtype=torch.float32, device=dev)}
+        for n in ("A1", "B1_gate", "B1_up", "A2", "B2"):
+            out["d" + n] = torch.empty_like(lora[n])
+        rc = self.lib.moe_lora_backward(self.h, T, r, C.c_float(scale), _ptr(dy), C.c_float(d_aux), _ptr(x), _ptr(W_r),
+                                        _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(lora["A1"]), _ptr(lora["B1_gate"]),
+                                        _ptr(lora["B1_up"]), _ptr(lora["A2"]), _ptr(lora["B2"]), _ptr(out["dx"]),
+                                        _ptr(out["dW_r"]), _ptr(out["dA1"]), _ptr(out["dB1_gate"]), _ptr(out["dB1_up"]),
+                                        _ptr(out["dA2"]), _ptr(out["dB2"]), _ptr(self.ws), self.ws.numel(),
+                                        self._stream())
+        _check(self.lib, rc, "moe_lora_backward")
+        return out
 
     def poll(self) -> None:
         """Synchronises and raises if a device-side bounded wait ran out."""

@@ -59,6 +59,12 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.dxp = take(rows_d);
   L.dxr = take(sizeof(uint16_t) * T * s.d);
   L.total = off;
+  const size_t rows64 = sizeof(uint16_t) * L.rows_max * 64;
+  L.lora_u = take(rows64);
+  L.lora_v = take(rows64);
+  L.lora_w = take(rows64);
+  L.lora_z = take(rows64);
+  L.lora_total = off;
   return L;
 }
 
@@ -282,7 +288,8 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
                                const float* b_r, const float* logits_in, const uint16_t* W_gate,
                                const uint16_t* W_up, const uint16_t* W_down, uint16_t* y, int32_t* topk_idx,
                                float* topk_w, int32_t* expert_counts, int32_t* perm, float* aux_loss,
-                               float* logits_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                               float* logits_out, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                               const LoraArgs* lora = nullptr) {
   if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   const Shape& s = c->s;
@@ -293,7 +300,7 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
     return MOE_ERR_INVALID_ARG;
   if (T * s.k > (int64_t(1) << 30)) return MOE_ERR_UNSUPPORTED;
   const WsLayout L = make_layout(s, T);
-  if (workspace_bytes < (training ? L.total : L.infer_total)) return MOE_ERR_WORKSPACE;
+  if (workspace_bytes < (lora ? L.lora_total : (training ? L.total : L.infer_total))) return MOE_ERR_WORKSPACE;
   moe_status rc = ensure_device(c);
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -322,12 +329,22 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
   if (T > 0) {
     {
       StageTimer tm(c, st, 2);
-      rc = launch_grouped_gemm(c, GEMM_F3, T, L, ws, io, st);
+      if (lora) {
+        rc = launch_lora_gemm(c, LORA_U, T, L, ws, io, *lora, st);
+        if (rc == MOE_OK) rc = launch_lora_gemm(c, LORA_F3, T, L, ws, io, *lora, st);
+      } else {
+        rc = launch_grouped_gemm(c, GEMM_F3, T, L, ws, io, st);
+      }
     }
     if (rc != MOE_OK) return rc;
     {
       StageTimer tm(c, st, 3);
-      rc = launch_grouped_gemm(c, GEMM_F4, T, L, ws, io, st);
+      if (lora) {
+        rc = launch_lora_gemm(c, LORA_V, T, L, ws, io, *lora, st);
+        if (rc == MOE_OK) rc = launch_lora_gemm(c, LORA_F4, T, L, ws, io, *lora, st);
+      } else {
+        rc = launch_grouped_gemm(c, GEMM_F4, T, L, ws, io, st);
+      }
     }
     if (rc != MOE_OK) return rc;
     {
@@ -367,13 +384,14 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
                                 const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
                                 const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
                                 uint16_t* dW_up, uint16_t* dW_down, float* acc_gate, float* acc_up, float* acc_down,
-                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                                void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                const LoraArgs* lora = nullptr) {
   const bool accumulate = acc_gate != nullptr;
   if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   const Shape& s = c->s;
   if (!W_r || !W_gate || !W_up || !W_down || !dW_r || !workspace) return MOE_ERR_INVALID_ARG;
-  if (accumulate ? (!acc_up || !acc_down) : (!dW_gate || !dW_up || !dW_down)) return MOE_ERR_INVALID_ARG;
+  if (!lora && (accumulate ? (!acc_up || !acc_down) : (!dW_gate || !dW_up || !dW_down))) return MOE_ERR_INVALID_ARG;
   if (accumulate && (!aligned16(acc_gate) || !aligned16(acc_up) || !aligned16(acc_down))) return MOE_ERR_INVALID_ARG;
   if (T > 0 && (!dy || !x || !dx)) return MOE_ERR_INVALID_ARG;
   if (!aligned16(dy) || !aligned16(x) || !aligned16(W_r) || !aligned16(W_gate) || !aligned16(W_up) ||
@@ -381,7 +399,7 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
       !aligned16(workspace))
     return MOE_ERR_INVALID_ARG;
   const WsLayout L = make_layout(s, T);
-  if (workspace_bytes < L.total) return MOE_ERR_WORKSPACE;
+  if (workspace_bytes < (lora ? L.lora_total : L.total)) return MOE_ERR_WORKSPACE;
   moe_status rc = ensure_device(c);
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -398,26 +416,39 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     StageTimer tm(c, st, 5);
     launch_gather_rows(s, T, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st);
   }
-  if (T > 0) {
-    StageTimer tm(c, st, 6);
-    rc = launch_grouped_gemm(c, GEMM_B2, T, L, ws, io, st);
+  if (lora) {
+    // base weights frozen: no dW_gate / dW_up / dW_down; the adapter gradients come from skinny GEMMs
+    const LoraOp seq[] = {LORA_W, LORA_B2, LORA_DB2, LORA_DA2, LORA_Z, LORA_B4, LORA_DB1, LORA_DA1};
+    const int stage_of[] = {6, 6, 7, 7, 8, 8, 9, 9};
+    for (int i = 0; i < 8 && rc == MOE_OK; ++i) {
+      const bool row_op = seq[i] == LORA_W || seq[i] == LORA_B2 || seq[i] == LORA_Z || seq[i] == LORA_B4;
+      if (row_op && T == 0) continue;
+      StageTimer tm(c, st, stage_of[i]);
+      rc = launch_lora_gemm(c, seq[i], T, L, ws, io, *lora, st);
+    }
+    if (rc != MOE_OK) return rc;
+  } else {
+    if (T > 0) {
+      StageTimer tm(c, st, 6);
+      rc = launch_grouped_gemm(c, GEMM_B2, T, L, ws, io, st);
+    }
+    if (rc != MOE_OK) return rc;
+    {
+      StageTimer tm(c, st, 7);
+      rc = launch_grouped_gemm(c, GEMM_B3, T, L, ws, io, st);
+    }
+    if (rc != MOE_OK) return rc;
+    if (T > 0) {
+      StageTimer tm(c, st, 8);
+      rc = launch_grouped_gemm(c, GEMM_B4, T, L, ws, io, st);
+    }
+    if (rc != MOE_OK) return rc;
+    {
+      StageTimer tm(c, st, 9);
+      rc = launch_grouped_gemm(c, GEMM_B5, T, L, ws, io, st);
+    }
+    if (rc != MOE_OK) return rc;
   }
-  if (rc != MOE_OK) return rc;
-  {
-    StageTimer tm(c, st, 7);
-    rc = launch_grouped_gemm(c, GEMM_B3, T, L, ws, io, st);
-  }
-  if (rc != MOE_OK) return rc;
-  if (T > 0) {
-    StageTimer tm(c, st, 8);
-    rc = launch_grouped_gemm(c, GEMM_B4, T, L, ws, io, st);
-  }
-  if (rc != MOE_OK) return rc;
-  {
-    StageTimer tm(c, st, 9);
-    rc = launch_grouped_gemm(c, GEMM_B5, T, L, ws, io, st);
-  }
-  if (rc != MOE_OK) return rc;
   {
     StageTimer tm(c, st, 10);
     launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
@@ -465,6 +496,52 @@ moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16_t* dy, 
   if (!dW_gate || !dW_up || !dW_down) return MOE_ERR_INVALID_ARG;
   return backward_impl(ctx, T, dy, d_aux, x, W_r, W_gate, W_up, W_down, dx, dW_r, db_r, nullptr, nullptr, nullptr, dW_gate,
                        dW_up, dW_down, workspace, workspace_bytes, cuda_stream);
+}
+
+// ------------------------------------------------------------------------------------------ expert LoRA
+static bool lora_args_ok(const moe_ctx_impl* c, int32_t rank, const void* A1, const void* B1g, const void* B1u,
+                         const void* A2, const void* B2) {
+  (void)c;
+  return rank >= 8 && rank <= 64 && rank % 8 == 0 && A1 && B1g && B1u && A2 && B2 && aligned16(A1) && aligned16(B1g) &&
+         aligned16(B1u) && aligned16(A2) && aligned16(B2);
+}
+
+size_t moe_lora_workspace_bytes(const moe_ctx* ctx, int64_t T) {
+  if (!ctx || T < 0) return 0;
+  return make_layout(reinterpret_cast<const moe_ctx_impl*>(ctx)->s, T).lora_total;
+}
+
+moe_status moe_lora_forward(moe_ctx* ctx, int64_t T, int32_t rank, float scale, const uint16_t* x, const uint16_t* W_r,
+                            const float* b_r, const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
+                            const uint16_t* A1, const uint16_t* B1_gate, const uint16_t* B1_up, const uint16_t* A2,
+                            const uint16_t* B2, uint16_t* y, int32_t* topk_idx, float* topk_w, int32_t* expert_counts,
+                            float* aux_loss, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !lora_args_ok(reinterpret_cast<moe_ctx_impl*>(ctx), rank, A1, B1_gate, B1_up, A2, B2))
+    return MOE_ERR_INVALID_ARG;
+  LoraArgs lo;
+  lo.rank = rank; lo.scale = scale;
+  lo.A1 = A1; lo.B1g = B1_gate; lo.B1u = B1_up; lo.A2 = A2; lo.B2 = B2;
+  return forward_impl(true, ctx, T, x, W_r, b_r, nullptr, W_gate, W_up, W_down, y, topk_idx, topk_w, expert_counts,
+                      nullptr, aux_loss, nullptr, workspace, workspace_bytes, cuda_stream, &lo);
+}
+
+moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, float scale, const uint16_t* dy, float d_aux,
+                             const uint16_t* x, const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                             const uint16_t* W_down, const uint16_t* A1, const uint16_t* B1_gate,
+                             const uint16_t* B1_up, const uint16_t* A2, const uint16_t* B2, uint16_t* dx, float* dW_r,
+                             uint16_t* dA1, uint16_t* dB1_gate, uint16_t* dB1_up, uint16_t* dA2, uint16_t* dB2,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !lora_args_ok(reinterpret_cast<moe_ctx_impl*>(ctx), rank, A1, B1_gate, B1_up, A2, B2))
+    return MOE_ERR_INVALID_ARG;
+  if (!dA1 || !dB1_gate || !dB1_up || !dA2 || !dB2 || !aligned16(dA1) || !aligned16(dB1_gate) || !aligned16(dB1_up) ||
+      !aligned16(dA2) || !aligned16(dB2))
+    return MOE_ERR_INVALID_ARG;
+  LoraArgs lo;
+  lo.rank = rank; lo.scale = scale;
+  lo.A1 = A1; lo.B1g = B1_gate; lo.B1u = B1_up; lo.A2 = A2; lo.B2 = B2;
+  lo.dA1 = dA1; lo.dB1g = dB1_gate; lo.dB1u = dB1_up; lo.dA2 = dA2; lo.dB2 = dB2;
+  return backward_impl(ctx, T, dy, d_aux, x, W_r, W_gate, W_up, W_down, dx, dW_r, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, nullptr, nullptr, workspace, workspace_bytes, cuda_stream, &lo);
 }
 
 // ------------------------------------------------------------------------------------------ host-buffer step

@@ -57,6 +57,10 @@ struct WsLayout {
   size_t dxr;          // bf16[T * d]  router term of dx (dl W_r^T)
   size_t infer_total;  // bytes a forward-only call needs (tables, xp, act, o)
   size_t total;
+  // expert-LoRA calls only (beyond `total`): 64-wide row buffers u = s xp A1, v = s act A2, w = s dy B2^T,
+  // z = s (dhg B1g^T + dhu B1u^T), bf16 [rows_max, 64], columns beyond the rank are zero
+  size_t lora_u, lora_v, lora_w, lora_z;
+  size_t lora_total;
   int64_t rows_max;    // upper bound of the padded row total for T tokens
   int64_t max_m_tiles;
   int64_t tok_tiles;
@@ -134,6 +138,31 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
                                const GemmIO& io, cudaStream_t st);
 struct GemmParams;
 moe_status launch_pair_gemm(moe_ctx_impl* ctx, GemmKind kind, const GemmParams& p, cudaStream_t st);  // gemm2.cu
+// Low-rank adapters of an expert-LoRA call (all device pointers, bf16): A1 [E,d,r], B1g / B1u [E,r,f], A2 [E,f,r],
+// B2 [E,r,d]; gradients in the same shapes.
+struct LoraArgs {
+  int rank = 0;
+  float scale = 0.f;
+  const uint16_t *A1 = nullptr, *B1g = nullptr, *B1u = nullptr, *A2 = nullptr, *B2 = nullptr;
+  uint16_t *dA1 = nullptr, *dB1g = nullptr, *dB1u = nullptr, *dA2 = nullptr, *dB2 = nullptr;
+};
+enum LoraOp {
+  LORA_U = 0,  // u = s xp A1
+  LORA_F3,     // [hg|hu] = xp [Wg|Wu] + u [B1g|B1u], SwiGLU epilogue
+  LORA_V,      // v = s act A2
+  LORA_F4,     // o = act Wd + v B2
+  LORA_W,      // w = s dy_rows B2^T
+  LORA_B2,     // da = dy_rows Wd^T + w A2^T, SwiGLU-backward epilogue
+  LORA_DB2,    // dB2 = v^T dy_rows
+  LORA_DA2,    // dA2 = act^T w
+  LORA_Z,      // z = s (dhg B1g^T + dhu B1u^T)
+  LORA_B4,     // dxp = dhg Wg^T + dhu Wu^T + z A1^T
+  LORA_DB1,    // dB1g | dB1u = u^T [dhg | dhu]
+  LORA_DA1     // dA1 = xp^T z
+};
+moe_status launch_lora_gemm(moe_ctx_impl* ctx, LoraOp op, int64_t T, const WsLayout& L, char* ws, const GemmIO& io,
+                            const LoraArgs& lo, cudaStream_t st);
+
 // true when the tensor-core router / dW_r / dx kernels apply (their TMA maps need E % 8 == 0)
 inline bool router_on_tensor_cores(const Shape& s) { return s.E % 8 == 0; }
 // psum_part rows written by the router: one per warp of a 128-token tile (tensor cores) or per ROUTER_TOK tokens (SIMT)

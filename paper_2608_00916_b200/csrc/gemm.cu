@@ -479,4 +479,198 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   return MOE_ERR_INVALID_ARG;
 }
 
+// Backward operations of the expert-LoRA variant (see launch_lora_gemm below, which prepares `p`).
+static moe_status launch_lora_gemm_bwd(moe_ctx_impl* ctx, LoraOp op, int64_t T, const WsLayout& L, char* ws,
+                                       const GemmIO& io, const LoraArgs& lo, GemmParams p, cudaStream_t st) {
+  (void)T;
+  const Shape& s = ctx->s;
+  const int d = s.d, f = s.f, E = s.E, r = lo.rank;
+  const int64_t R = L.rows_max;
+  void* fn = ctx->encode_fn;
+  auto B16 = [&](size_t off) { return reinterpret_cast<uint16_t*>(ws + off); };
+  uint16_t *xp = B16(L.xp), *hg = B16(L.hg), *hu = B16(L.hu), *act = B16(L.act), *dyr = B16(L.o), *dhg = B16(L.dhg),
+           *dhu = B16(L.dhu), *dxp = B16(L.dxp), *u = B16(L.lora_u), *v = B16(L.lora_v), *w = B16(L.lora_w),
+           *z = B16(L.lora_z);
+  const uint32_t skinny_tx = A_BYTES + CHUNK_BYTES;
+  bool ok = true;
+  switch (op) {
+    case LORA_W:  // w[R,64] = s dy_rows B2[e]^T      (B4 kind, one segment, K-major B of 64 rows)
+      ok = map_2d(fn, &p.mapA0, dyr, R, d, 128) && map_3d(fn, &p.mapB0, lo.B2, E, r, d, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.n_tiles = 1;
+      p.k_blocks = d / BK;
+      p.nseg = 1;
+      p.mma_n = 64; p.stage_tx = skinny_tx;
+      p.N_total = 64;
+      p.out0 = w;
+      p.ld_out = 64;
+      p.out_scale = lo.scale;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B4>(ctx, p, st);
+    case LORA_Z:  // z[R,64] = s (dhg B1g[e]^T + dhu B1u[e]^T)   (B4 kind, two segments)
+      ok = map_2d(fn, &p.mapA0, dhg, R, f, 128) && map_2d(fn, &p.mapA1, dhu, R, f, 128) &&
+           map_3d(fn, &p.mapB0, lo.B1g, E, r, f, 64) && map_3d(fn, &p.mapB1, lo.B1u, E, r, f, 64);
+      p.n_tiles = 1;
+      p.k_blocks = f / BK;
+      p.nseg = 2;
+      p.mma_n = 64; p.stage_tx = skinny_tx;
+      p.N_total = 64;
+      p.out0 = z;
+      p.ld_out = 64;
+      p.out_scale = lo.scale;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B4>(ctx, p, st);
+    case LORA_B2:  // da = dy_rows Wd^T + w A2^T, SwiGLU-backward epilogue
+      ok = map_2d(fn, &p.mapA0, dyr, R, d, 128) && map_3d(fn, &p.mapB0, io.W_down, E, f, d, 256) &&
+           map_2d(fn, &p.mapA2, w, R, 64, 128) && map_3d(fn, &p.mapB2, lo.A2, E, f, r, 256);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.n_tiles = (f + 255) / 256;
+      p.k_blocks = d / BK;
+      p.k_blocks1 = 1;
+      p.N_total = f;
+      p.in0 = hg; p.in1 = hu;
+      p.out0 = dhg; p.out1 = dhu;
+      p.ld_out = f;
+      p.outf = reinterpret_cast<float*>(ws + L.dg_part);
+      p.rows_max = L.rows_max;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B2>(ctx, p, st);
+    case LORA_B4:  // dxp = dhg Wg^T + dhu Wu^T + z A1^T
+      ok = map_2d(fn, &p.mapA0, dhg, R, f, 128) && map_2d(fn, &p.mapA1, dhu, R, f, 128) &&
+           map_3d(fn, &p.mapB0, io.W_gate, E, d, f, 256) && map_3d(fn, &p.mapB1, io.W_up, E, d, f, 256) &&
+           map_2d(fn, &p.mapA2, z, R, 64, 128) && map_3d(fn, &p.mapB2, lo.A1, E, d, r, 256);
+      p.n_tiles = (d + 255) / 256;
+      p.k_blocks = f / BK;
+      p.nseg = 2;
+      p.k_blocks1 = 1;
+      p.N_total = d;
+      p.out0 = dxp;
+      p.ld_out = d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B4>(ctx, p, st);
+    case LORA_DB2:  // dB2[e][r,d] = v_e^T dy_rows_e      (B3 kind, M = rank)
+      ok = map_2d(fn, &p.mapA0, v, R, 64, 64) && map_2d(fn, &p.mapB0, dyr, R, d, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.m_tiles = 1;
+      p.n_tiles = (d + 255) / 256;
+      p.M_total = r;
+      p.N_total = d;
+      p.out0 = lo.dB2;
+      p.ld_out = d;
+      p.expert_stride = static_cast<int64_t>(r) * d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B3>(ctx, p, st);
+    case LORA_DA2:  // dA2[e][f,r] = act_e^T w_e           (B3 kind, N = rank)
+    case LORA_DA1:  // dA1[e][d,r] = xp_e^T z_e
+      ok = map_2d(fn, &p.mapA0, op == LORA_DA2 ? act : xp, R, op == LORA_DA2 ? f : d, 64) &&
+           map_2d(fn, &p.mapB0, op == LORA_DA2 ? w : z, R, 64, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.M_total = op == LORA_DA2 ? f : d;
+      p.m_tiles = (p.M_total + 127) / 128;
+      p.n_tiles = 1;
+      p.b_chunks = 1; p.mma_n = 64; p.stage_tx = skinny_tx;
+      p.N_total = r;
+      p.out0 = op == LORA_DA2 ? lo.dA2 : lo.dA1;
+      p.ld_out = r;
+      p.expert_stride = static_cast<int64_t>(p.M_total) * r;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B3>(ctx, p, st);
+    case LORA_DB1:  // dB1g[e] | dB1u[e] [r,f] = u_e^T [dhg_e | dhu_e]   (B5 kind, M = rank)
+      ok = map_2d(fn, &p.mapA0, u, R, 64, 64) && map_2d(fn, &p.mapB0, dhg, R, f, 64) &&
+           map_2d(fn, &p.mapB1, dhu, R, f, 64);
+      p.mapA1 = p.mapA0;
+      p.m_tiles = 1;
+      p.n_tiles = (f + 127) / 128;
+      p.M_total = r;
+      p.N_total = f;
+      p.out0 = lo.dB1g; p.out1 = lo.dB1u;
+      p.ld_out = f;
+      p.expert_stride = static_cast<int64_t>(r) * f;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_B5>(ctx, p, st);
+    default:
+      break;
+  }
+  return MOE_ERR_INVALID_ARG;
+}
+
+// ------------------------------------------------------------------------------------------ expert LoRA
+// The adapted layer reuses the kernels above with different operands: the low-rank path enters each row GEMM as one
+// extra 64-deep K segment ([xp | u] [[W]; [B1]], ...), the four 64-wide row buffers u, v, w, z come from skinny
+// instances (N = 64) of the F4 / B4 kinds, and the adapter gradients from instances of the B3 / B5 kinds whose M or
+// N is the rank.  All on one-CTA tiles.
+moe_status launch_lora_gemm(moe_ctx_impl* ctx, LoraOp op, int64_t T, const WsLayout& L, char* ws, const GemmIO& io,
+                            const LoraArgs& lo, cudaStream_t st) {
+  const Shape& s = ctx->s;
+  const int d = s.d, f = s.f, E = s.E, r = lo.rank;
+  const int64_t R = L.rows_max;
+  void* fn = ctx->encode_fn;
+  auto B16 = [&](size_t off) { return reinterpret_cast<uint16_t*>(ws + off); };
+  uint16_t *xp = B16(L.xp), *hg = B16(L.hg), *hu = B16(L.hu), *act = B16(L.act), *o = B16(L.o), *dhg = B16(L.dhg),
+           *dhu = B16(L.dhu), *dxp = B16(L.dxp), *u = B16(L.lora_u), *v = B16(L.lora_v), *w = B16(L.lora_w),
+           *z = B16(L.lora_z);
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.sched = reinterpret_cast<const int32_t*>(ws + L.sched);
+  p.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
+  p.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+  p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
+  p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
+  p.status = reinterpret_cast<int32_t*>(ws + L.status);
+  p.E = E;
+  p.b_chunks = 4;
+  p.mma_n = BN;
+  p.stage_tx = STAGE_BYTES;
+  p.nseg = 1;
+  p.out_scale = 1.f;
+  p.row_gate = reinterpret_cast<const float*>(ws + L.row_gate);
+  const uint32_t skinny_tx = A_BYTES + CHUNK_BYTES;  // a 128 x 64 A tile and one 64 x 64 B tile
+  bool ok = true;
+  switch (op) {
+    case LORA_U:  // u[R,64] = s xp A1[e]            (F4 kind, N = 64)
+    case LORA_V:  // v[R,64] = s act A2[e]
+      ok = map_2d(fn, &p.mapA0, op == LORA_U ? xp : act, R, op == LORA_U ? d : f, 128) &&
+           map_3d(fn, &p.mapB0, op == LORA_U ? lo.A1 : lo.A2, E, op == LORA_U ? d : f, r, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.n_tiles = 1;
+      p.k_blocks = (op == LORA_U ? d : f) / BK;
+      p.b_chunks = 1; p.mma_n = 64; p.stage_tx = skinny_tx;
+      p.N_total = 64;
+      p.out0 = op == LORA_U ? u : v;
+      p.ld_out = 64;
+      p.out_scale = lo.scale;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_F4>(ctx, p, st);
+    case LORA_F3:  // [hg|hu] = xp [Wg|Wu] + u [B1g|B1u]
+      ok = map_2d(fn, &p.mapA0, xp, R, d, 128) && map_3d(fn, &p.mapB0, io.W_gate, E, d, f, 64) &&
+           map_3d(fn, &p.mapB1, io.W_up, E, d, f, 64) && map_2d(fn, &p.mapA2, u, R, 64, 128) &&
+           map_3d(fn, &p.mapB2, lo.B1g, E, r, f, 64) && map_3d(fn, &p.mapB3, lo.B1u, E, r, f, 64);
+      p.mapA1 = p.mapA0;
+      p.n_tiles = (f + 127) / 128;
+      p.k_blocks = d / BK;
+      p.k_blocks1 = 1;
+      p.N_total = f;
+      p.out0 = hg; p.out1 = hu; p.out2 = act;
+      p.ld_out = f;
+      p.save_pre = 1;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_F3>(ctx, p, st);
+    case LORA_F4:  // o = act Wd + v B2
+      ok = map_2d(fn, &p.mapA0, act, R, f, 128) && map_3d(fn, &p.mapB0, io.W_down, E, f, d, 64) &&
+           map_2d(fn, &p.mapA2, v, R, 64, 128) && map_3d(fn, &p.mapB2, lo.B2, E, r, d, 64);
+      p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      p.n_tiles = (d + 255) / 256;
+      p.k_blocks = f / BK;
+      p.k_blocks1 = 1;
+      p.N_total = d;
+      p.out0 = o;
+      p.ld_out = d;
+      if (!ok) return MOE_ERR_CUDA;
+      return launch_kind<GEMM_F4>(ctx, p, st);
+    default:
+      break;
+  }
+  return launch_lora_gemm_bwd(ctx, op, T, L, ws, io, lo, p, st);
+}
+
 }  // namespace moe

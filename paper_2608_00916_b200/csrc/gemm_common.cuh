@@ -491,17 +491,12 @@ __device__ __forceinline__ void epilogue_prefetch(const GemmParams& p, int64_t r
 template <int KIND>
 __device__ __forceinline__ void wgrad_zero_fill(const GemmParams& p, int e, int m, int n0) {
   if (m >= p.M_total || p.acc_fp32) return;  // accumulate mode: an expert without tokens adds nothing
-  float z[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) z[i] = 0.f;
-  for (int c = 0; c < 8; ++c) {
-    uint16_t* base = p.out0;
-    int col = n0 + c * 32;
-    if (KIND == GEMM_B5) {
-      base = (c >= 4) ? p.out1 : p.out0;
-      col = n0 + (c & 3) * 32;
-    }
-    if (col < p.N_total) store_bf16x32(base + e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + col, z);
+  constexpr int span = (KIND == GEMM_B5) ? 128 : 256;
+  const int cols = min(span, p.N_total - n0);
+  for (int c = 0; c < cols; c += 8) {  // 16-byte pieces: the output width is a multiple of 8
+    const int64_t off = e * p.expert_stride + static_cast<int64_t>(m) * p.ld_out + n0 + c;
+    *reinterpret_cast<uint4*>(p.out0 + off) = make_uint4(0, 0, 0, 0);
+    if (KIND == GEMM_B5) *reinterpret_cast<uint4*>(p.out1 + off) = make_uint4(0, 0, 0, 0);
   }
 }
 

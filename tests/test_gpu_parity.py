@@ -322,6 +322,47 @@ def test_step_host_matches_the_device_path():
         assert torch.equal(host[n], bw[n].view(torch.int16).cpu()), n
 
 
+@pytest.mark.parametrize("T,d,E,k,f,rank,seed", [
+    (600, 256, 8, 2, 256, 16, 71),    # the paper's rank
+    (1000, 512, 16, 4, 384, 16, 72),  # ragged tails, f not a multiple of 256
+    (333, 192, 5, 3, 320, 8, 73),     # smallest rank, SIMT router path, widths not multiples of 128
+    (257, 128, 12, 12, 64, 64, 74),   # largest rank, k = E
+    (50, 128, 32, 2, 128, 24, 75),    # most experts empty
+])
+def test_expert_lora_against_the_oracle(T, d, E, k, f, rank, seed):
+    """Expert LoRA through moe_lora_forward / moe_lora_backward against the oracle's definition (the plain layer
+    evaluated with W + s A B; adapter gradients by the chain rule from the effective-weight gradients)."""
+    shape = synth.MoEShape(T, d, E, k, f)
+    inp = synth.make_inputs(shape, seed, x_std=1.0)
+    lo = synth.make_lora(shape, seed, rank=rank, std=0.05)
+    scale = 2.0
+    wargs = (inp["W_gate"], inp["W_up"], inp["W_down"], lo["A1"], lo["B1_gate"], lo["B1_up"], lo["A2"], lo["B2"], scale)
+    ofw = orc.lora_forward(inp["x"], inp["W_r"], *wargs, k)
+    obw = orc.lora_backward(ofw, inp["dy"], 0.02, inp["x"], inp["W_r"], *wargs)
+    # the adapters must matter in this test: the adapted output differs visibly from the base layer's
+    base = orc.forward(inp["x"], inp["W_r"], inp["W_gate"], inp["W_up"], inp["W_down"], k)
+    assert rel_fro(base["y"], ofw["y"]) > 0.05
+    from gpu_util import to_dev_bf16
+    r = Run(inp, k)
+    v = r.dev
+    dlo = {n: to_dev_bf16(lo[n]) for n in ("A1", "B1_gate", "B1_up", "A2", "B2")}
+    fw = r.layer.lora_forward(v["x"], v["W_r"], v["W_gate"], v["W_up"], v["W_down"], dlo, scale)
+    r.layer.poll()
+    assert np.array_equal(fw["idx"].cpu().numpy(), ofw["idx"])
+    assert np.array_equal(fw["counts"].cpu().numpy(), ofw["counts"])
+    assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+    bw = r.layer.lora_backward(v["dy"], 0.02)
+    r.layer.poll()
+    assert rel_fro(from_dev_bf16(bw["dx"]), obw["dx"]) <= TOL
+    assert rel_fro(bw["dW_r"].cpu().numpy(), obw["dW_r"]) <= TOL
+    for n in ("dA1", "dB1_gate", "dB1_up", "dA2", "dB2"):
+        got = from_dev_bf16(bw[n])
+        assert rel_fro(got, obw[n]) <= TOL, n
+        for e in range(E):
+            if ofw["counts"][e] == 0:
+                assert not got[e].any(), (n, e)
+
+
 def test_bounded_wait_reports_timeout_and_context_survives():
     """A device-side wait that can never complete gives up, the status word says so, and the same context and
     workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
