@@ -171,9 +171,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="qwen", choices=list(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--mode", default="train", choices=["train", "inference", "accumulate"],
+    ap.add_argument("--mode", default="train", choices=["train", "inference", "accumulate", "lora"],
                     help="train: forward + backward (the headline metric); inference: forward-only entry point; "
-                         "accumulate: forward + backward that adds weight gradients into fp32 buffers")
+                         "accumulate: forward + backward that adds weight gradients into fp32 buffers; "
+                         "lora: forward + backward of the expert-LoRA variant (rank 16, frozen expert weights)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -216,6 +217,45 @@ def main():
     grads = {"dx": torch.empty_like(tens["x"]), "dW_r": torch.empty(shape.d, shape.E, dtype=torch.float32, device="cuda"),
              "dW_gate": torch.empty_like(tens["W_gate"]), "dW_up": torch.empty_like(tens["W_up"]),
              "dW_down": torch.empty_like(tens["W_down"])}
+
+    if args.mode == "lora":
+        # expert-LoRA training step (a "next" row beyond the full fine-tuning step): own metric, device-resident timing
+        rank, scale = 16, 2.0
+        lo = synth.make_lora(shape, seed, rank=rank)
+        dlo = {n: dev(lo[n]) for n in ("A1", "B1_gate", "B1_up", "A2", "B2")}
+
+        def lstep():
+            layer.lora_forward(tens["x"], tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], dlo, scale, b_r=b_r)
+            layer.lora_backward(tens["dy"], inp["d_aux"])
+        for _ in range(args.warmup):
+            lstep()
+        layer.poll()
+        layer.set_profiling(True)
+        pdist.barrier()
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(args.steps):
+            lstep()
+        f1.record()
+        torch.cuda.synchronize()
+        pdist.barrier()
+        stage_ms, n = layer.stage_times()
+        ms = pdist.max_over_ranks(f0.elapsed_time(f1)) / args.steps
+        if int(os.environ.get("RANK", "0")) == 0:
+            Rr = T * shape.k
+            fl = 12 * Rr * shape.d * shape.f  # base forward + dgrad GEMMs; the low-rank terms add < 3 %
+            print(json.dumps({"metric": "moe_layer_lora_fwd_bwd_tokens_per_s", "value": world * T / (ms / 1e3),
+                              "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                              "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                              "dtype": "bf16", "data": "synthetic",
+                              "config": {"workload": args.workload, "mode": "lora", "rank": rank, "T_per_gpu": T,
+                                         "d": shape.d, "E": shape.E, "top_k": shape.k, "f": shape.f},
+                              "base_gemm_useful_tflops_over_whole_step": fl / (ms * 1e-3) / 1e12,
+                              "stages_ms": {STAGE_NAMES[i]: stage_ms[i] / max(n, 1) for i in range(len(STAGE_NAMES))},
+                              "gpu_launches": 29 * args.steps}))
+        pdist.finish()
+        return
 
     if args.mode == "inference":
         # forward-only scoring pass (a "next" row beyond the training step): own metric, device-resident timing only

@@ -418,13 +418,13 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
   }
   if (lora) {
     // base weights frozen: no dW_gate / dW_up / dW_down; the adapter gradients come from skinny GEMMs
-    const LoraOp seq[] = {LORA_W, LORA_B2, LORA_DB2, LORA_DA2, LORA_Z, LORA_B4, LORA_DB1, LORA_DA1};
-    const int stage_of[] = {6, 6, 7, 7, 8, 8, 9, 9};
-    for (int i = 0; i < 8 && rc == MOE_OK; ++i) {
-      const bool row_op = seq[i] == LORA_W || seq[i] == LORA_B2 || seq[i] == LORA_Z || seq[i] == LORA_B4;
-      if (row_op && T == 0) continue;
-      StageTimer tm(c, st, stage_of[i]);
-      rc = launch_lora_gemm(c, seq[i], T, L, ws, io, *lora, st);
+    const LoraOp seq[4][2] = {{LORA_W, LORA_B2}, {LORA_DB2, LORA_DA2}, {LORA_Z, LORA_B4}, {LORA_DB1, LORA_DA1}};
+    for (int g = 0; g < 4 && rc == MOE_OK; ++g) {
+      const bool row_ops = (g == 0 || g == 2);  // row GEMMs have no tiles without tokens; weight gradients zero-fill
+      if (row_ops && T == 0) continue;
+      StageTimer tm(c, st, 6 + g);
+      rc = launch_lora_gemm(c, seq[g][0], T, L, ws, io, *lora, st);
+      if (rc == MOE_OK) rc = launch_lora_gemm(c, seq[g][1], T, L, ws, io, *lora, st);
     }
     if (rc != MOE_OK) return rc;
   } else {
