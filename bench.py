@@ -27,8 +27,8 @@ import numpy as np  # noqa: E402
 from paper_2608_00916_b200 import synth  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-LAUNCHES_PER_STEP = 19  # router, hist, scan, scatter, gather, 2 GEMMs, combine; gather(dy), 4 GEMMs, router-bwd,
-#                         dW_r GEMM + reduce, dx-router GEMM + unpermute-sum
+LAUNCHES_PER_STEP = 18  # router, hist, scan, scatter, row scatter, 2 GEMMs, combine; row scatter (dy), 4 GEMMs,
+#                         router-bwd, dW_r GEMM + reduce, dx-router GEMM + unpermute-sum (profiles/launch_list_qwen.md)
 # dram bytes per launch of the dominant kernel taken from the committed ncu capture (profiles/), by stage name;
 # None where no capture has been taken for the workload.
 NCU_TRAFFIC = {  # profiles/grouped_gemms_qwen_dram_traffic.md
