@@ -80,7 +80,6 @@ struct Traits {
   static constexpr bool STATIC_M = (KIND == GEMM_RT || KIND == GEMM_DX);  // token tiles, no expert lookup
   static constexpr int A_MN = WGRAD ? 1 : 0;
   static constexpr int B_MN = (KIND == GEMM_B2 || KIND == GEMM_B4 || KIND == GEMM_DX) ? 0 : 1;
-  static constexpr int NSEG = (KIND == GEMM_B4 || KIND == GEMM_DX) ? 2 : 1;
   // width of output covered by one N tile (F3 / B5 / DWR pair a 128-wide tile with a second 128-wide operand)
   static constexpr int N_SPAN = (KIND == GEMM_F3 || KIND == GEMM_B5 || KIND == GEMM_DWR) ? 128 : 256;
 };
@@ -201,29 +200,6 @@ __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl,
   }
 }
 
-__device__ __forceinline__ void store_bf16x32(uint16_t* dst, const float (&v)[32]) {
-  uint4* q = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint4 w;
-    w.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);
-    w.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
-    w.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
-    w.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
-    q[i] = w;
-  }
-}
-__device__ __forceinline__ void load_bf16x32(const uint16_t* src, float (&v)[32]) {
-  const uint4* q = reinterpret_cast<const uint4*>(src);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint4 w = q[i];
-    unpack_bf16x2(w.x, v[8 * i + 0], v[8 * i + 1]);
-    unpack_bf16x2(w.y, v[8 * i + 2], v[8 * i + 3]);
-    unpack_bf16x2(w.z, v[8 * i + 4], v[8 * i + 5]);
-    unpack_bf16x2(w.w, v[8 * i + 6], v[8 * i + 7]);
-  }
-}
 __device__ __forceinline__ float fast_sigmoid(float h) { return __fdividef(1.f, 1.f + __expf(-h)); }
 
 
