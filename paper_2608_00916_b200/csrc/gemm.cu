@@ -323,13 +323,16 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
   p.timers = getenv("MOE_GEMM_TIMERS") ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
   // CTA pairs (256 x 256 tiles, half of B per SM) or one-CTA tiles (128 x 256)?  Pairs move a third less operand
-  // data per flop, which under the power cap is worth ~12 % on long-K shapes; their cost is the dummy half-tile of
-  // every expert with an odd number of 128-row blocks (row GEMMs only).  Weight gradients pair along the weight
-  // dimension and have no such waste, so they always pair; row GEMMs pair when the expected waste (64 rows per
-  // expert) stays under 3 % of the routed rows.
+  // data per flop, which under the power cap is worth ~10 % on long-K tiles.  Row GEMMs pay for them with the dummy
+  // half-tile of every expert that has an odd number of 128-row blocks, so they pair only when that expected waste
+  // (64 rows per expert) stays under 3 % of the routed rows.  Weight gradients pair along the weight dimension
+  // without waste, but their K loop is the expert's row count: below ~768 rows per expert the epilogue (two coupled
+  // CTAs draining one tile) bounds them and one-CTA tiles are faster (measured: 512 rows/expert 232 vs 247 us,
+  // 1024 rows/expert 392 vs 350 us for the down-projection gradient at the Qwen3-30B-A3B shape).
   const bool wgrad_kind = kind == GEMM_B3 || kind == GEMM_B5;
+  const double rows_per_expert = static_cast<double>(T) * s.k / E;
   const bool pair = ctx->tile_mode == 1 ||
-                    (ctx->tile_mode == 0 && (wgrad_kind || 64.0 * E < 0.03 * static_cast<double>(T) * s.k));
+                    (ctx->tile_mode == 0 && (wgrad_kind ? rows_per_expert >= 768.0 : 64.0 < 0.03 * rows_per_expert));
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
   p.b_chunks = 4;
