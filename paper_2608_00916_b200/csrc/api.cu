@@ -48,7 +48,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.infer_total = off;  // everything above is all a forward-only call touches
   L.hg = take(rows_f);
   L.hu = take(rows_f);
-  L.dg_part = take(sizeof(float) * ((s.f + 255) / 256) * L.rows_max);
+  L.dg_part = take(sizeof(float) * 2 * ((s.f + 255) / 256) * L.rows_max);
   L.dg = take(sizeof(float) * R);
   L.dl = take(sizeof(float) * T * s.E);
   L.dl_hi = take(sizeof(uint16_t) * (T * s.E + 64));
@@ -452,7 +452,7 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
   {
     StageTimer tm(c, st, 10);
     launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
-                      gates, reinterpret_cast<const float*>(ws + L.dg_part), (s.f + 255) / 256, L.rows_max, inv,
+                      gates, reinterpret_cast<const float*>(ws + L.dg_part), 2 * ((s.f + 255) / 256), L.rows_max, inv,
                       reinterpret_cast<float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts), d_aux, dl,
                       reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo), st);
   }

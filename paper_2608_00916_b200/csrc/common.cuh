@@ -44,7 +44,7 @@ struct WsLayout {
   size_t gates;        // float[T*k]
   size_t inv;          // int32[T*k]  padded row of pair (t, j)
   size_t row_gate;     // float[rows_max] gate of a padded row, 0 for pad rows
-  size_t dg_part;      // float[ceil(f/256) * rows_max] per-row partial sums of dg, one slice per dgrad-down column tile
+  size_t dg_part;      // float[2 * ceil(f/256) * rows_max] per-row partial sums of dg, two slices per dgrad-down column tile
   size_t dg;           // float[T*k]
   size_t dl;           // float[T*E]
   size_t dl_hi, dl_lo; // bf16[T*E]   dl split into two bf16 terms (hi + lo) for the tensor-core contractions

@@ -27,14 +27,16 @@
 namespace moe {
 
 template <int KIND>
-__global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __grid_constant__ GemmParams p) {
+__global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
+    grouped_gemm_kernel(const __grid_constant__ GemmParams p) {
   using TR = Traits<KIND>;
+  constexpr int EPI_WARPS = (KIND == GEMM_RT) ? 4 : 8;
   extern __shared__ unsigned char gemm_smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
   __shared__ uint32_t tmem_base_slot;
   __shared__ float s_bias[KIND == GEMM_RT ? MAX_E : 1];  // router bias (zero beyond E)
   if (KIND == GEMM_RT)
-    for (int i = threadIdx.x; i < MAX_E; i += GEMM_THREADS) s_bias[i] = (p.bias && i < p.N_total) ? p.bias[i] : 0.f;
+    for (int i = threadIdx.x; i < MAX_E; i += blockDim.x) s_bias[i] = (p.bias && i < p.N_total) ? p.bias[i] : 0.f;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(gemm_smem_raw) + 1023u) & ~1023u;
@@ -51,7 +53,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 128);
+      mbar_init(tempty_bar(a), 32 * EPI_WARPS);
     }
     fence_mbar_init();
     tma_prefetch_desc(&p.mapA0);
@@ -160,10 +162,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       atomicExch(p.status, DEV_TIMEOUT);
       p.status[1] = 200 + KIND;
     }
-  } else {
-    // ------------------------------------------------------------------ epilogue (4 warps, 128 TMEM lanes)
-    const int ew = warp & 3;  // TMEM lane quadrant this warp may read
-    EpiStage es{smem_base + STAGES * STAGE_BYTES + ew * (EPI_UNITS * EPI_UNIT_BYTES), 0u};
+  } else if (warp < 2 + EPI_WARPS) {
+    // ------------------------------------------------------------------ epilogue (128 TMEM lanes; two warps per
+    // lane quadrant, each draining half of the tile's columns - the routing epilogue needs whole rows and uses one)
+    const int ew = warp & 3;           // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;  // which half of the columns
+    constexpr int NHALF = EPI_WARPS / 4;
+    EpiStage es{smem_base + STAGES * STAGE_BYTES + (warp - 2) * (EPI_UNITS * EPI_UNIT_BYTES), 0u};
     uint32_t tc = 0;
     bool ok = true;
     long long t_idle = 0, t_begin = clock64();
@@ -174,6 +179,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       const int rin = ew * 32 + lane;  // row inside the tile
       if (tl.nkb == 0) {
         // weight gradient of an expert without tokens: zeros
+        if (half != 0) continue;
         if (KIND == GEMM_DWR) {
           const int m = tl.m0 + rin;
           if (m < p.M_total)
@@ -188,7 +194,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
-      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, true, tl.e, tl.m0 + rin);
+      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, half == 0, tl.e, tl.m0 + rin);
       const long long w0 = clock64();
       if (!mbar_wait(tfull_bar(acc), aph)) {
         ok = false;
@@ -201,7 +207,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       if (KIND == GEMM_F3 || KIND == GEMM_B2) {
         expert_epilogue<KIND>(p, tl.e, row, (TR::WGRAD ? tl.m0 : tl.row0) + ew * 32, tl.n0, taddr, true,
                               TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
-                              es, lane);
+                              es, lane, half, NHALF);
       } else if (KIND == GEMM_RT) {
         if (p.N_total <= 128)
           routing_epilogue_regs(p, s_bias, row, tl.row0 / BM, ew, taddr, lane);
@@ -211,7 +217,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
         // fp32 partial of dW_r for this token slice: hi and lo halves of dl share one accumulator pair
         const int m = tl.m0 + rin;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 2 * half; c < 2 * half + 2; ++c) {
           uint32_t rh[32], rl[32];
           tmem_ld32(taddr + c * 32, rh);
           tmem_ld32(taddr + 128 + c * 32, rl);
@@ -232,12 +238,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
       } else {
         expert_epilogue<KIND>(p, tl.e, row, (TR::WGRAD ? tl.m0 : tl.row0) + ew * 32, tl.n0, taddr, true,
                               TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
-                              es, lane);
+                              es, lane, half, NHALF);
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
     }
-    if (p.timers && lane == 0 && ew == 0) {
+    if (p.timers && lane == 0 && ew == 0 && half == 0) {
       atomicAdd(p.timers + 5, static_cast<unsigned long long>(clock64() - t_begin));  // epilogue warp: total
       atomicAdd(p.timers + 6, static_cast<unsigned long long>(t_idle));               // waiting for a finished accumulator
       atomicAdd(p.timers + 7, 1ull);                                                  // CTAs counted
@@ -294,7 +300,7 @@ static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream
       return MOE_ERR_CUDA;
     attr_done[KIND] = true;
   }
-  grouped_gemm_kernel<KIND><<<ctx->sm_count, GEMM_THREADS, GEMM_SMEM, st>>>(p);
+  grouped_gemm_kernel<KIND><<<ctx->sm_count, KIND == GEMM_RT ? 192 : GEMM_THREADS, GEMM_SMEM, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

@@ -20,7 +20,7 @@
 namespace moe {
 
 constexpr int STAGES2 = 6;
-constexpr int GEMM2_THREADS = GEMM_THREADS;
+constexpr int GEMM2_THREADS = 192;  // warps: 0 TMA producer, 1 MMA issuer, 2..5 epilogue
 constexpr int BH_BYTES = 128 * BK * 2;              // this CTA's half of B: 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;    // 32 KB
 constexpr size_t GEMM2_SMEM = static_cast<size_t>(STAGES2) * STAGE2_BYTES + EPI_BYTES + 1024;

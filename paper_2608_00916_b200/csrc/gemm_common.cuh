@@ -12,14 +12,15 @@ constexpr int A_BYTES = BM * BK * 2;       // 16 KB
 constexpr int B_BYTES = BN * BK * 2;       // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-major tile: 8 KB
-constexpr int GEMM_THREADS = 192;  // warps: 0 TMA producer, 1 MMA issuer, 2..5 epilogue
+constexpr int GEMM_THREADS = 320;  // one-CTA kernel, warps: 0 TMA producer, 1 MMA issuer, 2..9 epilogue (two per TMEM lane
+                                   // quadrant, each taking half of the tile's columns)
 constexpr int ACC_COLS = 256;
 constexpr int TMEM_COLS = 512;
 // Epilogue staging: every epilogue warp owns EPI_UNITS units of 32 rows x 32 bf16 columns (64-byte rows, XOR
 // swizzle) through which it transposes its results for coalesced global stores.
 constexpr int EPI_UNIT_BYTES = 32 * 64;
 constexpr int EPI_UNITS = 2;
-constexpr int EPI_BYTES = 4 * EPI_UNITS * EPI_UNIT_BYTES;  // 4 epilogue warps: 32 KB
+constexpr int EPI_BYTES = 8 * EPI_UNITS * EPI_UNIT_BYTES;  // up to 8 epilogue warps: 32 KB
 constexpr size_t GEMM_SMEM = static_cast<size_t>(STAGES) * STAGE_BYTES + EPI_BYTES + 1024;
 
 struct GemmParams {
@@ -288,10 +289,14 @@ __device__ __forceinline__ void stage_accum32(EpiStage& es, float* out, int64_t 
 // clips a slab that overhangs the tensor.  Every tcgen05.ld is executed by all lanes.
 template <int KIND>
 __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int64_t row, int slab, int n0,
-                                                uint32_t taddr, bool write, int rows_valid, EpiStage& es, int lane) {
+                                                uint32_t taddr, bool write, int rows_valid, EpiStage& es, int lane,
+                                                int half = 0, int nhalf = 1) {
+  // with two epilogue warps per lane quadrant (nhalf = 2) this warp handles half of the 32-column chunks
+  const int c4_lo = half * (4 / nhalf), c4_hi = c4_lo + 4 / nhalf;  // of 4 chunks (F3: gate + up pairs)
+  const int c8_lo = half * (8 / nhalf), c8_hi = c8_lo + 8 / nhalf;  // of 8 chunks
   if (KIND == GEMM_F3) {
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
+    for (int c = c4_lo; c < c4_hi; ++c) {
       uint32_t rg[32], ru[32];
       tmem_ld32(taddr + c * 32, rg);
       tmem_ld32(taddr + 128 + c * 32, ru);
@@ -321,10 +326,10 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
     uint4 nh[4], nu[4];
     const float gate = write ? p.row_gate[row] : 0.f;
     float dgp = 0.f;  // this row's share of dg = <dy, o> = <da, silu(hg) hu> over the tile's columns
-    const bool rd0 = write && n0 < p.N_total;
+    const bool rd0 = write && n0 + c8_lo * 32 < p.N_total;
     if (rd0) {
-      const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + n0);
-      const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + n0);
+      const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + n0 + c8_lo * 32);
+      const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + n0 + c8_lo * 32);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         nh[i] = __ldg(qh + i);
@@ -332,7 +337,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       }
     }
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
+    for (int c = c8_lo; c < c8_hi; ++c) {
       uint4 ch[4], cu[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -340,7 +345,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
         cu[i] = nu[i];
       }
       const int col = n0 + c * 32;
-      if (write && c + 1 < 8 && col + 32 < p.N_total) {
+      if (write && c + 1 < c8_hi && col + 32 < p.N_total) {
         const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + col + 32);
         const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + col + 32);
 #pragma unroll
@@ -378,7 +383,11 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
         stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
       }
     }
-    if (write) p.outf[static_cast<int64_t>(n0 / 256) * p.rows_max + row] = dgp;
+    // two partial slices per column tile, one per epilogue warp of the lane quadrant
+    if (write) {
+      p.outf[static_cast<int64_t>(n0 / 256 * 2 + half) * p.rows_max + row] = dgp;
+      if (nhalf == 1) p.outf[static_cast<int64_t>(n0 / 256 * 2 + 1) * p.rows_max + row] = 0.f;
+    }
   } else if (Traits<KIND>::WGRAD && KIND != GEMM_DWR && p.acc_fp32) {
     // accumulate mode of the weight gradients: fp32 read-modify-write, old values fetched one chunk ahead
     auto dst_of = [&](int c) -> float* {
@@ -387,15 +396,15 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       return (write && col < p.N_total) ? fb + e * p.expert_stride + static_cast<int64_t>(slab) * p.ld_out + col : nullptr;
     };
     float4 gn[8];
-    float* dn = dst_of(0);
+    float* dn = dst_of(c8_lo);
     if (dn) accum_load(dn, p.ld_out, rows_valid, lane, gn);
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
+    for (int c = c8_lo; c < c8_hi; ++c) {
       float4 g[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) g[i] = gn[i];
       float* dc = dn;
-      dn = c + 1 < 8 ? dst_of(c + 1) : nullptr;
+      dn = c + 1 < c8_hi ? dst_of(c + 1) : nullptr;
       if (dn) accum_load(dn, p.ld_out, rows_valid, lane, gn);
       uint32_t rd[32];
       tmem_ld32(taddr + c * 32, rd);
@@ -408,7 +417,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
   } else {
     // plain bf16 store: F4, B4, DX (row GEMMs), B3, B5 (weight gradients)
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
+    for (int c = c8_lo; c < c8_hi; ++c) {
       uint32_t rd[32];
       tmem_ld32(taddr + c * 32, rd);
       tmem_ld_wait();
