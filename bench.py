@@ -339,23 +339,44 @@ def main():
             host[n] = torch.empty(inp["W_gate"].size if n != "dW_down" else inp["W_down"].size, dtype=torch.int16).pin_memory()
         dev_buf = torch.empty(layer.e2e_device_bytes(T), dtype=torch.uint8, device="cuda")
         layer.step_host(T, dev_buf, host, inp["d_aux"], copy_weights=True)  # uploads the weights once (untimed)
-        for _ in range(2):
-            layer.step_host(T, dev_buf, host, inp["d_aux"], copy_weights=False)
+        # timed: the pipelined host step (two slots in flight, as a training loop that prefetches its next batch
+        # would call it); every step still uploads its x, dy and downloads its y, dx, aux inside the timed region
+        slots = [dict(host, y=torch.empty(T, shape.d, dtype=torch.int16).pin_memory(),
+                      dx=torch.empty(T, shape.d, dtype=torch.int16).pin_memory(),
+                      aux=torch.empty(1, dtype=torch.float32).pin_memory()) for _ in range(2)]
+
+        def run_pipelined(n):
+            layer.step_host_begin(0, T, dev_buf, slots[0], inp["d_aux"])
+            for i in range(1, n):
+                layer.step_host_begin(i % 2, T, dev_buf, slots[i % 2], inp["d_aux"])
+                layer.step_host_end((i - 1) % 2)
+            layer.step_host_end((n - 1) % 2)
+        run_pipelined(3)
         pdist.barrier()
         torch.cuda.synchronize()
+        n_e2e = max(4, min(args.steps, 20))
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record()
+        run_pipelined(n_e2e)  # returns after the last step's results have reached the host buffers
+        p1.record()
+        torch.cuda.synchronize()
+        pdist.barrier()
+        e2e_ms = pdist.max_over_ranks(p0.elapsed_time(p1)) / n_e2e
+        layer.poll()
+        # the blocking single-call form for comparison
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        n_e2e = max(3, min(args.steps, 10))
-        for _ in range(n_e2e):
+        for _ in range(3):
             layer.step_host(T, dev_buf, host, inp["d_aux"], copy_weights=False)
         e1.record()
         torch.cuda.synchronize()
-        pdist.barrier()
-        e2e_ms = pdist.max_over_ranks(e0.elapsed_time(e1)) / n_e2e
+        blocking_ms = e0.elapsed_time(e1) / 3
         td = 2 * T * shape.d
         e2e = {"value": world * T / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": 2 * td,
-               "d2h_bytes_per_step": 2 * td + 4, "ms_per_step": e2e_ms,
-               "note": "x, dy in and y, dx, aux out every step; weights and weight gradients stay on the device"}
+               "d2h_bytes_per_step": 2 * td + 4, "ms_per_step": e2e_ms, "ms_per_step_blocking_call": blocking_ms,
+               "note": "moe_step_host_begin/end with two slots in flight: x, dy in and y, dx, aux out every step; the closing "
+                       "CUDA event is recorded after the last step's results reached the host; weights and weight "
+                       "gradients stay on the device"}
         del dev_buf
 
     if rank != 0:

@@ -217,6 +217,18 @@ MOE_API moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, cons
                          float* dW_r, uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down,
                          void* dev /* device */, size_t dev_bytes, void* cuda_stream);
 
+/* Pipelined form of moe_step_host for training loops that prefetch the next batch: moe_step_host_begin enqueues one
+ * whole step (x, dy in; forward; backward; y, aux, dx out) for slot 0 or 1 and returns without waiting;
+ * moe_step_host_end(slot) blocks until that slot's y, aux_loss and dx have arrived in the host buffers.  With both
+ * slots in flight (begin(0), begin(1), end(0), begin(0), end(1), ...) the upload of the next batch and the download
+ * of the previous results overlap the current step's kernels.  Weights must be resident (one earlier moe_step_host
+ * with copy_weights = 1); the weight gradients of the most recent step stay on the device.  Host buffers of a slot
+ * must stay untouched between its begin and end.  Device-side status is reported by moe_poll_status. */
+MOE_API moe_status moe_step_host_begin(moe_ctx* ctx, int slot, int64_t T, const uint16_t* x, const uint16_t* dy,
+                                       float d_aux, uint16_t* y, float* aux_loss, uint16_t* dx, void* dev,
+                                       size_t dev_bytes, void* cuda_stream);
+MOE_API moe_status moe_step_host_end(moe_ctx* ctx, int slot);
+
 /* Router weight gradient without any device allocation:  dW_r[d,E] = sum_t x[t,:]^T dl[t,:].
  * (The paper has no counterpart of this call; it exists for integration reasons only.)
  *

@@ -18,7 +18,8 @@ EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_fi
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
            "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout",
            "moe_forward_inference", "moe_inference_workspace_bytes", "moe_backward_accumulate",
-           "moe_lora_workspace_bytes", "moe_lora_forward", "moe_lora_backward"]
+           "moe_lora_workspace_bytes", "moe_lora_forward", "moe_lora_backward",
+           "moe_step_host_begin", "moe_step_host_end"]
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -68,6 +69,10 @@ def load_library() -> C.CDLL:
     lib.moe_backward.restype = C.c_int
     lib.moe_backward_accumulate.argtypes = lib.moe_backward.argtypes
     lib.moe_backward_accumulate.restype = C.c_int
+    lib.moe_step_host_begin.argtypes = [vp, C.c_int, i64, vp, vp, C.c_float, vp, vp, vp, vp, sz, vp]
+    lib.moe_step_host_begin.restype = C.c_int
+    lib.moe_step_host_end.argtypes = [vp, C.c_int]
+    lib.moe_step_host_end.restype = C.c_int
     lib.moe_lora_workspace_bytes.argtypes = [vp, i64]
     lib.moe_lora_workspace_bytes.restype = sz
     lib.moe_lora_forward.argtypes = [vp, i64, C.c_int32, C.c_float] + [vp] * 16 + [vp, sz, vp]
@@ -299,6 +304,16 @@ class MoELayer:
     def poll(self) -> None:
         """Synchronises and raises if a device-side bounded wait ran out."""
         _check(self.lib, self.lib.moe_poll_status(self.h, _ptr(self.ws), self._stream()), "device status")
+
+    def step_host_begin(self, slot: int, T, dev_buf, host, d_aux: float):
+        """Enqueues one pipelined host step for slot 0/1 (host: pinned x, dy in; y, aux, dx out); see step_host_end."""
+        hp = lambda n: C.c_void_p(host[n].data_ptr())
+        rc = self.lib.moe_step_host_begin(self.h, slot, T, hp("x"), hp("dy"), C.c_float(d_aux), hp("y"), hp("aux"),
+                                          hp("dx"), _ptr(dev_buf), dev_buf.numel(), self._stream())
+        _check(self.lib, rc, "moe_step_host_begin")
+
+    def step_host_end(self, slot: int):
+        _check(self.lib, self.lib.moe_step_host_end(self.h, slot), "moe_step_host_end")
 
     def selftest_timeout(self) -> None:
         """Launches the kernel whose bounded wait runs out (see moe_selftest_timeout); poll() then raises."""

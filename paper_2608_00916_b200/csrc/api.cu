@@ -137,6 +137,8 @@ void moe_destroy(moe_ctx* ctx) {
     cudaStreamDestroy(c->s_in);
     cudaStreamDestroy(c->s_out);
     for (int i = 0; i < 6; ++i) cudaEventDestroy(c->e2e_ev[i]);
+    for (int sl = 0; sl < 2; ++sl)
+      for (int i = 0; i < 5; ++i) cudaEventDestroy(c->pipe_ev[sl][i]);
   }
   delete c;
 }
@@ -547,6 +549,7 @@ moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, float scale,
 // ------------------------------------------------------------------------------------------ host-buffer step
 struct E2ELayout {
   size_t x, dy, y, dx, W_r, Wg, Wu, Wd, dWr, dWg, dWu, dWd, idx, gates, counts, aux, ws, total;
+  size_t x1, dy1, y1, dx1, aux1;  // second slot of the pipelined host steps
 };
 static E2ELayout e2e_layout(const Shape& s, int64_t T) {
   E2ELayout L;
@@ -567,8 +570,24 @@ static E2ELayout e2e_layout(const Shape& s, int64_t T) {
   L.counts = take(sizeof(int32_t) * s.E);
   L.aux = take(256);
   L.ws = take(make_layout(s, T).total);
+  L.x1 = take(td); L.dy1 = take(td); L.y1 = take(td); L.dx1 = take(td);
+  L.aux1 = take(256);
   L.total = off;
   return L;
+}
+
+static moe_status e2e_setup(moe_ctx_impl* c) {
+  if (c->e2e_created) return MOE_OK;
+  if (cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  for (int i = 0; i < 6; ++i)
+    if (cudaEventCreateWithFlags(&c->e2e_ev[i], cudaEventDisableTiming) != cudaSuccess) return MOE_ERR_CUDA;
+  for (int sl = 0; sl < 2; ++sl)
+    for (int i = 0; i < 5; ++i)
+      if (cudaEventCreateWithFlags(&c->pipe_ev[sl][i], cudaEventDisableTiming) != cudaSuccess) return MOE_ERR_CUDA;
+  c->e2e_created = 1;
+  return MOE_OK;
 }
 
 size_t moe_e2e_device_bytes(const moe_ctx* ctx, int64_t T) {
@@ -593,14 +612,7 @@ moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16
   const size_t td = sizeof(uint16_t) * T * s.d, w = sizeof(uint16_t) * s.E * s.d * s.f;
   // Copies run on two private streams so that they overlap the compute stream: dy arrives while forward runs,
   // y leaves while backward runs; only the copy of x before forward and of dx after backward are exposed.
-  if (!c->e2e_created) {
-    if (cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    for (int i = 0; i < 6; ++i)
-      if (cudaEventCreateWithFlags(&c->e2e_ev[i], cudaEventDisableTiming) != cudaSuccess) return MOE_ERR_CUDA;
-    c->e2e_created = 1;
-  }
+  if (e2e_setup(c) != MOE_OK) return MOE_ERR_CUDA;
   cudaEvent_t ev_start = c->e2e_ev[0], ev_x = c->e2e_ev[1], ev_dy = c->e2e_ev[2], ev_fwd = c->e2e_ev[3],
               ev_bwd = c->e2e_ev[4], ev_out = c->e2e_ev[5];
   bool ok = true;
@@ -652,6 +664,66 @@ moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16
   if (!ok) return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
   return moe_poll_status(ctx, D + L.ws, cuda_stream);
+}
+
+// Pipelined host steps: begin enqueues one step (copies in, forward, backward, copies out) for slot 0 or 1 and
+// returns; end waits for that slot's results.  With two slots in flight the upload of the next batch and the
+// download of the previous results overlap the current step's kernels.
+moe_status moe_step_host_begin(moe_ctx* ctx, int slot, int64_t T, const uint16_t* x, const uint16_t* dy, float d_aux,
+                               uint16_t* y, float* aux_loss, uint16_t* dx, void* dev, size_t dev_bytes,
+                               void* cuda_stream) {
+  if (!ctx || T < 0 || (slot != 0 && slot != 1) || !dev || !x || !dy || !y || !dx || !aux_loss) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  const Shape& s = c->s;
+  const E2ELayout L = e2e_layout(s, T);
+  if (dev_bytes < L.total) return MOE_ERR_WORKSPACE;
+  if (e2e_setup(c) != MOE_OK) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* D = static_cast<char*>(dev);
+  const size_t td = sizeof(uint16_t) * T * s.d;
+  const size_t ox = slot ? L.x1 : L.x, ody = slot ? L.dy1 : L.dy, oy = slot ? L.y1 : L.y, odx = slot ? L.dx1 : L.dx,
+               oaux = slot ? L.aux1 : L.aux;
+  cudaEvent_t* ev = c->pipe_ev[slot];  // 0 x in, 1 dy in, 2 forward done, 3 backward done, 4 results out
+  bool ok = true;
+  // this slot's device buffers were last read by the slot's previous backward and its previous copy-out
+  if (c->pipe_used[slot]) {
+    ok = ok && cudaStreamWaitEvent(c->s_in, ev[3], 0) == cudaSuccess && cudaStreamWaitEvent(c->s_in, ev[4], 0) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(D + ox, x, td, cudaMemcpyHostToDevice, c->s_in) == cudaSuccess &&
+       cudaEventRecord(ev[0], c->s_in) == cudaSuccess &&
+       cudaMemcpyAsync(D + ody, dy, td, cudaMemcpyHostToDevice, c->s_in) == cudaSuccess &&
+       cudaEventRecord(ev[1], c->s_in) == cudaSuccess;
+  if (!ok) return MOE_ERR_CUDA;
+  const size_t wsb = make_layout(s, T).total;
+  auto U = [&](size_t off) { return reinterpret_cast<uint16_t*>(D + off); };
+  if (cudaStreamWaitEvent(st, ev[0], 0) != cudaSuccess) return MOE_ERR_CUDA;
+  if (c->pipe_used[slot] && cudaStreamWaitEvent(st, ev[4], 0) != cudaSuccess) return MOE_ERR_CUDA;  // y, dx of this slot are free
+  moe_status rc = moe_forward(ctx, T, U(ox), U(L.W_r), nullptr, nullptr, U(L.Wg), U(L.Wu), U(L.Wd), U(oy),
+                              reinterpret_cast<int32_t*>(D + L.idx), reinterpret_cast<float*>(D + L.gates),
+                              reinterpret_cast<int32_t*>(D + L.counts), nullptr, reinterpret_cast<float*>(D + oaux),
+                              nullptr, D + L.ws, wsb, cuda_stream);
+  if (rc != MOE_OK) return rc;
+  ok = cudaEventRecord(ev[2], st) == cudaSuccess && cudaStreamWaitEvent(c->s_out, ev[2], 0) == cudaSuccess &&
+       cudaMemcpyAsync(y, D + oy, td, cudaMemcpyDeviceToHost, c->s_out) == cudaSuccess &&
+       cudaMemcpyAsync(aux_loss, D + oaux, sizeof(float), cudaMemcpyDeviceToHost, c->s_out) == cudaSuccess &&
+       cudaStreamWaitEvent(st, ev[1], 0) == cudaSuccess;
+  if (!ok) return MOE_ERR_CUDA;
+  rc = moe_backward(ctx, T, U(ody), d_aux, U(ox), U(L.W_r), U(L.Wg), U(L.Wu), U(L.Wd), U(odx),
+                    reinterpret_cast<float*>(D + L.dWr), nullptr, U(L.dWg), U(L.dWu), U(L.dWd), D + L.ws, wsb,
+                    cuda_stream);
+  if (rc != MOE_OK) return rc;
+  ok = cudaEventRecord(ev[3], st) == cudaSuccess && cudaStreamWaitEvent(c->s_out, ev[3], 0) == cudaSuccess &&
+       cudaMemcpyAsync(dx, D + odx, td, cudaMemcpyDeviceToHost, c->s_out) == cudaSuccess &&
+       cudaEventRecord(ev[4], c->s_out) == cudaSuccess;
+  c->pipe_used[slot] = 1;
+  return ok ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_step_host_end(moe_ctx* ctx, int slot) {
+  if (!ctx || (slot != 0 && slot != 1)) return MOE_ERR_INVALID_ARG;
+  moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  if (!c->e2e_created || !c->pipe_used[slot]) return MOE_ERR_INVALID_ARG;
+  return cudaEventSynchronize(c->pipe_ev[slot][4]) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 }  // extern "C"

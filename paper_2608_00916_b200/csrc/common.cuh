@@ -83,6 +83,8 @@ struct moe_ctx_impl {
   // moe_step_host: copy-in / copy-out streams and the events that order them against the compute stream
   cudaStream_t s_in, s_out;
   cudaEvent_t e2e_ev[6];
+  cudaEvent_t pipe_ev[2][5];  // pipelined host steps, per slot: x in, dy in, forward done, backward done, results out
+  int pipe_used[2];
   int e2e_created;
   int64_t prof_read;   // pairs already reported by moe_stage_times
 };

@@ -320,6 +320,31 @@ def test_step_host_matches_the_device_path():
     assert torch.equal(host["dW_r"], bw["dW_r"].cpu())
     for n in ("dW_gate", "dW_up", "dW_down"):
         assert torch.equal(host[n], bw[n].view(torch.int16).cpu()), n
+    # pipelined form: two slots in flight, six steps alternating between two different batches
+    inp2 = synth.make_inputs(shape, 89)
+    inp2["W_r"], inp2["W_gate"], inp2["W_up"], inp2["W_down"] = inp["W_r"], inp["W_gate"], inp["W_up"], inp["W_down"]
+    r2 = Run(inp2, 4)
+    fw2 = r2.forward()
+    bw2 = r2.backward(inp["d_aux"], want_db=False)
+    slots = []
+    for sl, src in ((0, inp), (1, inp2)):
+        slots.append({"x": torch.from_numpy(src["x"].view(np.int16)).pin_memory(),
+                      "dy": torch.from_numpy(src["dy"].view(np.int16)).pin_memory(),
+                      "y": torch.zeros(T, d, dtype=torch.int16).pin_memory(),
+                      "dx": torch.zeros(T, d, dtype=torch.int16).pin_memory(), "aux": torch.zeros(1).pin_memory()})
+    want = [(fw, bw), (fw2, bw2)]
+    layer.step_host_begin(0, T, dev_buf, slots[0], inp["d_aux"])
+    for i in range(1, 6):
+        layer.step_host_begin(i % 2, T, dev_buf, slots[i % 2], inp["d_aux"])
+        prev = (i - 1) % 2
+        layer.step_host_end(prev)
+        assert torch.equal(slots[prev]["y"], want[prev][0]["y"].view(torch.int16).cpu()), i
+        assert torch.equal(slots[prev]["dx"], want[prev][1]["dx"].view(torch.int16).cpu()), i
+        slots[prev]["y"].zero_()
+        slots[prev]["dx"].zero_()
+    layer.step_host_end(1)
+    assert torch.equal(slots[1]["dx"], bw2["dx"].view(torch.int16).cpu())
+    layer.poll()
 
 
 @pytest.mark.parametrize("T,d,E,k,f,rank,seed", [
