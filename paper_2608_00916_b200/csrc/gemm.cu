@@ -1,11 +1,11 @@
 // Grouped GEMMs of the MoE layer on tcgen05 tensor cores (sm_100a).
 //
 // One persistent, warp-specialised kernel template serves the six contractions of the layer:
-//   F3  [hg|hu] = xp  W_gate[e] | W_up[e]          + SwiGLU epilogue (writes hg, hu, act)
+//   F3  [hg|hu] = xp  W_gate[e] | W_up[e]          + SwiGLU epilogue (writes hg, hu and act = gate silu(hg) hu)
 //   F4  o       = act W_down[e]
-//   B2  da      = d_o W_down[e]^T                   + SwiGLU-backward epilogue (reads hg, hu; writes dhg, dhu)
+//   B2  da      = dy_rows W_down[e]^T               + SwiGLU-backward epilogue (reads hg, hu; writes dhg, dhu, dg partials)
 //   B4  dxp     = dhg W_gate[e]^T + dhu W_up[e]^T   (one accumulator, two K segments)
-//   B3  dW_down[e]          = act_e^T d_o_e         (K = rows of expert e, one CTA owns a whole output tile)
+//   B3  dW_down[e]          = act_e^T dy_rows_e     (K = rows of expert e, one CTA owns a whole output tile)
 //   B5  dW_gate[e]|dW_up[e] = xp_e^T [dhg_e|dhu_e]
 // and the three contractions of the router, whose operands are bf16 (or fp32 split exactly into two bf16 terms),
 // so that a bf16 MMA with fp32 accumulation is an fp32 contraction up to summation order:
@@ -18,9 +18,10 @@
 // row-major [K, cols] is an MN-major operand, and the UMMA instruction takes either.
 // Row buffers are expert-major with each expert's segment padded to 128 rows of zeros, so an M tile never
 // straddles two experts and the ragged K of the weight gradients needs no masking.
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer (owns the TMEM allocation), warps 2..5 epilogue.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer (owns the TMEM allocation), warps 2..9 epilogue (2..5 for the
+// routing kind).  The expert-LoRA variant runs on the same template (launch_lora_gemm at the end of this file).
 // Every mbarrier wait is bounded; on a timeout the kernel records it in the status word and leaves.
-#include <stdlib.h>
+#include <stdlib.h>  // getenv (MOE_GEMM_TIMERS)
 
 #include "gemm_common.cuh"
 

@@ -1,5 +1,7 @@
 // Router (fp32 logits, softmax, top-k with lowest-index tie-break, renormalised gates) and the
-// deterministic token permutation (per-tile histogram, prefix scan, stable scatter, row gather).
+// deterministic token permutation (per-tile histogram, prefix scan, stable scatter, row copy).  The router kernel here
+// is the SIMT path (expert counts that are not a multiple of 8, or caller-supplied logits); otherwise the logits are
+// contracted on the tensor cores (gemm.cu, kind RT).
 #include "common.cuh"
 
 namespace moe {
