@@ -295,10 +295,16 @@ def main():
                "dW_up": torch.zeros(shape.E, shape.d, shape.f, device="cuda"),
                "dW_down": torch.zeros(shape.E, shape.f, shape.d, device="cuda")}
 
+    reducer = pdist.GradAllReducer() if (acc is not None and world > 1) else None
+
     def step():
         layer.forward(tens["x"], tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], b_r=b_r, want_perm=False)
         if acc is not None:
+            if reducer is not None:
+                reducer.wait()  # the previous step's gradient all-reduce (it overlapped this step's forward)
             layer.backward_accumulate(tens["dy"], inp["d_aux"], acc)
+            if reducer is not None:
+                reducer.start([acc["dW_gate"], acc["dW_up"], acc["dW_down"], acc["dW_r"]])
         else:
             layer.backward(tens["dy"], inp["d_aux"], grads=grads)
 

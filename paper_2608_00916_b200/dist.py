@@ -68,6 +68,72 @@ def job_throughput(tokens_this_rank: int, ms_this_rank: float) -> float:
     return total / (ms / 1e3)
 
 
+class GradAllReducer:
+    """Sums the weight-gradient buffers of the data-parallel ranks (the one exchange step of the sharded layer: tokens
+    are split over the ranks, experts are replicated, so dW_gate / dW_up / dW_down / dW_r must be added up).
+
+    The buffers (fp32, as filled by MoELayer.backward_accumulate) are cut along the expert axis into buckets; each
+    bucket is all-reduced asynchronously on the process group (NCCL over NVLink on GPUs, gloo on CPU).  start() may be
+    called as soon as the kernels that write the buffers have been enqueued: on CUDA it makes a side stream wait for an
+    event recorded on the compute stream, so the reduction overlaps whatever the compute stream runs next (the router
+    gradient and the unpermute); wait() joins before the optimizer reads the buffers.  With one rank both are no-ops."""
+
+    def __init__(self, experts_per_bucket: int = 16):
+        self.experts_per_bucket = max(1, int(experts_per_bucket))
+        self._work = []
+        self._side = None
+        self._done = None
+
+    def buckets(self, tensors):
+        """(tensor, first expert, last expert + 1) slices in launch order; tensors without an expert axis (dW_r) last."""
+        out = []
+        for t in tensors:
+            if t.dim() == 3:
+                for e0 in range(0, t.shape[0], self.experts_per_bucket):
+                    out.append((t, e0, min(t.shape[0], e0 + self.experts_per_bucket)))
+        for t in tensors:
+            if t.dim() != 3:
+                out.append((t, 0, t.shape[0]))
+        return out
+
+    def start(self, tensors) -> None:
+        if _state["world"] <= 1:
+            return
+        import torch
+        import torch.distributed as dist
+        on_cuda = tensors[0].is_cuda
+        if on_cuda:
+            if self._side is None:
+                self._side = torch.cuda.Stream()
+            ev = torch.cuda.Event()
+            ev.record(torch.cuda.current_stream())
+            self._side.wait_event(ev)
+        ctx = torch.cuda.stream(self._side) if on_cuda else _NullCtx()
+        with ctx:
+            for t, e0, e1 in self.buckets(tensors):
+                self._work.append(dist.all_reduce(t[e0:e1], op=dist.ReduceOp.SUM, async_op=True))
+            if on_cuda:
+                self._done = torch.cuda.Event()
+                self._done.record(self._side)
+
+    def wait(self) -> None:
+        import torch
+        for w in self._work:
+            w.wait()
+        self._work = []
+        if self._done is not None:
+            torch.cuda.current_stream().wait_event(self._done)
+            self._done = None
+
+
+class _NullCtx:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        return False
+
+
 def finish() -> None:
     if _state["world"] > 1:
         import torch.distributed as dist

@@ -47,6 +47,50 @@ def test_two_gloo_ranks():
     assert x0 != x1 and y0 != y1                      # different token batches per rank
 
 
+def _reduce_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    import torch
+    from oracle import moe_oracle as orc
+    from paper_2608_00916_b200 import dist as pdist
+    from paper_2608_00916_b200 import synth
+    pdist.init(world, rank, backend="gloo")
+    shape = synth.MoEShape(48, 64, 6, 2, 64)
+    base = synth.make_inputs(shape, 700, threads=1)
+    mine = synth.make_inputs(shape, pdist.shard_seed(700, rank), threads=1)
+    fw = orc.forward(mine["x"], base["W_r"], base["W_gate"], base["W_up"], base["W_down"], 2)
+    bw = orc.backward(fw, mine["dy"], 0.0, mine["x"], base["W_r"], base["W_gate"], base["W_up"], base["W_down"])
+    acc = [torch.from_numpy(bw[n].astype(np.float32)).clone() for n in ("dW_gate", "dW_up", "dW_down", "dW_r")]
+    local = [a.clone() for a in acc]
+    red = pdist.GradAllReducer(experts_per_bucket=4)
+    assert [(e0, e1) for t, e0, e1 in red.buckets(acc) if t.dim() == 3][:2] == [(0, 4), (4, 6)]
+    red.start(acc)
+    red.wait()
+    q.put((rank, [a.numpy() for a in acc], [a.numpy() for a in local]))
+    pdist.finish()
+
+
+def test_gradient_all_reduce_over_two_gloo_ranks():
+    """Data-parallel ranks hold different token batches and replicated experts; after GradAllReducer every rank holds
+    the sum of both ranks' weight gradients (bucketed along the expert axis, asynchronous)."""
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29850 + os.getpid() % 100
+    procs = [ctx.Process(target=_reduce_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted((q.get(timeout=120) for _ in procs), key=lambda x: x[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (_, red0, loc0), (_, red1, loc1) = res
+    for a0, a1, l0, l1 in zip(red0, red1, loc0, loc1):
+        np.testing.assert_allclose(a0, l0 + l1, rtol=1e-6, atol=1e-7)
+        np.testing.assert_array_equal(a0, a1)
+        assert np.abs(l0 - l1).max() > 0
+
+
 def test_token_split_is_balanced():
     from paper_2608_00916_b200 import dist as pdist
     for total, world in ((16384, 8), (8191, 4), (5, 8)):
