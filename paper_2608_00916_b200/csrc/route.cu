@@ -255,20 +255,62 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
   const int G = SCAN_THREADS / E;
   if (tid < G * E) {
     const int g = tid / E, e = tid - g * E;
-    // eight loads in flight per thread; the partial sums are combined in a fixed order
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    int b = g;
-    for (; b + 7 * G < psum_rows; b += 8 * G) {
+    // sixteen loads in flight per thread; the partial sums are combined in a fixed order
+    float acc[16];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) acc[u] += psum_part[static_cast<int64_t>(b + u * G) * E + e];
+    for (int u = 0; u < 16; ++u) acc[u] = 0.f;
+    int b = g;
+    for (; b + 15 * G < psum_rows; b += 16 * G) {
+#pragma unroll
+      for (int u = 0; u < 16; ++u) acc[u] += psum_part[static_cast<int64_t>(b + u * G) * E + e];
     }
     for (; b < psum_rows; b += G) acc[0] += psum_part[static_cast<int64_t>(b) * E + e];
-    s_ps[tid] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+#pragma unroll
+    for (int st = 8; st >= 1; st >>= 1)
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (u < st) acc[u] += acc[u + st];
+    s_ps[tid] = acc[0];
   }
   __syncthreads();
   // exclusive prefix of every expert's column of tile_counts along the tiles: one warp per expert, 32 tiles per step
   {
     const int lane = tid & 31, wid = tid >> 5;
+    constexpr int NW = SCAN_THREADS / 32;
+    if (tok_tiles <= 64 && E <= 8 * NW) {
+      // common case: every expert column of this warp (at most 8) is loaded before the first scan, so the whole phase
+      // costs one memory round trip
+      int c[8][2];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int e = wid + i * NW;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int tl = 32 * u + lane;
+          c[i][u] = (e < E && tl < tok_tiles) ? tile_counts[static_cast<int64_t>(tl) * E + e] : 0;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int e = wid + i * NW;
+        if (e < E) {
+          int run = 0;
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int tl = 32 * u + lane;
+            int inc = c[i][u];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+              const int v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+              if (lane >= off) inc += v;
+            }
+            if (tl < tok_tiles) tile_counts[static_cast<int64_t>(tl) * E + e] = run + inc - c[i][u];
+            run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+          }
+          if (lane == 0) s_cnt[e] = run;
+        }
+      }
+    } else
     for (int e = wid; e < E; e += SCAN_THREADS / 32) {
       int run = 0;
       for (int tb = 0; tb < tok_tiles; tb += 256) {  // up to 8 steps of 32 tiles with all their loads in flight
