@@ -200,10 +200,9 @@ class MoELayer:
         if logits_in is not None:
             assert logits_in.dtype == torch.float32 and tuple(logits_in.shape) == (T, E) and logits_in.is_contiguous()
         fn = self.lib.moe_forward_inference if inference else self.lib.moe_forward
-        rc = fn(self.h, T, _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(logits_in), _ptr(W_gate), _ptr(W_up),
-                                  _ptr(W_down), _ptr(out["y"]), _ptr(out["idx"]), _ptr(out["gates"]),
-                                  _ptr(out["counts"]), _ptr(out["perm"]), _ptr(out["aux"]), _ptr(out["logits"]),
-                                  _ptr(self.ws), self.ws.numel(), self._stream())
+        rc = fn(self.h, T, _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(logits_in), _ptr(W_gate), _ptr(W_up), _ptr(W_down),
+                _ptr(out["y"]), _ptr(out["idx"]), _ptr(out["gates"]), _ptr(out["counts"]), _ptr(out["perm"]),
+                _ptr(out["aux"]), _ptr(out["logits"]), _ptr(self.ws), self.ws.numel(), self._stream())
         _check(self.lib, rc, "moe_forward")
         self._saved = None if inference else (x, W_r, W_gate, W_up, W_down)
         return out
@@ -219,14 +218,14 @@ class MoELayer:
         assert dy.dtype == torch.bfloat16 and tuple(dy.shape) == (T, d) and dy.is_contiguous()
         dev = x.device
         g = grads or {}
-        out = {
-            "dx": g.get("dx", None) if g.get("dx", None) is not None else torch.empty(T, d, dtype=torch.bfloat16, device=dev),
-            "dW_r": g.get("dW_r") if g.get("dW_r") is not None else torch.empty(d, E, dtype=torch.float32, device=dev),
-            "db_r": torch.empty(E, dtype=torch.float32, device=dev) if want_db else None,
-            "dW_gate": g.get("dW_gate") if g.get("dW_gate") is not None else torch.empty(E, d, f, dtype=torch.bfloat16, device=dev),
-            "dW_up": g.get("dW_up") if g.get("dW_up") is not None else torch.empty(E, d, f, dtype=torch.bfloat16, device=dev),
-            "dW_down": g.get("dW_down") if g.get("dW_down") is not None else torch.empty(E, f, d, dtype=torch.bfloat16, device=dev),
-        }
+
+        def buf(name, shape, dtype):
+            return g[name] if g.get(name) is not None else torch.empty(*shape, dtype=dtype, device=dev)
+
+        out = {"dx": buf("dx", (T, d), torch.bfloat16), "dW_r": buf("dW_r", (d, E), torch.float32),
+               "db_r": torch.empty(E, dtype=torch.float32, device=dev) if want_db else None,
+               "dW_gate": buf("dW_gate", (E, d, f), torch.bfloat16), "dW_up": buf("dW_up", (E, d, f), torch.bfloat16),
+               "dW_down": buf("dW_down", (E, f, d), torch.bfloat16)}
         rc = self.lib.moe_backward(self.h, T, _ptr(dy), C.c_float(d_aux), _ptr(x), _ptr(W_r), _ptr(W_gate), _ptr(W_up),
                                    _ptr(W_down), _ptr(out["dx"]), _ptr(out["dW_r"]), _ptr(out["db_r"]),
                                    _ptr(out["dW_gate"]), _ptr(out["dW_up"]), _ptr(out["dW_down"]), _ptr(self.ws),
