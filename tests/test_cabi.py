@@ -81,3 +81,38 @@ def test_forward_rejects_bad_arguments_before_launch(lib):
     # missing weights
     args = [layer.h, 64, fake, fake, None, None, None, fake, fake] + [fake] * 7 + [fake, 1 << 30, None]
     assert lib.moe_forward(*args) == -1
+
+
+def test_other_entry_points_reject_bad_arguments_before_launch(lib):
+    """Argument errors of backward, the LoRA variant, the host-step calls and the static-scratch entry are reported as
+    codes without touching a device (the pointers are fakes that are never dereferenced)."""
+    layer = binding.MoELayer(128, 8, 128, 2)
+    vp = C.c_void_p
+    fake = vp(4096)
+    big = 1 << 40
+    # backward: T < 0, missing dW buffers, small workspace
+    assert lib.moe_backward(layer.h, -1, fake, C.c_float(0), *([fake] * 11), fake, big, None) == -1
+    assert lib.moe_backward(layer.h, 8, fake, C.c_float(0), fake, fake, fake, fake, fake, fake, fake, None, None, fake,
+                            fake, fake, big, None) == -1
+    assert lib.moe_backward(layer.h, 8, fake, C.c_float(0), *([fake] * 11), fake, 64, None) == -3
+    assert lib.moe_backward_accumulate(layer.h, 8, fake, C.c_float(0), fake, fake, fake, fake, fake, fake, fake, None,
+                                       None, fake, fake, fake, big, None) == -1
+    # LoRA: rank must be a multiple of 8 in [8, 64]; adapters must be present
+    for bad_rank in (0, 4, 12, 72):
+        assert lib.moe_lora_forward(layer.h, 8, bad_rank, C.c_float(1), *([fake] * 16), fake, big, None) == -1
+    args = [fake] * 16
+    args[6] = None  # A1 missing
+    assert lib.moe_lora_forward(layer.h, 8, 16, C.c_float(1), *args, fake, big, None) == -1
+    assert lib.moe_lora_forward(layer.h, 8, 16, C.c_float(1), *([fake] * 16), fake, 64, None) == -3
+    assert layer.lib.moe_lora_workspace_bytes(layer.h, 64) > layer.workspace_bytes(64) > layer.inference_workspace_bytes(64)
+    # host steps: bad slot, missing buffers, small device buffer
+    assert lib.moe_step_host_begin(layer.h, 2, 8, fake, fake, C.c_float(0), fake, fake, fake, fake, big, None) == -1
+    assert lib.moe_step_host_begin(layer.h, 0, 8, None, fake, C.c_float(0), fake, fake, fake, fake, big, None) == -1
+    assert lib.moe_step_host_begin(layer.h, 0, 8, fake, fake, C.c_float(0), fake, fake, fake, fake, 64, None) == -3
+    assert lib.moe_step_host_end(layer.h, 0) == -1  # nothing was begun
+    assert lib.moe_step_host(layer.h, 8, 0, None, *([fake] * 5), C.c_float(0), *([fake] * 7), fake, big, None) == -1
+    # static-scratch entry: shape limits
+    assert lib.moe_router_wgrad_static(8, 100, 8, fake, fake, fake, None) == -1      # d not a multiple of 64
+    assert lib.moe_router_wgrad_static(8, 128, 300, fake, fake, fake, None) == -1    # E > 256
+    assert lib.moe_router_wgrad_static(8, 4096, 128, fake, fake, fake, None) == -2   # beyond the built-in scratch
+    assert lib.moe_selftest_timeout(None, fake, None) == -1
