@@ -326,6 +326,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.sched = reinterpret_cast<const int32_t*>(ws + L.sched);
   p.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
   p.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+  p.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
   p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
   p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
   p.timers = getenv("MOE_GEMM_TIMERS") ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
@@ -624,6 +625,7 @@ moe_status launch_lora_gemm(moe_ctx_impl* ctx, LoraOp op, int64_t T, const WsLay
   p.sched = reinterpret_cast<const int32_t*>(ws + L.sched);
   p.tile_expert = reinterpret_cast<const int32_t*>(ws + L.tile_expert);
   p.pad_offsets = reinterpret_cast<const int32_t*>(ws + L.pad_offsets);
+  p.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
   p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
   p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
   p.status = reinterpret_cast<int32_t*>(ws + L.status);

@@ -47,7 +47,7 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
     tl.m0 = (rem / p.n_tiles) * 2 * BM + rank * BM;
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
     tl.row0 = p.pad_offsets[tl.e];
-    tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
+    tl.nkb = (p.counts[tl.e] + BK - 1) / BK;  // the rest of the 128-row padding is zeros
     tl.write = true;
   } else {
     const int pr = t / p.n_tiles;

@@ -29,6 +29,7 @@ struct GemmParams {
   const int32_t* sched;        // [0] number of 128-row tiles
   const int32_t* tile_expert;  // expert of each 128-row tile
   const int32_t* pad_offsets;  // padded segment starts, E + 1 entries
+  const int32_t* counts;       // rows per expert (weight gradients stop their K loop at the last 64-row block with data)
   const int32_t* expert_order; // weight gradients: experts by row count, largest first
   const int32_t* pair_tab;     // CTA-pair kernels: per pair of row blocks {expert, first row, blocks (1|2), 0}
   int32_t* status;
@@ -119,7 +120,7 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
       tl.nkb = max(0, min(p.split_rows, p.rows_total - tl.row0)) / BK;
     } else {
       tl.row0 = p.pad_offsets[tl.e];
-      tl.nkb = (p.pad_offsets[tl.e + 1] - tl.row0) / BK;
+      tl.nkb = (p.counts[tl.e] + BK - 1) / BK;  // the rest of the 128-row padding is zeros
     }
   } else if (Traits<KIND>::STATIC_M) {
     const int mt = t / p.n_tiles;
