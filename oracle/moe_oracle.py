@@ -253,6 +253,37 @@ def token_rows(t: int, fw_route: dict, x_bits, Wg_bits, Wu_bits, Wd_bits, dtype=
     return y
 
 
+def token_backward(t: int, fw_route: dict, dy_bits, d_aux: float, x_bits, Wr_bits, Wg_bits, Wu_bits, Wd_bits,
+                   dtype=np.float64):
+    """dx[t,:] and dl[t,:] alone, from the routing of ``fw_route`` (used where the full layer is too large to run):
+    the chain rule through the k experts of token t, its gates, and the auxiliary loss (whose counts come from the
+    routing of all tokens)."""
+    k = fw_route["idx"].shape[1]
+    T, E = fw_route["p"].shape
+    x = widen_bf16(x_bits[t:t + 1], dtype)
+    dy = widen_bf16(dy_bits[t], dtype)
+    g = fw_route["gates"][t]
+    dg = np.zeros(k, dtype=dtype)
+    dx = np.zeros(x.shape[1], dtype=dtype)
+    for j in range(k):
+        e = int(fw_route["idx"][t, j])
+        Wg, Wu, Wd = widen_bf16(Wg_bits[e], dtype), widen_bf16(Wu_bits[e], dtype), widen_bf16(Wd_bits[e], dtype)
+        hg, hu, a, o = expert_ffn(x, Wg, Wu, Wd)
+        dg[j] = float(dy @ o[0])
+        da = (g[j] * dy) @ Wd.T
+        sig = 1.0 / (1.0 + np.exp(-hg[0]))
+        dhg = da * hu[0] * sig * (1.0 + hg[0] * (1.0 - sig))
+        dhu = da * hg[0] * sig
+        dx += dhg @ Wg.T + dhu @ Wu.T
+    p = fw_route["p"][t]
+    dl = np.zeros(E, dtype=dtype)
+    dl[fw_route["idx"][t].astype(np.int64)] = g * (dg - float((g * dg).sum()))
+    dp = d_aux * E * (fw_route["counts"].astype(dtype) / (T * k)) / T
+    dl += p * (dp - float((p * dp).sum()))
+    dx += dl @ widen_bf16(Wr_bits, dtype).T
+    return dx, dl
+
+
 def route_only(x_bits, Wr_bits, k: int, E: int, b_r=None, logits_in=None, dtype=np.float64) -> dict:
     """Routing part of ``forward`` alone (logits, p, idx, gates, counts, offsets, perm, inv, aux)."""
     if logits_in is not None:

@@ -484,6 +484,13 @@ def sampled_parity(name, n_tokens=48):
     ref_dwr = synth.bf16_bits_to_f64(inp["x"]).T @ dl
     assert rel_fro(bw["dW_r"].cpu().numpy(), ref_dwr) <= 1e-3
     assert torch.isfinite(bw["dx"].float()).all()
+    # dx and dl rows of sampled tokens against the oracle's per-token backward
+    btoks = toks[: max(4, n_tokens // 4)]
+    ref_dx, ref_dl = zip(*(orc.token_backward(int(t), rt, inp["dy"], inp["d_aux"], inp["x"], inp["W_r"], inp["W_gate"],
+                                              inp["W_up"], inp["W_down"]) for t in btoks))
+    got_dx = from_dev_bf16(bw["dx"][torch.from_numpy(btoks).cuda()])
+    assert rel_fro(got_dx, np.stack(ref_dx)) <= TOL
+    assert rel_fro(dl[btoks], np.stack(ref_dl)) <= TOL
 
 
 def test_full_qwen_config_sampled():

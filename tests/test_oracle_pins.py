@@ -306,6 +306,11 @@ def test_sampled_helpers_agree_with_full_pass():
     for t in (0, 7, 17):
         np.testing.assert_allclose(orc.token_rows(t, rt, inp["x"], inp["W_gate"], inp["W_up"], inp["W_down"]),
                                    fw["y"][t], rtol=1e-12, atol=1e-15)
+    for t in (0, 7, 17):
+        dx_t, dl_t = orc.token_backward(t, rt, inp["dy"], 0.1, inp["x"], inp["W_r"], inp["W_gate"], inp["W_up"],
+                                        inp["W_down"])
+        np.testing.assert_allclose(dx_t, bw["dx"][t], rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(dl_t, bw["dl"][t], rtol=1e-10, atol=1e-14)
     for e in range(5):
         a, b_, c = orc.expert_grads(e, rt, inp["dy"], inp["x"], inp["W_gate"], inp["W_up"], inp["W_down"])
         np.testing.assert_allclose(a, bw["dW_gate"][e], rtol=1e-11, atol=1e-14)
