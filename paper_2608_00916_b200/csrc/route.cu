@@ -273,70 +273,22 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
     s_ps[tid] = acc[0];
   }
   __syncthreads();
-  // exclusive prefix of every expert's column of tile_counts along the tiles: one warp per expert, 32 tiles per step
-  {
-    const int lane = tid & 31, wid = tid >> 5;
-    constexpr int NW = SCAN_THREADS / 32;
-    if (tok_tiles <= 64 && E <= 8 * NW) {
-      // common case: every expert column of this warp (at most 8) is loaded before the first scan, so the whole phase
-      // costs one memory round trip
-      int c[8][2];
+  // exclusive prefix of every expert's column of tile_counts along the tiles.  One thread per expert, so that the
+  // lanes of a warp touch consecutive addresses (a warp per column with a lane per tile costs one memory wavefront per
+  // lane - 16 k cycles of this one-block kernel went there); 32 loads are in flight before the first dependent store.
+  for (int e = tid; e < E; e += SCAN_THREADS) {
+    int run = 0;
+    for (int t0 = 0; t0 < tok_tiles; t0 += 32) {
+      int c[32];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int e = wid + i * NW;
+      for (int u = 0; u < 32; ++u) c[u] = (t0 + u < tok_tiles) ? tile_counts[static_cast<int64_t>(t0 + u) * E + e] : 0;
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int tl = 32 * u + lane;
-          c[i][u] = (e < E && tl < tok_tiles) ? tile_counts[static_cast<int64_t>(tl) * E + e] : 0;
-        }
+      for (int u = 0; u < 32; ++u) {
+        if (t0 + u < tok_tiles) tile_counts[static_cast<int64_t>(t0 + u) * E + e] = run;
+        run += c[u];
       }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int e = wid + i * NW;
-        if (e < E) {
-          int run = 0;
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int tl = 32 * u + lane;
-            int inc = c[i][u];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-              const int v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
-              if (lane >= off) inc += v;
-            }
-            if (tl < tok_tiles) tile_counts[static_cast<int64_t>(tl) * E + e] = run + inc - c[i][u];
-            run += __shfl_sync(0xFFFFFFFFu, inc, 31);
-          }
-          if (lane == 0) s_cnt[e] = run;
-        }
-      }
-    } else
-    for (int e = wid; e < E; e += SCAN_THREADS / 32) {
-      int run = 0;
-      for (int tb = 0; tb < tok_tiles; tb += 256) {  // up to 8 steps of 32 tiles with all their loads in flight
-        int c[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int tl = tb + 32 * u + lane;
-          c[u] = tl < tok_tiles ? tile_counts[static_cast<int64_t>(tl) * E + e] : 0;
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int tl = tb + 32 * u + lane;
-          if (tb + 32 * u < tok_tiles) {
-            int inc = c[u];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-              const int v = __shfl_up_sync(0xFFFFFFFFu, inc, off);
-              if (lane >= off) inc += v;
-            }
-            if (tl < tok_tiles) tile_counts[static_cast<int64_t>(tl) * E + e] = run + inc - c[u];
-            run += __shfl_sync(0xFFFFFFFFu, inc, 31);
-          }
-        }
-      }
-      if (lane == 0) s_cnt[e] = run;
     }
+    s_cnt[e] = run;
   }
   __syncthreads();
   for (int e = tid; e < E; e += SCAN_THREADS) {
