@@ -426,12 +426,15 @@ def main():
                "sample": f"first {sample_T} tokens of the batch through the fp32 numpy oracle, forward + backward, "
                          f"all {shape.E} experts' weights"}
 
+    w_gb = 3 * shape.E * shape.d * shape.f * 2 / 1e9
+    l2_note = (f"inputs larger than L2 ({w_gb:.2f} GB of expert weights streamed per pass); no explicit flush"
+               if w_gb > 0.2 else f"working set ({w_gb * 1e3:.0f} MB of weights) fits in L2: L2-warm, launch-bound numbers")
     line = {"metric": "moe_layer_fwd_bwd_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "mode": args.mode, "T_per_gpu": T, "d": shape.d, "E": shape.E, "top_k": shape.k,
                        "f": shape.f, "parallelism": f"dp{world} over tokens, experts replicated (EP=1), no collective",
-                       "l2": "inputs larger than L2 (1.2 GB of expert weights streamed per pass); no explicit flush",
+                       "l2": l2_note,
                        "redrawn_tokens": inp["meta"]["redrawn"]},
             "grouped_gemm_tflops": gemm_tflops,
             "grouped_gemm_frac_of_sustained_bf16": gemm_tflops / peaks["bf16_tflops_sustained"],
