@@ -27,8 +27,6 @@ import numpy as np  # noqa: E402
 from paper_2608_00916_b200 import synth  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-LAUNCHES_PER_STEP = 18  # router, hist, scan, scatter, row scatter, 2 GEMMs, combine; row scatter (dy), 4 GEMMs,
-#                         router-bwd, dW_r GEMM + reduce, dx-router GEMM + unpermute-sum (profiles/launch_list_qwen.md)
 # dram bytes per launch of the dominant kernel taken from the committed ncu capture (profiles/), by stage name;
 # None where no capture has been taken for the workload.
 NCU_TRAFFIC = {  # profiles/grouped_gemms_qwen_dram_traffic.md
@@ -42,8 +40,11 @@ def load_peaks():
     if os.path.exists(p):
         with open(p) as fh:
             d = json.load(fh)
-        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
-    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+        out = {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+        out["sm_max_mhz"] = float(d.get("sm_max_mhz", 1965.0))
+        out["sustained_sm_mhz"] = float(d.get("clocks_under_load", {}).get("sm_mhz_median", 1297.0))
+        return out
+    return dict(FALLBACK_PEAKS) | {"source": "fallback", "sm_max_mhz": 1965.0, "sustained_sm_mhz": 1300.0}
 
 
 def stage_work(shape: synth.MoEShape):
@@ -68,55 +69,122 @@ def stage_work(shape: synth.MoEShape):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples the SM clock and the throttle reasons of one GPU every few milliseconds (NVML through pynvml; falls back
+    to `nvidia-smi -lms 20`), each sample stamped with the host clock, so that summary(t0, t1) can keep only the samples
+    that fall inside the timed region.  Read-only: no GPU setting is touched."""
 
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, period_s: float = 0.004):
         self.idx = gpu_index
+        self.period = period_s
+        self.samples = []  # (host time, sm MHz, max MHz, set of reasons)
         self.proc = None
-        self.lines = []
+        self.th = None
+        self.stop_flag = False
+        self.source = None
 
     def start(self):
         try:
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.idx
+            if vis:
+                ent = vis.split(",")[self.idx].strip()
+                phys = int(ent) if ent.isdigit() else self.idx
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            mx = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            bits = {"hw_slowdown": pynvml.nvmlClocksEventReasonHwSlowdown if hasattr(pynvml, "nvmlClocksEventReasonHwSlowdown") else 0x8,
+                    "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+
+            def loop():
+                while not self.stop_flag:
+                    try:
+                        mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                        try:
+                            mask = int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                        except Exception:
+                            mask = int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                        self.samples.append((time.perf_counter(), mhz, mx, {n for n, b in bits.items() if mask & b}))
+                    except Exception:
+                        pass
+                    time.sleep(self.period)
+            self.th = threading.Thread(target=loop, daemon=True)
+            self.th.start()
+            self.source = "nvml"
+            return
+        except Exception:
+            pass
+        try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
+            self.source = "nvidia-smi"
         except Exception:
             self.proc = None
 
     def _read(self):
         for ln in self.proc.stdout:
-            self.lines.append(ln.strip())
-
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.25)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        for ln in self.lines:
             p = [x.strip() for x in ln.split(",")]
             if len(p) < 9:
                 continue
             try:
-                sm.append(float(p[1]))
-                mx.append(float(p[2]))
+                sm, mx = float(p[1]), float(p[2])
             except ValueError:
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+            rs = {n for n, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9])
+                  if v.lower().startswith("active")}
+            self.samples.append((time.perf_counter(), sm, mx, rs))
+
+    def stop(self):
+        self.stop_flag = True
+        if self.proc is not None:
+            time.sleep(0.05)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+        elif self.th is not None:
+            self.th.join(timeout=1)
+
+    def summary(self, t0: float, t1: float):
+        """Median SM clock and the union of throttle reasons over the samples taken in [t0, t1] (host clock)."""
+        if self.source is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["clock sampling unavailable"], "samples": 0}
+        inside = [x for x in self.samples if t0 <= x[0] <= t1]
+        note = None
+        if not inside and self.samples:  # region shorter than one sampling period: nearest sample
+            mid = 0.5 * (t0 + t1)
+            inside = [min(self.samples, key=lambda x: abs(x[0] - mid))]
+            note = "region shorter than the sampling period: nearest sample"
+        reasons = set()
+        for x in inside:
+            reasons |= x[3]
+        out = {"sm_mhz": float(np.median([x[1] for x in inside])) if inside else None,
+               "sm_max_mhz": max(x[2] for x in inside) if inside else None, "reasons": sorted(reasons),
+               "samples": len(inside), "source": self.source}
+        if note:
+            out["note"] = note
+        return out
+
+
+def choose_peak(peaks: dict, sm_mhz, sm_max_mhz):
+    """Which measured bf16 peak describes the regime the timed region ran in.  The sustained figure was measured with
+    the SM clock settled under the power cap (about 1300 MHz on this part), the burst figure near the maximum clock;
+    the timed region's own median clock decides, halfway between the two being the dividing line."""
+    sustained_mhz = float(peaks.get("sustained_sm_mhz", 1297.0))
+    top = float(sm_max_mhz or peaks.get("sm_max_mhz", 1965.0))
+    if sm_mhz is None:
+        return "sustained", peaks["bf16_tflops_sustained"]
+    if sm_mhz >= 0.5 * (sustained_mhz + top):
+        return "burst", peaks["bf16_tflops"]
+    return "sustained", peaks["bf16_tflops_sustained"]
 
 
 def oracle_sample_tokens_per_s(inp, shape, sample_T, repeats=1):
@@ -175,11 +243,21 @@ def main():
                     help="train: forward + backward (the headline metric); inference: forward-only entry point; "
                          "accumulate: forward + backward that adds weight gradients into fp32 buffers; "
                          "lora: forward + backward of the expert-LoRA variant (rank 16, frozen expert weights)")
+    ap.add_argument("--condition-seconds", type=float, default=2.0,
+                    help="untimed back-to-back steps before the timed region, so that the timed steps run in the "
+                         "power-capped steady state the sustained peak describes (0 disables)")
+    ap.add_argument("--micro-batches", type=int, default=4,
+                    help="accumulate mode: steps per accumulation window (gradients are summed over the ranks and the "
+                         "buffers zeroed once per window)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    from paper_2608_00916_b200 import dist as pdist
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # started by hand as `python bench.py --gpus N`: become the launcher of N ranks (one process per GPU)
+        raise SystemExit(pdist.launch_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -193,19 +271,22 @@ def main():
         return
 
     import torch
-    from paper_2608_00916_b200 import dist as pdist
-    from paper_2608_00916_b200.binding import MoELayer, STAGE_NAMES
+    from paper_2608_00916_b200.binding import MoELayer, STAGE_NAMES, kernel_launches
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the CUDA path has no CPU fallback)")
+    if world > torch.cuda.device_count():
+        raise SystemExit(f"bench.py: {world} ranks but only {torch.cuda.device_count()} visible GPUs")
     torch.cuda.set_device(local_rank)
     pdist.init(world, rank, backend="nccl")
 
-    # every rank draws its own token batch (data parallel over tokens, weights replicated: same seed for weights)
+    # every rank draws its own token batch (data parallel over tokens, weights replicated: same seed for weights);
+    # the batch of rank r > 0 is guarded against the SHARED router weight and bias
     inp = synth.make_inputs(shape, seed, x_std=x_std, skew=skew)
-    if world > 1:
-        shard = synth.make_inputs(shape, pdist.shard_seed(seed, rank), x_std=x_std, skew=False, guard=True)
+    if rank > 0:
+        shard = synth.make_tokens(shape, pdist.shard_seed(seed, rank), inp["W_r"], inp["b_r"], x_std=x_std)
         inp["x"], inp["dy"] = shard["x"], shard["dy"]
+        inp["meta"]["redrawn"] = shard["redrawn"]
 
     def dev(bits):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -235,6 +316,7 @@ def main():
         torch.cuda.synchronize()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record()
+        launches0 = kernel_launches()
         for _ in range(args.steps):
             lstep()
         f1.record()
@@ -253,7 +335,7 @@ def main():
                                          "d": shape.d, "E": shape.E, "top_k": shape.k, "f": shape.f},
                               "base_gemm_useful_tflops_over_whole_step": fl / (ms * 1e-3) / 1e12,
                               "stages_ms": {STAGE_NAMES[i]: stage_ms[i] / max(n, 1) for i in range(len(STAGE_NAMES))},
-                              "gpu_launches": 29 * args.steps}))
+                              "gpu_launches": kernel_launches() - launches0}))
         pdist.finish()
         return
 
@@ -269,6 +351,7 @@ def main():
         torch.cuda.synchronize()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record()
+        launches0 = kernel_launches()
         for _ in range(args.steps):
             fstep()
         f1.record()
@@ -284,7 +367,7 @@ def main():
                                                               "T_per_gpu": T, "d": shape.d, "E": shape.E,
                                                               "top_k": shape.k, "f": shape.f},
                               "grouped_gemm_useful_tflops_over_whole_pass": fl / (ms * 1e-3) / 1e12,
-                              "gpu_launches": 9 * args.steps}))
+                              "gpu_launches": kernel_launches() - launches0}))
         pdist.finish()
         return
 
@@ -296,14 +379,23 @@ def main():
                "dW_down": torch.zeros(shape.E, shape.f, shape.d, device="cuda")}
 
     reducer = pdist.GradAllReducer() if (acc is not None and world > 1) else None
+    window = max(1, args.micro_batches)
+    step_no = [0]
 
     def step():
         layer.forward(tens["x"], tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], b_r=b_r, want_perm=False)
         if acc is not None:
-            if reducer is not None:
-                reducer.wait()  # the previous step's gradient all-reduce (it overlapped this step's forward)
+            # an accumulation window of `window` micro-batches: the buffers start at zero, every step adds its weight
+            # gradients, the last step of the window is followed by the sum over the ranks (which then overlaps the next
+            # step's forward); the optimizer would consume the buffers where they are zeroed here
+            if step_no[0] % window == 0:
+                if reducer is not None:
+                    reducer.wait()
+                for t in acc.values():
+                    t.zero_()
             layer.backward_accumulate(tens["dy"], inp["d_aux"], acc)
-            if reducer is not None:
+            step_no[0] += 1
+            if reducer is not None and step_no[0] % window == 0:
                 reducer.start([acc["dW_gate"], acc["dW_up"], acc["dW_down"], acc["dW_r"]])
         else:
             layer.backward(tens["dy"], inp["d_aux"], grads=grads)
@@ -311,27 +403,43 @@ def main():
     for _ in range(args.warmup):
         step()
     layer.poll()
-    layer.set_profiling(True)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+    # untimed conditioning: the same step back to back until the power state has settled
+    cond_steps = 0
+    if args.condition_seconds > 0:
+        t_c = time.perf_counter()
+        while time.perf_counter() - t_c < args.condition_seconds:
+            for _ in range(10):
+                step()
+            torch.cuda.synchronize()
+            cond_steps += 10
+    layer.poll()
+    layer.set_profiling(True)
     pdist.barrier()
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = kernel_launches()
+    t_host0 = time.perf_counter()
     ev0.record()
     for _ in range(args.steps):
         step()
     ev1.record()
     torch.cuda.synchronize()
+    t_host1 = time.perf_counter()
+    launches = kernel_launches() - launches0
     # per-stage CUDA events were recorded on the stream inside the calls, one set per step
     stage_ms, prof_steps = layer.stage_times()
     pdist.barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = None
+    if rank == 0:
+        sampler.stop()
+        clocks = sampler.summary(t_host0, t_host1)
     layer.poll()
     layer.set_profiling(False)
-    ms_total = pdist.max_over_ranks(ev0.elapsed_time(ev1))
-    ms_step = ms_total / args.steps
-    value = world * T / (ms_step / 1e3)
+    ms_step = pdist.max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
+    value = pdist.job_throughput(T, ms_step)  # tokens of all ranks over the slowest rank's time
 
     # ---- end to end through the host-buffer entry point (weights resident, activations cross PCIe each step)
     e2e = None
@@ -391,6 +499,9 @@ def main():
 
     peaks = load_peaks()
     work = stage_work(shape)
+    regime, tensor_peak = choose_peak(peaks, clocks.get("sm_mhz"), clocks.get("sm_max_mhz"))
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    mhz = clocks.get("sm_mhz")
     stages = {}
     gemm_flops = gemm_ms = 0.0
     for i, name in enumerate(STAGE_NAMES):
@@ -398,7 +509,10 @@ def main():
         kind, amount = work[name]
         if kind == "tensor":
             ach = amount / (ms * 1e-3) / 1e12 if ms > 0 else 0.0
-            stages[name] = {"ms": ms, "TFLOP/s": ach, "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
+            stages[name] = {"ms": ms, "TFLOP/s": ach, "frac_of_sustained": ach / peaks["bf16_tflops_sustained"],
+                            "frac_of_burst": ach / peaks["bf16_tflops"]}
+            if mhz and ms > 0:
+                stages[name]["flop_per_clk_per_sm"] = amount / (ms * 1e-3 * mhz * 1e6 * sm_count)
             gemm_flops += amount
             gemm_ms += ms
         else:
@@ -407,10 +521,13 @@ def main():
     dom = max(STAGE_NAMES, key=lambda n: stages[n]["ms"])
     kind, amount = work[dom]
     if kind == "tensor":
-        roof = {"bound": "tensor", "kernel": dom, "achieved": stages[dom]["TFLOP/s"],
-                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": stages[dom]["TFLOP/s"] / peaks["bf16_tflops_sustained"],
-                "peak_source": peaks["source"] + " bf16 sustained (kernel timed inside a long step)",
+        roof = {"bound": "tensor", "kernel": dom, "achieved": stages[dom]["TFLOP/s"], "peak": tensor_peak,
+                "unit": "TFLOP/s", "frac": stages[dom]["TFLOP/s"] / tensor_peak,
+                "peak_source": f"{peaks['source']} bf16 {regime} (median SM clock of the timed region "
+                               f"{mhz} MHz; sustained peak measured at {peaks['sustained_sm_mhz']:.0f} MHz, burst near "
+                               f"{peaks['sm_max_mhz']:.0f} MHz)",
+                "frac_of_burst": stages[dom]["frac_of_burst"], "frac_of_sustained": stages[dom]["frac_of_sustained"],
+                "flop_per_clk_per_sm": stages[dom].get("flop_per_clk_per_sm"),
                 "traffic": NCU_TRAFFIC.get((args.workload, dom))}
     else:
         roof = {"bound": "hbm", "kernel": dom, "achieved": stages[dom]["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -433,14 +550,19 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "mode": args.mode, "T_per_gpu": T, "d": shape.d, "E": shape.E, "top_k": shape.k,
-                       "f": shape.f, "parallelism": f"dp{world} over tokens, experts replicated (EP=1), no collective",
+                       "f": shape.f,
+                       "parallelism": f"dp{world} over tokens, experts replicated (EP=1), "
+                                      + ("weight gradients all-reduced once per accumulation window"
+                                         if reducer is not None else "no data-path collective"),
+                       "conditioning": f"{cond_steps} untimed steps (>= {args.condition_seconds} s) before the timed region",
                        "l2": l2_note,
                        "redrawn_tokens": inp["meta"]["redrawn"]},
             "grouped_gemm_tflops": gemm_tflops,
             "grouped_gemm_frac_of_sustained_bf16": gemm_tflops / peaks["bf16_tflops_sustained"],
             "grouped_gemm_frac_of_burst_bf16": gemm_tflops / peaks["bf16_tflops"],
+            "grouped_gemm_frac_of_regime_peak": gemm_tflops / tensor_peak, "regime": regime,
             "roofline": roof, "stages": stages, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-            "gpu_launches": LAUNCHES_PER_STEP * args.steps}
+            "gpu_launches": launches}
     print(json.dumps(line))
     pdist.finish()
 

@@ -70,15 +70,20 @@ typedef enum {
   MOE_ERR_UNSUPPORTED = -2,
   MOE_ERR_WORKSPACE = -3,   /* workspace_bytes smaller than moe_workspace_bytes(ctx, T) */
   MOE_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                       */
-  MOE_ERR_DEVICE_TIMEOUT = -5 /* a bounded device-side wait ran out                      */
+  MOE_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait ran out                     */
+  MOE_ERR_DEVICE_BOUNDS = -6   /* a device-side bounds check failed (MOE_FLAG_DEBUG_CHECKS) */
 } moe_status;
 
 /* Number of per-stage timers filled by moe_stage_times (see below). */
 #define MOE_NUM_STAGES 16
 
-/* Creates a context for one layer shape on the current device.  Allocates host memory only. */
+/* Creates a context for one layer shape.  Allocates host memory only.  The first call that launches work binds
+ * the context to the device that is current then; later calls with another device current are refused with
+ * MOE_ERR_INVALID_ARG (one context per device). */
 MOE_API moe_status moe_create(const moe_config* cfg /* host */, moe_ctx** out /* host */);
 MOE_API void moe_destroy(moe_ctx* ctx);
+/* Device the context is bound to, or -1 while no call has launched work yet (or ctx is NULL). */
+MOE_API int moe_ctx_device(const moe_ctx* ctx);
 
 /* Bytes of workspace needed for a call with T tokens (0 if ctx is NULL or T < 0).  The workspace holds
  * the routing tables and the activations that moe_forward saves for moe_backward. */
@@ -95,13 +100,19 @@ MOE_API moe_status moe_workspace_find(const moe_ctx* ctx, int64_t T, const char*
 
 MOE_API const char* moe_status_string(moe_status s);
 
-/* Synchronises the stream and returns the device-side status word of the workspace. */
+/* Synchronises the stream and reports the device-side status word of the workspace.  The word is sticky: the
+ * first failure a kernel records stays there - no later kernel or call overwrites or clears it - until this call
+ * (or moe_step_host_end) has returned it once; reporting acknowledges it, after which the context and the
+ * workspace are usable again.  A workspace no call has used yet reports MOE_OK. */
 MOE_API moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_stream);
+
+/* Number of kernels the library has launched in this process so far (all contexts; copies and memsets not counted). */
+MOE_API long long moe_kernel_launches(void);
 
 /* Exercises the device-side failure path without faulting anything: launches one tiny kernel whose bounded wait
  * (on a barrier nothing signals) runs out after a few thousand polls; the kernel records the timeout in the
- * workspace's status word and returns.  A following moe_poll_status reports MOE_ERR_DEVICE_TIMEOUT; the context
- * stays usable and the next moe_forward clears the word.  The layer's kernels bound every wait the same way
+ * workspace's status word and returns.  A following moe_poll_status - also one that comes after further
+ * moe_forward / moe_backward calls - reports MOE_ERR_DEVICE_TIMEOUT once; the context stays usable.  The layer's kernels bound every wait the same way
  * (about a second); nothing in the library makes a GPU fault, trap or hang on purpose. */
 MOE_API moe_status moe_selftest_timeout(moe_ctx* ctx, void* workspace, void* cuda_stream);
 
@@ -211,6 +222,8 @@ MOE_API moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, floa
  * downloads their gradients; with 0 the weights must already be resident from an earlier call.  The copies run on
  * two streams of the context so that dy arrives while forward runs and y leaves while backward runs. */
 MOE_API size_t moe_e2e_device_bytes(const moe_ctx* ctx, int64_t T);
+/* Byte offset, inside `dev`, of the layer workspace the host-buffer calls use (what moe_poll_status wants). */
+MOE_API size_t moe_e2e_workspace_offset(const moe_ctx* ctx, int64_t T);
 MOE_API moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16_t* x, const uint16_t* W_r,
                          const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
                          const uint16_t* dy, float d_aux, uint16_t* y, float* aux_loss, uint16_t* dx,
@@ -223,7 +236,8 @@ MOE_API moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, cons
  * slots in flight (begin(0), begin(1), end(0), begin(0), end(1), ...) the upload of the next batch and the download
  * of the previous results overlap the current step's kernels.  Weights must be resident (one earlier moe_step_host
  * with copy_weights = 1); the weight gradients of the most recent step stay on the device.  Host buffers of a slot
- * must stay untouched between its begin and end.  Device-side status is reported by moe_poll_status. */
+ * must stay untouched between its begin and end.  moe_step_host_end returns MOE_ERR_DEVICE_TIMEOUT (once) when a
+ * kernel up to and including that slot's step recorded a failure in the workspace's status word. */
 MOE_API moe_status moe_step_host_begin(moe_ctx* ctx, int slot, int64_t T, const uint16_t* x, const uint16_t* dy,
                                        float d_aux, uint16_t* y, float* aux_loss, uint16_t* dx, void* dev,
                                        size_t dev_bytes, void* cuda_stream);
@@ -244,8 +258,10 @@ MOE_API moe_status moe_step_host_end(moe_ctx* ctx, int slot);
  *
  * Cost and rules.  The scratch is MOE_STATIC_MAX_DE * 8 floats = 8 MiB of device memory on every GPU that loads the
  * library, held until the process ends.  The first call on a device looks up the array's device address
- * (cudaGetSymbolAddress, with that device current); make that first call during start-up, ahead of any stream
- * capture.  All calls on one GPU share the array: two calls whose kernels can overlap on the GPU (different streams,
+ * (cudaGetSymbolAddress, with that device current) and, where the CUDA runtime loads modules lazily, is also the
+ * moment the library image with its 8 MiB array is loaded onto that device; make that first call during start-up, ahead
+ * of any stream capture.  The address is cached per device for the life of the process: after cudaDeviceReset on a
+ * device the cached address is stale and this entry point must not be used on it again.  All calls on one GPU share the array: two calls whose kernels can overlap on the GPU (different streams,
  * different threads) race on it and must be ordered by the caller.  The array keeps whatever the previous call
  * left; that is harmless because each call overwrites every partial it later reads. */
 #define MOE_STATIC_MAX_DE 262144

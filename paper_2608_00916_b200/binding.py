@@ -19,7 +19,8 @@ EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_fi
            "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout",
            "moe_forward_inference", "moe_inference_workspace_bytes", "moe_backward_accumulate",
            "moe_lora_workspace_bytes", "moe_lora_forward", "moe_lora_backward",
-           "moe_step_host_begin", "moe_step_host_end"]
+           "moe_step_host_begin", "moe_step_host_end", "moe_kernel_launches", "moe_ctx_device",
+           "moe_e2e_workspace_offset"]
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -81,8 +82,14 @@ def load_library() -> C.CDLL:
     lib.moe_lora_backward.restype = C.c_int
     lib.moe_e2e_device_bytes.argtypes = [vp, i64]
     lib.moe_e2e_device_bytes.restype = sz
+    lib.moe_e2e_workspace_offset.argtypes = [vp, i64]
+    lib.moe_e2e_workspace_offset.restype = sz
     lib.moe_step_host.argtypes = [vp, i64, C.c_int] + [vp] * 6 + [C.c_float] + [vp] * 7 + [vp, sz, vp]
     lib.moe_step_host.restype = C.c_int
+    lib.moe_kernel_launches.argtypes = []
+    lib.moe_kernel_launches.restype = C.c_longlong
+    lib.moe_ctx_device.argtypes = [vp]
+    lib.moe_ctx_device.restype = C.c_int
     lib.moe_selftest_timeout.argtypes = [vp, vp, vp]
     lib.moe_selftest_timeout.restype = C.c_int
     lib.moe_router_wgrad_static.argtypes = [i64, C.c_int32, C.c_int32, vp, vp, vp, vp]
@@ -94,6 +101,11 @@ def load_library() -> C.CDLL:
 def _check(lib, rc: int, what: str) -> None:
     if rc != 0:
         raise MoEError(f"{what}: {lib.moe_status_string(rc).decode()} ({rc})")
+
+
+def kernel_launches() -> int:
+    """Kernels the library has launched in this process so far."""
+    return int(load_library().moe_kernel_launches())
 
 
 def _ptr(t):
@@ -332,6 +344,9 @@ class MoELayer:
     # ---- host-buffer step (end-to-end timing)
     def e2e_device_bytes(self, T: int) -> int:
         return int(self.lib.moe_e2e_device_bytes(self.h, T))
+
+    def e2e_workspace_offset(self, T: int) -> int:
+        return int(self.lib.moe_e2e_workspace_offset(self.h, T))
 
     def step_host(self, T, dev_buf, host, d_aux: float, copy_weights: bool):
         """host: dict of pinned CPU tensors x, W_r, W_gate, W_up, W_down, dy and outputs y, aux, dx, dW_r, dW_gate,

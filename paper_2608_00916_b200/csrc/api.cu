@@ -1,6 +1,8 @@
 // C ABI of the MoE layer library (see include/moe.h): argument checks, workspace layout, kernel sequencing.
+#include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 
 #include "common.cuh"
@@ -8,6 +10,9 @@
 namespace moe {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static std::atomic<long long> g_kernel_launches{0};
+void note_launch(int n) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
 
 WsLayout make_layout(const Shape& s, int64_t T) {
   WsLayout L;
@@ -68,10 +73,12 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   return L;
 }
 
+// The first call that needs the device binds the context to the current one (SM count, tensor-map encoder, the
+// per-device kernel attributes); every later call must come with the same device current.
 static moe_status ensure_device(moe_ctx_impl* c) {
-  if (c->encode_fn) return MOE_OK;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+  if (c->encode_fn) return dev == c->device ? MOE_OK : MOE_ERR_INVALID_ARG;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return MOE_ERR_CUDA;
   if (prop.major != 10) return MOE_ERR_UNSUPPORTED;  // tcgen05 / TMEM kernels: sm_100a only, no fallback
@@ -83,7 +90,18 @@ static moe_status ensure_device(moe_ctx_impl* c) {
       q != cudaDriverEntryPointSuccess)
     return MOE_ERR_CUDA;
   c->encode_fn = fn;
+  c->gemm_timers = getenv("MOE_GEMM_TIMERS") != nullptr;
+  memset(c->attr_done, 0, sizeof(c->attr_done));
   return MOE_OK;
+}
+
+// Acknowledges a reported failure: the word returns to DEV_OK only if it still holds the code the host has seen.
+__global__ void status_ack_kernel(int32_t* status, int seen) {
+  if (atomicCAS(status, seen, DEV_OK) == seen) status[1] = 0;
+}
+
+static moe_status status_to_code(int v) {
+  return v == DEV_OK ? MOE_OK : (v == DEV_BOUNDS ? MOE_ERR_DEVICE_BOUNDS : MOE_ERR_DEVICE_TIMEOUT);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -119,6 +137,7 @@ moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
   if (!c) return MOE_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
   c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
+  c->device = -1;  // bound by the first call that launches work
   c->tile_mode = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 1 : ((cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 2 : 0);
   *out = reinterpret_cast<moe_ctx*>(c);
   return MOE_OK;
@@ -137,8 +156,10 @@ void moe_destroy(moe_ctx* ctx) {
     cudaStreamDestroy(c->s_in);
     cudaStreamDestroy(c->s_out);
     for (int i = 0; i < 6; ++i) cudaEventDestroy(c->e2e_ev[i]);
-    for (int sl = 0; sl < 2; ++sl)
+    for (int sl = 0; sl < 2; ++sl) {
       for (int i = 0; i < 5; ++i) cudaEventDestroy(c->pipe_ev[sl][i]);
+      if (c->pipe_status[sl]) cudaFreeHost(c->pipe_status[sl]);
+    }
   }
   delete c;
 }
@@ -193,10 +214,12 @@ const char* moe_status_string(moe_status s) {
   switch (s) {
     case MOE_OK: return "ok";
     case MOE_ERR_INVALID_ARG: return "invalid argument";
-    case MOE_ERR_UNSUPPORTED: return "unsupported device or configuration (sm_100a required)";
+    case MOE_ERR_UNSUPPORTED:
+      return "unsupported: the device is not sm_100a, or the shape is beyond what this entry point handles";
     case MOE_ERR_WORKSPACE: return "workspace too small";
     case MOE_ERR_CUDA: return "CUDA call failed";
     case MOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case MOE_ERR_DEVICE_BOUNDS: return "a device-side bounds check failed (debug checks)";
   }
   return "unknown status";
 }
@@ -205,14 +228,25 @@ moe_status moe_poll_status(moe_ctx* ctx, const void* workspace, void* cuda_strea
   if (!ctx || !workspace) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   const WsLayout L = make_layout(c->s, 0);
-  int32_t st[2] = {0, 0};
+  int32_t st[4] = {0, 0, 0, 0};
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  if (cudaMemcpyAsync(st, static_cast<const char*>(workspace) + L.status, sizeof(st), cudaMemcpyDeviceToHost, s) !=
-      cudaSuccess)
-    return MOE_ERR_CUDA;
+  int32_t* dev_status = reinterpret_cast<int32_t*>(const_cast<char*>(static_cast<const char*>(workspace)) + L.status);
+  if (cudaMemcpyAsync(st, dev_status, sizeof(st), cudaMemcpyDeviceToHost, s) != cudaSuccess) return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return MOE_ERR_CUDA;
-  return st[0] == DEV_OK ? MOE_OK : MOE_ERR_DEVICE_TIMEOUT;
+  if (st[2] != STATUS_COOKIE0 || st[3] != STATUS_COOKIE1) return MOE_OK;  // no call has used this workspace yet
+  if (st[0] == DEV_OK) return MOE_OK;
+  // reported: acknowledge, so that the next failure can be recorded
+  status_ack_kernel<<<1, 1, 0, s>>>(dev_status, st[0]);
+  note_launch();
+  if (cudaStreamSynchronize(s) != cudaSuccess) return MOE_ERR_CUDA;
+  return status_to_code(st[0]);
 }
+
+int moe_ctx_device(const moe_ctx* ctx) {
+  return ctx ? reinterpret_cast<const moe_ctx_impl*>(ctx)->device : -1;
+}
+
+long long moe_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 // One CTA waits, with the library's bounded-wait helper cut down to a few thousand polls, on an mbarrier that
 // nothing ever signals; the wait gives up, records DEV_TIMEOUT in the status word and the kernel returns normally.
@@ -220,6 +254,12 @@ __global__ void selftest_timeout_kernel(int32_t* status) {
   __shared__ __align__(8) uint64_t bar;
   const uint32_t b = static_cast<uint32_t>(__cvta_generic_to_shared(&bar));
   if (threadIdx.x == 0) {
+    if (status[2] != STATUS_COOKIE0 || status[3] != STATUS_COOKIE1) {  // workspace not seen before
+      status[0] = DEV_OK;
+      status[1] = 0;
+      status[2] = STATUS_COOKIE0;
+      status[3] = STATUS_COOKIE1;
+    }
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b) : "memory");
     bool done = false;
     for (int i = 0; i < 4096 && !done; ++i) {
@@ -233,10 +273,7 @@ __global__ void selftest_timeout_kernel(int32_t* status) {
           : "memory");
       done = ok != 0;
     }
-    if (!done) {
-      atomicExch(status, DEV_TIMEOUT);
-      status[1] = 9000;
-    }
+    if (!done) record_status(status, DEV_TIMEOUT, 9000);
   }
 }
 
@@ -246,6 +283,7 @@ moe_status moe_selftest_timeout(moe_ctx* ctx, void* workspace, void* cuda_stream
   const WsLayout L = make_layout(c->s, 0);
   selftest_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + L.status));
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -312,6 +350,7 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
   io.x = x; io.W_r = W_r; io.b_r = b_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
   io.idx_out = topk_idx; io.gates_out = topk_w; io.logits_out = logits_out;
   const bool tc_router = router_on_tensor_cores(s) && logits_in == nullptr;
+  launch_prepare(L, ws, st);  // before any kernel that may record a status
   {
     StageTimer tm(c, st, 0);
     if (T > 0 && tc_router) {
@@ -586,6 +625,10 @@ static moe_status e2e_setup(moe_ctx_impl* c) {
   for (int sl = 0; sl < 2; ++sl)
     for (int i = 0; i < 5; ++i)
       if (cudaEventCreateWithFlags(&c->pipe_ev[sl][i], cudaEventDisableTiming) != cudaSuccess) return MOE_ERR_CUDA;
+  for (int sl = 0; sl < 2; ++sl)
+    if (cudaHostAlloc(reinterpret_cast<void**>(&c->pipe_status[sl]), 4 * sizeof(int32_t), cudaHostAllocDefault) !=
+        cudaSuccess)
+      return MOE_ERR_CUDA;
   c->e2e_created = 1;
   return MOE_OK;
 }
@@ -593,6 +636,11 @@ static moe_status e2e_setup(moe_ctx_impl* c) {
 size_t moe_e2e_device_bytes(const moe_ctx* ctx, int64_t T) {
   if (!ctx || T < 0) return 0;
   return e2e_layout(reinterpret_cast<const moe_ctx_impl*>(ctx)->s, T).total;
+}
+
+size_t moe_e2e_workspace_offset(const moe_ctx* ctx, int64_t T) {
+  if (!ctx || T < 0) return 0;
+  return e2e_layout(reinterpret_cast<const moe_ctx_impl*>(ctx)->s, T).ws;
 }
 
 moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16_t* x, const uint16_t* W_r,
@@ -712,8 +760,12 @@ moe_status moe_step_host_begin(moe_ctx* ctx, int slot, int64_t T, const uint16_t
                     reinterpret_cast<float*>(D + L.dWr), nullptr, U(L.dWg), U(L.dWu), U(L.dWd), D + L.ws, wsb,
                     cuda_stream);
   if (rc != MOE_OK) return rc;
+  // the status block of the workspace travels with the slot's results
+  c->pipe_status_dev = reinterpret_cast<int32_t*>(D + L.ws + make_layout(s, 0).status);
   ok = cudaEventRecord(ev[3], st) == cudaSuccess && cudaStreamWaitEvent(c->s_out, ev[3], 0) == cudaSuccess &&
        cudaMemcpyAsync(dx, D + odx, td, cudaMemcpyDeviceToHost, c->s_out) == cudaSuccess &&
+       cudaMemcpyAsync(c->pipe_status[slot], c->pipe_status_dev, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost,
+                       c->s_out) == cudaSuccess &&
        cudaEventRecord(ev[4], c->s_out) == cudaSuccess;
   c->pipe_used[slot] = 1;
   return ok ? MOE_OK : MOE_ERR_CUDA;
@@ -723,7 +775,13 @@ moe_status moe_step_host_end(moe_ctx* ctx, int slot) {
   if (!ctx || (slot != 0 && slot != 1)) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
   if (!c->e2e_created || !c->pipe_used[slot]) return MOE_ERR_INVALID_ARG;
-  return cudaEventSynchronize(c->pipe_ev[slot][4]) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  if (cudaEventSynchronize(c->pipe_ev[slot][4]) != cudaSuccess) return MOE_ERR_CUDA;
+  const int32_t* hs = c->pipe_status[slot];
+  if (hs[2] != STATUS_COOKIE0 || hs[3] != STATUS_COOKIE1 || hs[0] == DEV_OK) return MOE_OK;
+  // a kernel of this step (or an earlier, not yet reported one) recorded a failure: report it once, then acknowledge
+  status_ack_kernel<<<1, 1, 0, c->s_out>>>(c->pipe_status_dev, hs[0]);
+  note_launch();
+  return status_to_code(hs[0]);
 }
 
 }  // extern "C"

@@ -42,6 +42,7 @@ void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* g
                     uint16_t* y, cudaStream_t st) {
   if (T == 0) return;
   combine_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, o, gates, inv, y);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------------ router backward
@@ -140,6 +141,7 @@ void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int
   router_bwd_kernel<<<static_cast<unsigned>((T + 7) / 8), 256, 0, st>>>(T, s.E, s.k, logits, idx, gates, dg_part,
                                                                         dg_tiles, rows_max, inv, dg, counts, d_aux, dl,
                                                                         dl_hi, dl_lo);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------------ dW_r, db_r
@@ -241,9 +243,14 @@ void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, f
   if (!partials_ready) {
     dim3 grid(s.d / DW_BM, DWR_SPLIT);
     dwr_partial_kernel<<<grid, 256, sizeof(float) * DW_BK * s.E, st>>>(T, s.d, s.E, x, dl, part);
+    note_launch();
   }
   dwr_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(n, part, dW_r, accumulate ? 1 : 0);
-  if (db_r) dbr_kernel<<<(s.E + 31) / 32, 256, 0, st>>>(T, s.E, dl, db_r, accumulate ? 1 : 0);
+  note_launch();
+  if (db_r) {
+    dbr_kernel<<<(s.E + 31) / 32, 256, 0, st>>>(T, s.E, dl, db_r, accumulate ? 1 : 0);
+    note_launch();
+  }
 }
 
 // ------------------------------------------------------------------------------------------ unpermute backward
@@ -378,6 +385,7 @@ void launch_unpermute_sum(const Shape& s, int64_t T, const uint16_t* dxp, const 
                           uint16_t* dx, cudaStream_t st) {
   if (T == 0) return;
   unpermute_sum_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, dxp, inv, dxr, dx);
+  note_launch();
 }
 
 void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const float* dl,
@@ -385,6 +393,7 @@ void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const 
   if (T == 0) return;
   unpermute_bwd_kernel<<<static_cast<unsigned>((T + UB_TOK - 1) / UB_TOK), 256, sizeof(float) * UB_TOK * s.E, st>>>(
       T, s.d, s.E, s.k, dxp, inv, dl, W_r, dx);
+  note_launch();
 }
 
 }  // namespace moe

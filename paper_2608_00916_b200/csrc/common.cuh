@@ -20,6 +20,11 @@ constexpr int DWR_SPLIT = 8;     // token slices of the dW_r contraction
 // status word values written by kernels
 constexpr int DEV_OK = 0;
 constexpr int DEV_TIMEOUT = 1;
+constexpr int DEV_BOUNDS = 2;
+// A workspace whose status block carries this pair in words [2], [3] has been initialised by the library; anything
+// else is memory the library sees for the first time (its status word is then meaningless and gets cleared).
+constexpr int STATUS_COOKIE0 = 0x4D6F4531;
+constexpr int STATUS_COOKIE1 = 0x62323030;
 
 struct Shape {
   int d, E, f, k;
@@ -27,7 +32,7 @@ struct Shape {
 
 // Byte offsets of every internal buffer inside the caller's workspace (all 256-byte aligned).
 struct WsLayout {
-  size_t status;       // int32[16]   [0] device status, [1] where it happened
+  size_t status;       // int32[16]   [0] device status (first failure sticks), [1] where it happened, [2..3] cookie
   size_t timers;       // int64[GEMM_KINDS][8] cycle counters of the GEMM roles (filled only when MOE_GEMM_TIMERS is set)
   size_t counts;       // int32[E]    rows per expert
   size_t offsets;      // int32[E+1]  exclusive scan of counts (canonical, unpadded)
@@ -75,6 +80,10 @@ struct moe_ctx_impl {
   int device;
   void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
   int tile_mode;    // 0: choose per GEMM (see use_pair_tiles), 1: always CTA pairs, 2: always one-CTA tiles
+  int gemm_timers;  // MOE_GEMM_TIMERS was set when the context first touched its device
+  // cudaFuncSetAttribute (dynamic shared memory opt-in) is per device: remembered here, for the device the context is
+  // bound to, per kernel family (0: one-CTA kernels, 1: CTA-pair kernels) and GEMM kind
+  unsigned char attr_done[2][16];
   int profiling;
   cudaEvent_t ev[MOE_PROF_RING][MOE_NUM_STAGES][2];
   unsigned char ev_used[MOE_PROF_RING][MOE_NUM_STAGES];
@@ -86,10 +95,14 @@ struct moe_ctx_impl {
   cudaEvent_t pipe_ev[2][5];  // pipelined host steps, per slot: x in, dy in, forward done, backward done, results out
   int pipe_used[2];
   int e2e_created;
+  int32_t* pipe_status[2];  // pinned host copies of the device status block, one per slot of the pipelined host steps
+  int32_t* pipe_status_dev; // the status block those copies come from
   int64_t prof_read;   // pairs already reported by moe_stage_times
 };
 
 // ---- launchers (route.cu)
+// first kernel of a forward call: zero row gates, initialise the status block of a workspace seen for the first time
+void launch_prepare(const WsLayout& L, char* ws, cudaStream_t st);
 void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
                    const float* logits_in, float* logits, int32_t* idx, float* gates, int32_t* idx_out,
                    float* gates_out, float* logits_out, float* psum_part, cudaStream_t st);
@@ -172,7 +185,15 @@ inline int64_t router_psum_rows(const Shape& s, int64_t T, bool logits_given) {
   return (router_on_tensor_cores(s) && !logits_given) ? 4 * ((T + 127) / 128) : (T + ROUTER_TOK - 1) / ROUTER_TOK;
 }
 
+// counts kernel launches of the library (process-wide; read through moe_kernel_launches)
+void note_launch(int n = 1);
+
 // ---- device helpers
+// Records a device-side failure.  The first failure sticks: later ones do not overwrite it, and no kernel ever resets
+// the word (the host acknowledges it after reporting it, see moe_poll_status).
+__device__ __forceinline__ void record_status(int32_t* status, int code, int where) {
+  if (atomicCAS(status, DEV_OK, code) == DEV_OK) status[1] = where;
+}
 __device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // .x = lo (low 16 bits), .y = hi

@@ -21,8 +21,6 @@
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer (owns the TMEM allocation), warps 2..9 epilogue (2..5 for the
 // routing kind).  The expert-LoRA variant runs on the same template (launch_lora_gemm at the end of this file).
 // Every mbarrier wait is bounded; on a timeout the kernel records it in the status word and leaves.
-#include <stdlib.h>  // getenv (MOE_GEMM_TIMERS)
-
 #include "gemm_common.cuh"
 
 namespace moe {
@@ -101,8 +99,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       atomicAdd(p.timers + 1, static_cast<unsigned long long>(t_wait));               // producer: waiting for a free stage
     }
     if (!ok && lane == 0) {
-      atomicExch(p.status, DEV_TIMEOUT);
-      p.status[1] = 100 + KIND;
+      record_status(p.status, DEV_TIMEOUT, 100 + KIND);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -160,8 +157,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       atomicAdd(p.timers + 4, static_cast<unsigned long long>(t_full));               // waiting for operands
     }
     if (!ok && lane == 0) {
-      atomicExch(p.status, DEV_TIMEOUT);
-      p.status[1] = 200 + KIND;
+      record_status(p.status, DEV_TIMEOUT, 200 + KIND);
     }
   } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------------------------ epilogue (128 TMEM lanes; two warps per
@@ -250,8 +246,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       atomicAdd(p.timers + 7, 1ull);                                                  // CTAs counted
     }
     if (!ok && lane == 0) {
-      atomicExch(p.status, DEV_TIMEOUT);
-      p.status[1] = 300 + KIND;
+      record_status(p.status, DEV_TIMEOUT, 300 + KIND);
     }
   }
 
@@ -294,14 +289,14 @@ static bool map_3d(void* fn, CUtensorMap* m, const void* base, int64_t E, int64_
 
 template <int KIND>
 static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream_t st) {
-  static bool attr_done[GEMM_KINDS] = {false};
-  if (!attr_done[KIND]) {
+  if (!ctx->attr_done[0][KIND]) {  // per device: the context is bound to one
     if (cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(GEMM_SMEM)) != cudaSuccess)
       return MOE_ERR_CUDA;
-    attr_done[KIND] = true;
+    ctx->attr_done[0][KIND] = 1;
   }
   grouped_gemm_kernel<KIND><<<ctx->sm_count, KIND == GEMM_RT ? 192 : GEMM_THREADS, GEMM_SMEM, st>>>(p);
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -329,7 +324,7 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.counts = reinterpret_cast<const int32_t*>(ws + L.counts);
   p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
   p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
-  p.timers = getenv("MOE_GEMM_TIMERS") ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
+  p.timers = ctx->gemm_timers ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
   // CTA pairs (256 x 256 tiles, half of B per SM) or one-CTA tiles (128 x 256)?  Pairs move a third less operand
   // data per flop, which under the power cap is worth ~10 % on long-K tiles.  Row GEMMs pay for them with the dummy
   // half-tile of every expert that has an odd number of 128-row blocks, so they pair only when that expected waste

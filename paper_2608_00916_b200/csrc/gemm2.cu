@@ -174,8 +174,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       atomicAdd(p.timers + 1, static_cast<unsigned long long>(t_wait));
     }
     if (!ok && lane == 0) {
-      atomicExch(p.status, DEV_TIMEOUT);
-      p.status[1] = 1100 + KIND;
+      record_status(p.status, DEV_TIMEOUT, 1100 + KIND);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
@@ -237,8 +236,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
         atomicAdd(p.timers + 4, static_cast<unsigned long long>(t_full));
       }
       if (!ok && lane == 0) {
-        atomicExch(p.status, DEV_TIMEOUT);
-        p.status[1] = 1200 + KIND;
+        record_status(p.status, DEV_TIMEOUT, 1200 + KIND);
       }
     }
   } else {
@@ -281,8 +279,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       atomicAdd(p.timers + 7, 1ull);
     }
     if (!ok && lane == 0) {
-      atomicExch(p.status, DEV_TIMEOUT);
-      p.status[1] = 1300 + KIND;
+      record_status(p.status, DEV_TIMEOUT, 1300 + KIND);
     }
   }
 
@@ -296,15 +293,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
 
 template <int KIND>
 static moe_status launch_pair_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream_t st) {
-  static bool attr_done[GEMM_KINDS] = {false};
-  if (!attr_done[KIND]) {
+  if (!ctx->attr_done[1][KIND]) {  // per device: the context is bound to one
     if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(GEMM2_SMEM)) != cudaSuccess)
       return MOE_ERR_CUDA;
-    attr_done[KIND] = true;
+    ctx->attr_done[1][KIND] = 1;
   }
   const int grid = ctx->sm_count & ~1;  // whole pairs
   grouped_gemm_pair_kernel<KIND><<<grid, GEMM2_THREADS, GEMM2_SMEM, st>>>(p);
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

@@ -2,6 +2,8 @@
 // deterministic token permutation (per-tile histogram, prefix scan, stable scatter, row copy).  The router kernel here
 // is the SIMT path (expert counts that are not a multiple of 8, or caller-supplied logits); otherwise the logits are
 // contracted on the tensor cores (gemm.cu, kind RT).
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace moe {
@@ -193,6 +195,7 @@ void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t*
   const size_t smem = sizeof(float) * (RT_CH * ROUTER_TOK + ROUTER_TOK * s.E + 8 * s.E);
   router_kernel<<<blocks, 256, smem, st>>>(T, s.d, s.E, s.k, x, W_r, b_r, logits_in, logits, idx, gates, idx_out,
                                            gates_out, logits_out, psum_part);
+  note_launch();
 }
 
 // ------------------------------------------------------------------------------------------ permutation
@@ -240,17 +243,13 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
                                                             int32_t* __restrict__ expert_order,
                                                             const float* __restrict__ psum_part,
                                                             float* __restrict__ psum, int32_t* __restrict__ counts_out,
-                                                            float* __restrict__ aux_out, int32_t* __restrict__ status) {
+                                                            float* __restrict__ aux_out) {
   __shared__ int s_cnt[MAX_E];
   __shared__ int s_pad[MAX_E + 1];
   __shared__ int s_pair[MAX_E + 1];
   __shared__ float s_term[MAX_E];
   __shared__ float s_ps[SCAN_THREADS];
   const int tid = threadIdx.x;
-  if (tid == 0) {
-    status[0] = DEV_OK;
-    status[1] = 0;
-  }
   // column sums of p: G groups of threads stride over the partial rows
   const int G = SCAN_THREADS / E;
   if (tid < G * E) {
@@ -442,6 +441,29 @@ void launch_gather_rows(const Shape& s, int64_t T, const WsLayout& L, const char
   scatter_rows_kernel<<<tok_blocks + s.E, 256, 0, st>>>(
       T, s.d, s.k, s.E, tok_blocks, src, reinterpret_cast<const int32_t*>(ws + L.inv),
       reinterpret_cast<const int32_t*>(ws + L.counts), reinterpret_cast<const int32_t*>(ws + L.pad_offsets), rows);
+  note_launch();
+}
+
+// First kernel of every forward call: clears the row gates (pad rows must read 0) and makes sure the workspace's status
+// block is initialised.  A status block that already carries the cookie is left alone, so a failure recorded by an
+// earlier call stays visible until the host has reported it; memory seen for the first time gets a clean block.
+__global__ void __launch_bounds__(256) prepare_kernel(int32_t* __restrict__ status, float* __restrict__ row_gate,
+                                                      int64_t rows) {
+  if (blockIdx.x == 0 && threadIdx.x == 0 && (status[2] != STATUS_COOKIE0 || status[3] != STATUS_COOKIE1)) {
+    status[0] = DEV_OK;
+    status[1] = 0;
+    status[2] = STATUS_COOKIE0;
+    status[3] = STATUS_COOKIE1;
+  }
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; i < rows; i += static_cast<int64_t>(gridDim.x) * 256)
+    row_gate[i] = 0.f;
+}
+
+void launch_prepare(const WsLayout& L, char* ws, cudaStream_t st) {
+  const int blocks = static_cast<int>(std::min<int64_t>(296, std::max<int64_t>(1, (L.rows_max + 255) / 256)));
+  prepare_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + L.status),
+                                         reinterpret_cast<float*>(ws + L.row_gate), L.rows_max);
+  note_launch();
 }
 
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
@@ -450,8 +472,10 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
   int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
   const int tiles = static_cast<int>(L.tok_tiles);
   const size_t msm = sizeof(uint32_t) * 8 * s.E;
-  cudaMemsetAsync(ws + L.row_gate, 0, sizeof(float) * L.rows_max, st);
-  if (tiles > 0) hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
+  if (tiles > 0) {
+    hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
+    note_launch();
+  }
   scan_kernel<<<1, SCAN_THREADS, 0, st>>>(T, s.E, s.k, tiles, psum_rows, tile_counts,
                                  reinterpret_cast<int32_t*>(ws + L.counts), reinterpret_cast<int32_t*>(ws + L.offsets),
                                  reinterpret_cast<int32_t*>(ws + L.pad_offsets),
@@ -460,13 +484,14 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
                                  reinterpret_cast<int32_t*>(ws + L.pair_tab),
                                  reinterpret_cast<int32_t*>(ws + L.expert_order),
                                  reinterpret_cast<const float*>(ws + L.psum_part),
-                                 reinterpret_cast<float*>(ws + L.psum), counts_out, aux_out,
-                                 reinterpret_cast<int32_t*>(ws + L.status));
+                                 reinterpret_cast<float*>(ws + L.psum), counts_out, aux_out);
+  note_launch();
   if (tiles > 0) {
     scatter_kernel<<<tiles, TOK_TILE, msm, st>>>(
         T, s.E, s.k, idx, tile_counts, reinterpret_cast<const int32_t*>(ws + L.offsets),
         reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const float*>(ws + L.gates),
         reinterpret_cast<int32_t*>(ws + L.inv), reinterpret_cast<float*>(ws + L.row_gate), perm_out);
+    note_launch();
     launch_gather_rows(s, T, L, ws, x, reinterpret_cast<uint16_t*>(ws + L.xp), st);
   }
 }

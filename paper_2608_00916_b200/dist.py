@@ -26,11 +26,42 @@ def shard_seed(seed: int, rank: int) -> int:
     return seed + 7919 * rank
 
 
-def tokens_per_rank(total_tokens: int, world: int, rank: int) -> int:
-    """Strong-scaling split of a fixed batch (not used by the weak-scaling benchmark): balanced, remainder to the
-    lowest ranks."""
-    base, rem = divmod(total_tokens, world)
-    return base + (1 if rank < rem else 0)
+def rank_environment(rank: int, world: int, port: int, base_env=None) -> dict:
+    """Environment of rank `rank` of a one-node job: what torch.distributed's env:// rendezvous and bench.py read."""
+    env = dict(os.environ if base_env is None else base_env)
+    env.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), LOCAL_WORLD_SIZE=str(world),
+               MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    env.setdefault("NCCL_DEBUG", "INFO")  # leaves the communicator's transport line (NVLS or not) in the log
+    return env
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_ranks(n: int, script: str, argv, port: int | None = None, python: str | None = None, timeout=None) -> int:
+    """Starts `n` copies of `python script argv...`, one per rank (rank r is meant for GPU r), waits for all of them
+    and returns the first non-zero exit code (0 if none).  Rank 0 inherits stdout; the other ranks' stdout is dropped
+    (they print nothing by contract), every rank keeps stderr."""
+    import subprocess
+    import sys
+    port = free_port() if port is None else port
+    procs = []
+    for r in range(n):
+        procs.append(subprocess.Popen([python or sys.executable, script, *argv], env=rank_environment(r, n, port),
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    for p in procs:
+        try:
+            code = p.wait(timeout=timeout)
+        except subprocess.TimeoutExpired:
+            p.kill()  # exactly the process started here
+            code = 124
+        rc = rc or code
+    return rc
 
 
 def barrier() -> None:

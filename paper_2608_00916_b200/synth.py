@@ -143,6 +143,32 @@ def zipf_bias(seed: int, E: int, sigma_l: float, alpha: float, s: float = 1.2) -
     return b.astype(np.float32)
 
 
+def _guard_tokens(x: np.ndarray, W_r: np.ndarray, b_r, k: int, seed: int, x_std: float) -> int:
+    """Redraws (in place) the token rows of x that violate the gap guard against router (W_r, b_r); returns how many
+    rows were redrawn in total."""
+    redrawn = 0
+    d = x.shape[1]
+    for attempt in range(64):
+        l = _guard_logits(x, W_r, b_r)
+        bad = np.nonzero(_gap_violations(l, k))[0]
+        if bad.size == 0:
+            return redrawn
+        g = _stream(seed, _TID["x_redraw"], attempt)
+        v = g.standard_normal((bad.size, d), dtype=np.float32) * np.float32(x_std)
+        x[bad] = f32_to_bf16_bits(v)
+        redrawn += int(bad.size)
+    raise RuntimeError("gap guard did not converge")
+
+
+def make_tokens(shape: MoEShape, seed: int, W_r: np.ndarray, b_r=None, x_std: float = 1.0, guard: bool = True,
+                threads: int = 8) -> dict:
+    """A token batch (x, dy) of its own seed for a router that is given: the batch of a data-parallel rank, whose
+    tokens must keep the gap guard against the weights every rank shares."""
+    x = normal_bf16(seed, "x", (shape.T, shape.d), x_std, threads)
+    redrawn = _guard_tokens(x, W_r, b_r, shape.k, seed, x_std) if (guard and shape.T > 0) else 0
+    return {"x": x, "dy": normal_bf16(seed, "dy", (shape.T, shape.d), 1.0, threads), "redrawn": redrawn}
+
+
 def make_inputs(shape: MoEShape, seed: int, x_std: float = 1.0, skew: bool = False, w_std: float = 0.02,
                 guard: bool = True, threads: int = 8) -> dict:
     """Draw one problem instance.
@@ -170,17 +196,7 @@ def make_inputs(shape: MoEShape, seed: int, x_std: float = 1.0, skew: bool = Fal
         meta["alpha"] = alpha
         meta["sigma_l"] = sigma_l
     if guard and T > 0:
-        for attempt in range(64):
-            l = _guard_logits(x, W_r, b_r)
-            bad = np.nonzero(_gap_violations(l, k))[0]
-            if bad.size == 0:
-                break
-            g = _stream(seed, _TID["x_redraw"], attempt)
-            v = g.standard_normal((bad.size, d), dtype=np.float32) * np.float32(x_std)
-            x[bad] = f32_to_bf16_bits(v)
-            meta["redrawn"] += int(bad.size)
-        else:
-            raise RuntimeError("gap guard did not converge")
+        meta["redrawn"] = _guard_tokens(x, W_r, b_r, k, seed, x_std)
         meta["histogram"] = _load_histogram(_guard_logits(x, W_r, b_r), k).tolist() if E <= 256 else None
     out = {
         "x": x, "W_r": W_r, "b_r": b_r,

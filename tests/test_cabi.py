@@ -116,3 +116,21 @@ def test_other_entry_points_reject_bad_arguments_before_launch(lib):
     assert lib.moe_router_wgrad_static(8, 128, 300, fake, fake, fake, None) == -1    # E > 256
     assert lib.moe_router_wgrad_static(8, 4096, 128, fake, fake, fake, None) == -2   # beyond the built-in scratch
     assert lib.moe_selftest_timeout(None, fake, None) == -1
+
+
+def test_context_binds_to_a_device_only_when_work_is_launched(lib):
+    """The per-device state of a context (SM count, tensor-map encoder, the kernels' shared-memory attributes) is
+    set up by the first call that launches work and belongs to the device current then.  Without a device the call
+    fails with a CUDA error and the context stays unbound; argument errors never bind it."""
+    import torch
+    layer = binding.MoELayer(128, 8, 128, 2)
+    assert lib.moe_ctx_device(layer.h) == -1 and lib.moe_ctx_device(None) == -1
+    vp = C.c_void_p
+    fake = vp(4096)
+    assert lib.moe_forward(layer.h, -1, *([fake] * 14), fake, 1 << 30, None) == -1
+    assert lib.moe_ctx_device(layer.h) == -1
+    if not torch.cuda.is_available():
+        # valid arguments, but no device to bind to: reported as a CUDA failure before any pointer is touched
+        assert lib.moe_forward(layer.h, 8, *([fake] * 14), fake, 1 << 30, None) == -4
+        assert lib.moe_ctx_device(layer.h) == -1
+    assert lib.moe_kernel_launches() >= 0

@@ -389,19 +389,66 @@ def test_expert_lora_against_the_oracle(T, d, E, k, f, rank, seed):
 
 
 def test_bounded_wait_reports_timeout_and_context_survives():
-    """A device-side wait that can never complete gives up, the status word says so, and the same context and
-    workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
+    """A device-side wait that can never complete gives up and the status word says so.  The word is sticky: a forward
+    and a backward enqueued after the failure do not erase it, the poll that reports it acknowledges it, and the same
+    context and workspace keep working afterwards (no fault, no hang: the wait is bounded by construction)."""
     from paper_2608_00916_b200.binding import MoEError
     inp = synth.make_inputs(synth.MoEShape(300, 128, 8, 2, 128), 25)
     ofw, obw = oracle_run(inp, 2, 0.0)
     r = Run(inp, 2)
     r.forward()  # allocates the workspace, status ok
     r.layer.selftest_timeout()
+    v = r.dev
+    r.layer.forward(v["x"], v["W_r"], v["W_gate"], v["W_up"], v["W_down"])  # neither call may clear the word
+    r.layer.backward(v["dy"], 0.0)
     with pytest.raises(MoEError, match="bounded device-side wait"):
         r.layer.poll()
-    fw = r.forward()  # clears the status word and runs normally
+    r.layer.poll()  # reported once; acknowledged
+    fw = r.forward()
     check_routing(fw, ofw)
     assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+    # a workspace the library has never seen (arbitrary bytes in its status block) starts clean
+    r2 = Run(inp, 2)
+    r2.layer._ensure_ws(300)
+    r2.layer.ws.fill_(0x5A)
+    r2.layer.poll()  # nothing ran on it yet: ok
+    fw2 = r2.forward()
+    check_routing(fw2, ofw)
+    r2.layer.selftest_timeout()
+    with pytest.raises(MoEError, match="bounded device-side wait"):
+        r2.layer.poll()
+
+
+def test_pipelined_host_steps_report_a_recorded_timeout():
+    """moe_step_host_end reads the status word together with the slot's results: a failure recorded before (or during)
+    the step comes back from end() once, and the following steps run clean."""
+    from paper_2608_00916_b200.binding import MoEError
+    shape = synth.MoEShape(256, 128, 8, 2, 128)
+    inp = synth.make_inputs(shape, 27)
+    layer = MoELayer(shape.d, shape.E, shape.f, shape.k)
+    T = shape.T
+    host = {n: torch.from_numpy(inp[n].view(np.int16)).pin_memory() for n in ("x", "dy", "W_r", "W_gate", "W_up", "W_down")}
+    host["y"] = torch.empty(T, shape.d, dtype=torch.int16).pin_memory()
+    host["dx"] = torch.empty(T, shape.d, dtype=torch.int16).pin_memory()
+    host["aux"] = torch.empty(1, dtype=torch.float32).pin_memory()
+    host["dW_r"] = torch.empty(shape.d, shape.E, dtype=torch.float32).pin_memory()
+    for n in ("dW_gate", "dW_up", "dW_down"):
+        host[n] = torch.empty(inp["W_gate"].size, dtype=torch.int16).pin_memory()
+    dev_buf = torch.empty(layer.e2e_device_bytes(T), dtype=torch.uint8, device="cuda")
+    layer.step_host(T, dev_buf, host, 0.01, copy_weights=True)
+    y_ok = host["y"].clone()
+    # the workspace of the host steps lives inside dev_buf: record a timeout in ITS status word
+    ws_off = layer.e2e_workspace_offset(T)
+    layer.ws, layer.T = dev_buf[ws_off:], T
+    layer.selftest_timeout()
+    layer.step_host_begin(0, T, dev_buf, host, 0.01)
+    with pytest.raises(MoEError, match="bounded device-side wait"):
+        layer.step_host_end(0)
+    host["y"].zero_()
+    layer.step_host_begin(1, T, dev_buf, host, 0.01)
+    layer.step_host_end(1)  # clean again
+    assert torch.equal(host["y"], y_ok)
+    layer.poll()
 
 
 def test_forward_backward_replay_from_a_cuda_graph():

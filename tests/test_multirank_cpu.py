@@ -20,7 +20,10 @@ def _worker(rank, world, port, q):
     pdist.init(world, rank, backend="gloo")
     shape = synth.MoEShape(64, 64, 8, 2, 64)
     base = synth.make_inputs(shape, 500, threads=1)          # weights: same seed on every rank
-    mine = synth.make_inputs(shape, pdist.shard_seed(500, rank), threads=1)
+    # the rank's own tokens, guarded against the router weight all ranks share
+    mine = base if rank == 0 else synth.make_tokens(shape, pdist.shard_seed(500, rank), base["W_r"], base["b_r"], threads=1)
+    gaps = synth._gap_violations(synth._guard_logits(mine["x"], base["W_r"], base["b_r"]), shape.k)
+    assert not gaps.any()
     fw = orc.forward(mine["x"], base["W_r"], base["W_gate"], base["W_up"], base["W_down"], 2)
     pdist.barrier()
     ms = 10.0 * (rank + 1)  # pretend rank r took 10 (r + 1) ms
@@ -58,7 +61,7 @@ def _reduce_worker(rank, world, port, q):
     pdist.init(world, rank, backend="gloo")
     shape = synth.MoEShape(48, 64, 6, 2, 64)
     base = synth.make_inputs(shape, 700, threads=1)
-    mine = synth.make_inputs(shape, pdist.shard_seed(700, rank), threads=1)
+    mine = base if rank == 0 else synth.make_tokens(shape, pdist.shard_seed(700, rank), base["W_r"], base["b_r"], threads=1)
     fw = orc.forward(mine["x"], base["W_r"], base["W_gate"], base["W_up"], base["W_down"], 2)
     bw = orc.backward(fw, mine["dy"], 0.0, mine["x"], base["W_r"], base["W_gate"], base["W_up"], base["W_down"])
     acc = [torch.from_numpy(bw[n].astype(np.float32)).clone() for n in ("dW_gate", "dW_up", "dW_down", "dW_r")]
@@ -91,8 +94,30 @@ def test_gradient_all_reduce_over_two_gloo_ranks():
         assert np.abs(l0 - l1).max() > 0
 
 
-def test_token_split_is_balanced():
+def test_rank_environment_of_the_launcher():
+    """What `bench.py --gpus N` hands to each rank it starts: rank, local rank, world size, loopback rendezvous, and
+    NCCL's communicator log line left on unless the caller chose otherwise.  No GPU is touched."""
     from paper_2608_00916_b200 import dist as pdist
-    for total, world in ((16384, 8), (8191, 4), (5, 8)):
-        parts = [pdist.tokens_per_rank(total, world, r) for r in range(world)]
-        assert sum(parts) == total and max(parts) - min(parts) <= 1
+    port = pdist.free_port()
+    assert 1024 < port < 65536
+    for world in (2, 8):
+        envs = [pdist.rank_environment(r, world, port, base_env={"PATH": "/bin"}) for r in range(world)]
+        assert [e["RANK"] for e in envs] == [str(r) for r in range(world)]
+        assert [e["LOCAL_RANK"] for e in envs] == [str(r) for r in range(world)]
+        assert all(e["WORLD_SIZE"] == str(world) and e["MASTER_ADDR"] == "127.0.0.1" and e["MASTER_PORT"] == str(port)
+                   for e in envs)
+        assert all(e["NCCL_DEBUG"] == "INFO" and e["PATH"] == "/bin" for e in envs)
+    assert pdist.rank_environment(0, 2, port, base_env={"NCCL_DEBUG": "WARN"})["NCCL_DEBUG"] == "WARN"
+
+
+def test_launcher_starts_gloo_ranks(tmp_path):
+    """The launcher behind `bench.py --gpus N` starts N processes that find each other: here two CPU ranks that
+    initialise gloo from the environment they were given and agree on the max-over-ranks time."""
+    from paper_2608_00916_b200 import dist as pdist
+    script = os.path.join(ROOT, "tests", "rank_probe.py")
+    rc = pdist.launch_ranks(2, script, [str(tmp_path)], timeout=180)
+    assert rc == 0
+    got = sorted((tmp_path / f"rank{r}.txt").read_text() for r in range(2))
+    assert got == ["0 2 0 20.0", "1 2 1 20.0"]
+    # a rank that fails makes the launcher report it
+    assert pdist.launch_ranks(2, script, [str(tmp_path), "fail-on-1"], timeout=180) != 0

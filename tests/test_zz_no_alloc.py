@@ -43,6 +43,20 @@ def test_static_scratch_entry_matches_backward_twice_in_a_row():
     assert torch.equal(again, got)
 
 
+def test_static_scratch_entry_at_its_size_limit_and_smallest_expert_count():
+    """d * E exactly at the limit with the widest register tile (E = 256), then the narrowest (E = 8), back to back on
+    the shared scratch; reference: the same contraction in float64 on the host."""
+    assert 1024 * 256 == binding.STATIC_MAX_DE
+    g = torch.Generator(device="cpu").manual_seed(7)
+    for T, d, E in ((700, 1024, 256), (257, 1024, 8)):
+        x = torch.randn(T, d, generator=g).to(torch.bfloat16).cuda()
+        dl = (0.01 * torch.randn(T, E, generator=g)).cuda()
+        got = binding.router_wgrad_static(x, dl)
+        torch.cuda.synchronize()
+        ref = x.double().cpu().numpy().T @ dl.double().cpu().numpy()
+        assert rel_fro(got.cpu().numpy(), ref) <= 1e-5, (T, d, E)
+
+
 def test_static_scratch_entry_refuses_shapes_beyond_its_scratch():
     lib = binding.load_library()
     d, E = 4096, 128  # d * E = 524288 > MOE_STATIC_MAX_DE
