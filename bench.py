@@ -64,7 +64,8 @@ def stage_work(shape: synth.MoEShape):
         "wgrad_gateup": ("tensor", 4 * R * d * f),
         "router_bwd": ("hbm", 8 * T * E + 12 * R),
         "dW_r": ("hbm", 2 * T * d + 4 * T * E + 4 * d * E),
-        "unpermute_bwd": ("hbm", 2 * R * d + 2 * T * d + 4 * T * E),
+        "unpermute_bwd": ("hbm", 2 * R * d + 2 * T * d + 2 * T * d),
+        "dx_router_term": ("hbm", 4 * T * E + 2 * T * d + 2 * d * E),
     }
 
 

@@ -61,6 +61,13 @@ typedef struct {
  * comparison measurements). */
 #define MOE_FLAG_CTA_PAIR_TILES 1
 #define MOE_FLAG_SINGLE_CTA_TILES 2
+/* Row GEMMs run every complete pair of 128-row blocks of an expert on a CTA pair and the leftover block of an odd
+ * count on a one-CTA tile (two launches, no half-empty pairs); weight gradients run on pairs. */
+#define MOE_FLAG_HYBRID_TILES 16
+/* moe_backward normally runs the router's gradient chain (dl, dW_r, db_r, the router term of dx) on a second stream of
+ * the context, forked and joined inside the call (the caller's stream sees one ordered call; the pattern is legal
+ * inside a stream capture).  This flag keeps everything on the caller's stream. */
+#define MOE_FLAG_NO_SIDE_STREAM 8
 
 typedef struct moe_ctx moe_ctx; /* opaque, lives in host memory */
 
@@ -123,7 +130,9 @@ MOE_API moe_status moe_selftest_timeout(moe_ctx* ctx, void* workspace, void* cud
  * of them if there were more), stores that number of pairs in *steps, and starts a new window.
  * Stage order: 0 router, 1 permute (histogram, scan, scatter, gather), 2 gate/up GEMM + SwiGLU,
  * 3 down GEMM, 4 combine, 5 combine-bwd (gather of dy rows), 6 dgrad-down + SwiGLU-bwd (+ dg), 7 wgrad-down, 8 dgrad gate/up,
- * 9 wgrad gate/up, 10 router-bwd (dl), 11 dW_r, 12 unpermute-bwd (dx), 13..15 unused. */
+ * 9 wgrad gate/up, 10 router-bwd (dl), 11 dW_r, 12 unpermute-bwd (dx), 13 router term of dx, 14..15 unused.
+ * Stages 10, 11 and 13 run on the context's second stream beside stages 7..9 (unless MOE_FLAG_NO_SIDE_STREAM), so the
+ * stage times then add up to more than the step. */
 #define MOE_PROF_RING 64
 MOE_API moe_status moe_set_profiling(moe_ctx* ctx, int enable);
 MOE_API moe_status moe_stage_times(moe_ctx* ctx, float* ms /* host */, int32_t* steps /* host */);
@@ -214,6 +223,68 @@ MOE_API moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, floa
                                      const uint16_t* B2, uint16_t* dx, float* dW_r, uint16_t* dA1, uint16_t* dB1_gate,
                                      uint16_t* dB1_up, uint16_t* dA2, uint16_t* dB2, void* workspace,
                                      size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------------------------------
+ * Expert parallelism (EP > 1).  The paper trains its MoE reranker with the experts spread over an EP group (Section
+ * "Expert-Parallel MoE Training": EP = 16; "MoE layers dispatch routed tokens only among the ranks within an EP
+ * group").  Rank r of `world` ranks owns the experts [r E/world, (r+1) E/world), keeps its own T tokens, and passes
+ * only its shard of the expert weights.  Token rows reach the owning rank, and expert outputs come back, through
+ * plain stores / loads of this library's kernels into PEER-MAPPED buffers (NVLink): every rank passes the table
+ * peer_own_ws[world] of all ranks' owner workspaces as they are mapped into its own address space (entry `rank` is
+ * its own; on one GPU the entries are ordinary device pointers).  The caller provides the two group operations the
+ * library does not do itself: the all-gather of the per-rank expert counts after moe_ep_route, and a barrier of the
+ * group between any two phases, because each phase reads what the previous one wrote on other ranks:
+ *
+ *   forward :  moe_ep_route | all-gather counts | moe_ep_plan | barrier | moe_ep_dispatch(x) | barrier |
+ *              moe_ep_expert_forward | barrier | moe_ep_combine
+ *   backward:  moe_ep_dispatch(dy, backward = 1) | barrier | moe_ep_expert_backward | barrier | moe_ep_router_backward
+ *
+ * Results are those of the one-GPU layer applied to the concatenation of the ranks' batches in rank order (same row
+ * order inside every expert), except that aux_loss, its gradient and dW_r / db_r are per rank, over the rank's own
+ * tokens (each rank is also a data-parallel rank for the router weight; sum dW_r over the group as for any replicated
+ * parameter).  Requirements: E a multiple of `world` and of 8, world <= MOE_EP_MAX_RANKS.
+ *
+ * Workspaces (caller-allocated): the SENDER workspace (moe_ep_send_workspace_bytes(ctx, T): routing state of the
+ * rank's tokens) and the OWNER workspace (moe_ep_own_workspace_bytes(ctx): tables and row buffers of the owned
+ * experts, sized for rows_cap received rows - the caller's bound on sum over ranks of rows routed to this rank, at
+ * most sum_r T_r * min(top_k, E/world); it is the owner workspace that peers map). */
+#define MOE_EP_MAX_RANKS 16
+MOE_API moe_status moe_ep_create(const moe_config* cfg /* host */, int32_t world, int32_t rank, int64_t rows_cap,
+                                 moe_ctx** out /* host */);
+MOE_API size_t moe_ep_send_workspace_bytes(const moe_ctx* ctx, int64_t T);
+MOE_API size_t moe_ep_own_workspace_bytes(const moe_ctx* ctx);
+/* Named internal buffers, for tests: own_side = 0: sender workspace ("counts" "logits" "idx" "gates" "inv" "dg" "dl"
+ * "ep_dest" "status"); own_side = 1: owner workspace (names of moe_workspace_find, E/world experts). */
+MOE_API moe_status moe_ep_workspace_find(const moe_ctx* ctx, int64_t T, int own_side, const char* name /* host */,
+                                         size_t* offset /* host */, size_t* bytes /* host */);
+/* Router over the rank's tokens: x [T,d], W_r [d,E] (all E experts), b_r [E] or NULL -> topk_idx [T,k], topk_w [T,k],
+ * counts_local [E] (rows this rank routes to each expert; the caller all-gathers these), aux_loss [1] (local). */
+MOE_API moe_status moe_ep_route(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
+                                int32_t* topk_idx, float* topk_w, int32_t* counts_local, float* aux_loss,
+                                void* send_ws, size_t send_ws_bytes, void* cuda_stream);
+/* all_counts [world, E] int32 (device; row r = counts_local of rank r).  Places this rank's rows inside the owners'
+ * buffers, builds the tile tables of the owned experts in own_ws and clears what must start at zero there. */
+MOE_API moe_status moe_ep_plan(moe_ctx* ctx, int64_t T, const int32_t* all_counts, void* send_ws, size_t send_ws_bytes,
+                               void* own_ws, size_t own_ws_bytes, void* cuda_stream);
+/* Writes the rank's token rows (src = x with backward = 0, src = dy with backward = 1; [T,d] bf16) into the owners'
+ * row buffers; the forward call also stores each row's gate beside it. */
+MOE_API moe_status moe_ep_dispatch(moe_ctx* ctx, int64_t T, const uint16_t* src, int backward,
+                                   void* const* peer_own_ws /* host array of device pointers */, void* send_ws,
+                                   size_t send_ws_bytes, void* cuda_stream);
+/* Expert GEMMs over the owned experts: W_gate, W_up [E/world,d,f], W_down [E/world,f,d] are the rank's shards. */
+MOE_API moe_status moe_ep_expert_forward(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up,
+                                         const uint16_t* W_down, void* own_ws, size_t own_ws_bytes, void* cuda_stream);
+/* y [T,d] of the rank's tokens from the owners' output rows. */
+MOE_API moe_status moe_ep_combine(moe_ctx* ctx, int64_t T, void* const* peer_own_ws /* host */, const void* send_ws,
+                                  size_t send_ws_bytes, uint16_t* y, void* cuda_stream);
+/* Backward GEMMs over the owned experts; dW_gate, dW_up [E/world,d,f], dW_down [E/world,f,d] bf16, overwritten. */
+MOE_API moe_status moe_ep_expert_backward(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up,
+                                          const uint16_t* W_down, uint16_t* dW_gate, uint16_t* dW_up,
+                                          uint16_t* dW_down, void* own_ws, size_t own_ws_bytes, void* cuda_stream);
+/* Router gradient and dx of the rank's tokens: dx [T,d] bf16, dW_r [d,E] fp32, db_r [E] fp32 or NULL (overwritten). */
+MOE_API moe_status moe_ep_router_backward(moe_ctx* ctx, int64_t T, float d_aux, const uint16_t* x, const uint16_t* W_r,
+                                          void* const* peer_own_ws /* host */, void* send_ws, size_t send_ws_bytes,
+                                          uint16_t* dx, float* dW_r, float* db_r, void* cuda_stream);
 
 /* Host-buffer convenience used for end-to-end timing: every tensor argument is a HOST pointer (pinned
  * memory recommended); the call copies inputs to the device buffers of `dev` (a device scratch of

@@ -11,16 +11,21 @@ LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
 NUM_STAGES = 16
 FLAG_CTA_PAIR_TILES = 1    # MOE_FLAG_CTA_PAIR_TILES of include/moe.h
 FLAG_SINGLE_CTA_TILES = 2  # MOE_FLAG_SINGLE_CTA_TILES
+FLAG_NO_SIDE_STREAM = 8    # MOE_FLAG_NO_SIDE_STREAM
+FLAG_HYBRID_TILES = 16     # MOE_FLAG_HYBRID_TILES
 STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine", "combine_bwd",
                "dgrad_down_swiglu_bwd", "wgrad_down", "dgrad_gateup", "wgrad_gateup", "router_bwd", "dW_r",
-               "unpermute_bwd"]
+               "unpermute_bwd", "dx_router_term"]
 EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_find", "moe_status_string",
            "moe_poll_status", "moe_set_profiling", "moe_stage_times", "moe_forward", "moe_backward",
            "moe_e2e_device_bytes", "moe_step_host", "moe_router_wgrad_static", "moe_selftest_timeout",
            "moe_forward_inference", "moe_inference_workspace_bytes", "moe_backward_accumulate",
            "moe_lora_workspace_bytes", "moe_lora_forward", "moe_lora_backward",
            "moe_step_host_begin", "moe_step_host_end", "moe_kernel_launches", "moe_ctx_device",
-           "moe_e2e_workspace_offset"]
+           "moe_e2e_workspace_offset", "moe_ep_create", "moe_ep_send_workspace_bytes", "moe_ep_own_workspace_bytes",
+           "moe_ep_workspace_find", "moe_ep_route", "moe_ep_plan", "moe_ep_dispatch", "moe_ep_expert_forward",
+           "moe_ep_combine", "moe_ep_expert_backward", "moe_ep_router_backward"]
+EP_MAX_RANKS = 16  # MOE_EP_MAX_RANKS of include/moe.h
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
 
@@ -90,6 +95,28 @@ def load_library() -> C.CDLL:
     lib.moe_kernel_launches.restype = C.c_longlong
     lib.moe_ctx_device.argtypes = [vp]
     lib.moe_ctx_device.restype = C.c_int
+    lib.moe_ep_create.argtypes = [C.POINTER(MoEConfig), C.c_int32, C.c_int32, i64, C.POINTER(vp)]
+    lib.moe_ep_create.restype = C.c_int
+    lib.moe_ep_send_workspace_bytes.argtypes = [vp, i64]
+    lib.moe_ep_send_workspace_bytes.restype = sz
+    lib.moe_ep_own_workspace_bytes.argtypes = [vp]
+    lib.moe_ep_own_workspace_bytes.restype = sz
+    lib.moe_ep_workspace_find.argtypes = [vp, i64, C.c_int, C.c_char_p, C.POINTER(sz), C.POINTER(sz)]
+    lib.moe_ep_workspace_find.restype = C.c_int
+    lib.moe_ep_route.argtypes = [vp, i64] + [vp] * 7 + [vp, sz, vp]
+    lib.moe_ep_route.restype = C.c_int
+    lib.moe_ep_plan.argtypes = [vp, i64, vp, vp, sz, vp, sz, vp]
+    lib.moe_ep_plan.restype = C.c_int
+    lib.moe_ep_dispatch.argtypes = [vp, i64, vp, C.c_int, C.POINTER(vp), vp, sz, vp]
+    lib.moe_ep_dispatch.restype = C.c_int
+    lib.moe_ep_expert_forward.argtypes = [vp, vp, vp, vp, vp, sz, vp]
+    lib.moe_ep_expert_forward.restype = C.c_int
+    lib.moe_ep_combine.argtypes = [vp, i64, C.POINTER(vp), vp, sz, vp, vp]
+    lib.moe_ep_combine.restype = C.c_int
+    lib.moe_ep_expert_backward.argtypes = [vp] + [vp] * 6 + [vp, sz, vp]
+    lib.moe_ep_expert_backward.restype = C.c_int
+    lib.moe_ep_router_backward.argtypes = [vp, i64, C.c_float, vp, vp, C.POINTER(vp), vp, sz, vp, vp, vp, vp]
+    lib.moe_ep_router_backward.restype = C.c_int
     lib.moe_selftest_timeout.argtypes = [vp, vp, vp]
     lib.moe_selftest_timeout.restype = C.c_int
     lib.moe_router_wgrad_static.argtypes = [i64, C.c_int32, C.c_int32, vp, vp, vp, vp]

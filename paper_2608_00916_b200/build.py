@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoe_b200.so")
-SOURCES = ["api.cu", "route.cu", "combine.cu", "gemm.cu", "gemm2.cu", "noalloc.cu"]
-HEADERS = ["common.cuh", "ptx.cuh", "gemm_common.cuh", os.path.join("..", "..", "include", "moe.h")]
+SOURCES = ["api.cu", "route.cu", "combine.cu", "gemm.cu", "gemm2.cu", "noalloc.cu", "ep.cu"]
+HEADERS = ["common.cuh", "ptx.cuh", "gemm_common.cuh", "tables.cuh", os.path.join("..", "..", "include", "moe.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -14,12 +14,13 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static std::atomic<long long> g_kernel_launches{0};
 void note_launch(int n) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
 
-WsLayout make_layout(const Shape& s, int64_t T) {
+WsLayout make_layout(const Shape& s, int64_t T, bool row_buffers) {
   WsLayout L;
   memset(&L, 0, sizeof(L));
   const int64_t R = T * s.k;
   L.max_m_tiles = (R + ROW_PAD - 1) / ROW_PAD + s.E;
   L.rows_max = L.max_m_tiles * ROW_PAD;
+  L.rows_alloc = row_buffers ? L.rows_max : 0;
   L.tok_tiles = (T + TOK_TILE - 1) / TOK_TILE;
   L.router_blocks = (T + ROUTER_TOK - 1) / ROUTER_TOK;
   size_t off = 0;
@@ -34,9 +35,11 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.offsets = take(sizeof(int32_t) * (s.E + 1));
   L.pad_offsets = take(sizeof(int32_t) * (s.E + 1));
   L.expert_order = take(sizeof(int32_t) * s.E);
-  L.sched = take(sizeof(int32_t) * 4);
+  L.sched = take(sizeof(int32_t) * 8);
   L.tile_expert = take(sizeof(int32_t) * L.max_m_tiles);
   L.pair_tab = take(sizeof(int32_t) * 4 * L.max_m_tiles);
+  L.fpair_tab = take(sizeof(int32_t) * 4 * L.max_m_tiles);
+  L.single_tab = take(sizeof(int32_t) * s.E);
   L.tile_counts = take(sizeof(int32_t) * (L.tok_tiles + 1) * s.E);
   // rows: one per SIMT router block, or four (one per epilogue warp) per 128-token tile of the tensor-core router
   L.psum_part = take(sizeof(float) * (L.router_blocks + 4 * ((T + 127) / 128) + 1) * s.E);
@@ -45,15 +48,16 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.idx = take(sizeof(int32_t) * R);
   L.gates = take(sizeof(float) * R);
   L.inv = take(sizeof(int32_t) * R);
-  L.row_gate = take(sizeof(float) * L.rows_max);
-  const size_t rows_d = sizeof(uint16_t) * L.rows_max * s.d, rows_f = sizeof(uint16_t) * L.rows_max * s.f;
+  L.ep_dest = take(sizeof(int32_t) * s.E);
+  L.row_gate = take(sizeof(float) * L.rows_alloc);
+  const size_t rows_d = sizeof(uint16_t) * L.rows_alloc * s.d, rows_f = sizeof(uint16_t) * L.rows_alloc * s.f;
   L.xp = take(rows_d);
   L.act = take(rows_f);
   L.o = take(rows_d);
   L.infer_total = off;  // everything above is all a forward-only call touches
   L.hg = take(rows_f);
   L.hu = take(rows_f);
-  L.dg_part = take(sizeof(float) * 2 * ((s.f + 255) / 256) * L.rows_max);
+  L.dg_part = take(sizeof(float) * 2 * ((s.f + 255) / 256) * L.rows_alloc);
   L.dg = take(sizeof(float) * R);
   L.dl = take(sizeof(float) * T * s.E);
   L.dl_hi = take(sizeof(uint16_t) * (T * s.E + 64));
@@ -64,7 +68,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
   L.dxp = take(rows_d);
   L.dxr = take(sizeof(uint16_t) * T * s.d);
   L.total = off;
-  const size_t rows64 = sizeof(uint16_t) * L.rows_max * 64;
+  const size_t rows64 = sizeof(uint16_t) * L.rows_alloc * 64;
   L.lora_u = take(rows64);
   L.lora_v = take(rows64);
   L.lora_w = take(rows64);
@@ -75,7 +79,7 @@ WsLayout make_layout(const Shape& s, int64_t T) {
 
 // The first call that needs the device binds the context to the current one (SM count, tensor-map encoder, the
 // per-device kernel attributes); every later call must come with the same device current.
-static moe_status ensure_device(moe_ctx_impl* c) {
+moe_status ensure_device(moe_ctx_impl* c) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
   if (c->encode_fn) return dev == c->device ? MOE_OK : MOE_ERR_INVALID_ARG;
@@ -91,6 +95,13 @@ static moe_status ensure_device(moe_ctx_impl* c) {
     return MOE_ERR_CUDA;
   c->encode_fn = fn;
   c->gemm_timers = getenv("MOE_GEMM_TIMERS") != nullptr;
+  if (c->use_side_stream) {
+    if (cudaStreamCreateWithFlags(&c->s_side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    c->side_created = 1;
+  }
   memset(c->attr_done, 0, sizeof(c->attr_done));
   return MOE_OK;
 }
@@ -138,7 +149,10 @@ moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
   memset(c, 0, sizeof(*c));
   c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
   c->device = -1;  // bound by the first call that launches work
-  c->tile_mode = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 1 : ((cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 2 : 0);
+  c->use_side_stream = (cfg->flags & MOE_FLAG_NO_SIDE_STREAM) ? 0 : 1;
+  c->tile_mode = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 1
+                 : (cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 2
+                 : (cfg->flags & MOE_FLAG_HYBRID_TILES) ? 3 : 0;
   *out = reinterpret_cast<moe_ctx*>(c);
   return MOE_OK;
 }
@@ -152,6 +166,12 @@ void moe_destroy(moe_ctx* ctx) {
         cudaEventDestroy(c->ev[r][i][0]);
         cudaEventDestroy(c->ev[r][i][1]);
       }
+  if (c->own) moe_destroy(reinterpret_cast<moe_ctx*>(c->own));
+  if (c->side_created) {
+    cudaStreamDestroy(c->s_side);
+    cudaEventDestroy(c->ev_fork);
+    cudaEventDestroy(c->ev_join);
+  }
   if (c->e2e_created) {
     cudaStreamDestroy(c->s_in);
     cudaStreamDestroy(c->s_out);
@@ -457,15 +477,53 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     StageTimer tm(c, st, 5);
     launch_gather_rows(s, T, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st);
   }
+  // The router's gradient chain (dl, dW_r, db_r and the router term of dx) needs only the dg partials that the
+  // dgrad-down GEMM leaves behind.  It is small and latency-bound, so it runs on a second stream of the context, forked
+  // after that GEMM and joined before the final unpermute, where it fills the tails of the three big GEMMs instead of
+  // standing in line behind them.  Without tokens, or with MOE_FLAG_NO_SIDE_STREAM, it runs in line.
+  bool forked = false;
+  auto router_chain = [&]() -> moe_status {
+    cudaStream_t rs = st;
+    if (T > 0 && c->use_side_stream) {
+      if (cudaEventRecord(c->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(c->s_side, c->ev_fork, 0) != cudaSuccess)
+        return MOE_ERR_CUDA;
+      rs = c->s_side;
+      forked = true;
+    }
+    {
+      StageTimer tm(c, rs, 10);
+      launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
+                        gates, reinterpret_cast<const float*>(ws + L.dg_part), 2 * ((s.f + 255) / 256), L.rows_max, inv,
+                        reinterpret_cast<float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts), d_aux, dl,
+                        reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo), rs);
+    }
+    {
+      StageTimer tm(c, rs, 11);
+      if (tc_router && T > 0) {
+        const moe_status r2 = launch_grouped_gemm(c, GEMM_DWR, T, L, ws, io, rs);
+        if (r2 != MOE_OK) return r2;
+      }
+      launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, tc_router && T > 0, rs, accumulate);
+    }
+    if (tc_router && T > 0) {
+      StageTimer tm(c, rs, 13);
+      const moe_status r2 = launch_grouped_gemm(c, GEMM_DX, T, L, ws, io, rs);
+      if (r2 != MOE_OK) return r2;
+    }
+    if (forked && cudaEventRecord(c->ev_join, c->s_side) != cudaSuccess) return MOE_ERR_CUDA;
+    return MOE_OK;
+  };
   if (lora) {
     // base weights frozen: no dW_gate / dW_up / dW_down; the adapter gradients come from skinny GEMMs
     const LoraOp seq[4][2] = {{LORA_W, LORA_B2}, {LORA_DB2, LORA_DA2}, {LORA_Z, LORA_B4}, {LORA_DB1, LORA_DA1}};
     for (int g = 0; g < 4 && rc == MOE_OK; ++g) {
       const bool row_ops = (g == 0 || g == 2);  // row GEMMs have no tiles without tokens; weight gradients zero-fill
-      if (row_ops && T == 0) continue;
-      StageTimer tm(c, st, 6 + g);
-      rc = launch_lora_gemm(c, seq[g][0], T, L, ws, io, *lora, st);
-      if (rc == MOE_OK) rc = launch_lora_gemm(c, seq[g][1], T, L, ws, io, *lora, st);
+      if (!(row_ops && T == 0)) {
+        StageTimer tm(c, st, 6 + g);
+        rc = launch_lora_gemm(c, seq[g][0], T, L, ws, io, *lora, st);
+        if (rc == MOE_OK) rc = launch_lora_gemm(c, seq[g][1], T, L, ws, io, *lora, st);
+      }
+      if (g == 0 && rc == MOE_OK) rc = router_chain();
     }
     if (rc != MOE_OK) return rc;
   } else {
@@ -473,6 +531,8 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
       StageTimer tm(c, st, 6);
       rc = launch_grouped_gemm(c, GEMM_B2, T, L, ws, io, st);
     }
+    if (rc != MOE_OK) return rc;
+    rc = router_chain();
     if (rc != MOE_OK) return rc;
     {
       StageTimer tm(c, st, 7);
@@ -490,26 +550,10 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     }
     if (rc != MOE_OK) return rc;
   }
-  {
-    StageTimer tm(c, st, 10);
-    launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
-                      gates, reinterpret_cast<const float*>(ws + L.dg_part), 2 * ((s.f + 255) / 256), L.rows_max, inv,
-                      reinterpret_cast<float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts), d_aux, dl,
-                      reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo), st);
-  }
-  {
-    StageTimer tm(c, st, 11);
-    if (tc_router && T > 0) {
-      rc = launch_grouped_gemm(c, GEMM_DWR, T, L, ws, io, st);
-      if (rc != MOE_OK) return rc;
-    }
-    launch_dwr(s, T, x, dl, reinterpret_cast<float*>(ws + L.dwr_part), dW_r, db_r, tc_router && T > 0, st, accumulate);
-  }
+  if (forked && cudaStreamWaitEvent(st, c->ev_join, 0) != cudaSuccess) return MOE_ERR_CUDA;
   {
     StageTimer tm(c, st, 12);
     if (tc_router && T > 0) {
-      rc = launch_grouped_gemm(c, GEMM_DX, T, L, ws, io, st);
-      if (rc != MOE_OK) return rc;
       launch_unpermute_sum(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv,
                            reinterpret_cast<const uint16_t*>(ws + L.dxr), dx, st);
     } else {

@@ -102,9 +102,13 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
   if (lane < k) {
     g = gates[t * k + lane];
     ej = idx[t * k + lane];
-    const int r = inv[t * k + lane];
-    for (int nt = 0; nt < dg_tiles; ++nt) dgj += dg_part[nt * rows_max + r];
-    dg[t * k + lane] = dgj;
+    if (dg_tiles > 0) {
+      const int r = inv[t * k + lane];
+      for (int nt = 0; nt < dg_tiles; ++nt) dgj += dg_part[nt * rows_max + r];
+      dg[t * k + lane] = dgj;
+    } else {
+      dgj = dg[t * k + lane];  // gathered by the caller (expert-parallel path: the partials live on the owner ranks)
+    }
   }
   float inner = g * dgj;
 #pragma unroll

@@ -38,9 +38,12 @@ struct WsLayout {
   size_t offsets;      // int32[E+1]  exclusive scan of counts (canonical, unpadded)
   size_t pad_offsets;  // int32[E+1]  exclusive scan of counts rounded up to ROW_PAD
   size_t expert_order; // int32[E]    experts sorted by row count, largest first
-  size_t sched;        // int32[4]    [0] number of 128-row tiles, [1] padded row total, [2] number of block pairs
+  size_t sched;        // int32[8]    [0] number of 128-row tiles, [1] padded row total, [2] number of block pairs (odd
+                       //             blocks included as half-empty pairs), [3] full pairs, [4] leftover single blocks
   size_t tile_expert;  // int32[max_m_tiles] expert of every 128-row tile
   size_t pair_tab;     // int32[4 * max_m_tiles] pairs of 128-row blocks of one expert: {expert, first row, blocks, 0}
+  size_t fpair_tab;    // int32[4 * max_m_tiles] full pairs only (both blocks exist)
+  size_t single_tab;   // int32[E] tile index of the last block of every expert with an odd number of blocks
   size_t tile_counts;  // int32[tok_tiles * E] per token-tile histogram, turned into a prefix along tiles
   size_t psum_part;    // float[router_blocks * E] per-block column sums of p
   size_t psum;         // float[E]
@@ -66,20 +69,29 @@ struct WsLayout {
   // z = s (dhg B1g^T + dhu B1u^T), bf16 [rows_max, 64], columns beyond the rank are zero
   size_t lora_u, lora_v, lora_w, lora_z;
   size_t lora_total;
+  size_t ep_dest;      // int32[E] expert-parallel sender: first row, in the owner's buffers, of this rank's rows of expert e
+  int64_t rows_alloc;  // rows the row buffers were actually sized for (0 in a layout without row buffers)
   int64_t rows_max;    // upper bound of the padded row total for T tokens
   int64_t max_m_tiles;
   int64_t tok_tiles;
   int64_t router_blocks;
 };
 
-WsLayout make_layout(const Shape& s, int64_t T);
+// row_buffers = false: the layout of a rank that only routes and combines (expert-parallel sender side): the
+// expert-major row buffers and everything sized by their row count are left out
+WsLayout make_layout(const Shape& s, int64_t T, bool row_buffers = true);
 
 struct moe_ctx_impl {
   Shape s;
   int sm_count;
   int device;
   void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
-  int tile_mode;    // 0: choose per GEMM (see use_pair_tiles), 1: always CTA pairs, 2: always one-CTA tiles
+  int use_side_stream;  // backward runs the router's gradient chain on s_side, beside the big GEMMs
+  int side_created;
+  cudaStream_t s_side;
+  cudaEvent_t ev_fork, ev_join;
+  int tile_mode;    // 0: choose per GEMM, 1: always CTA pairs (odd blocks as half-empty pairs), 2: always one-CTA tiles,
+                    // 3: row GEMMs as full pairs + one-CTA tiles for the leftover blocks, weight gradients on pairs
   int gemm_timers;  // MOE_GEMM_TIMERS was set when the context first touched its device
   // cudaFuncSetAttribute (dynamic shared memory opt-in) is per device: remembered here, for the device the context is
   // bound to, per kernel family (0: one-CTA kernels, 1: CTA-pair kernels) and GEMM kind
@@ -98,8 +110,15 @@ struct moe_ctx_impl {
   int32_t* pipe_status[2];  // pinned host copies of the device status block, one per slot of the pipelined host steps
   int32_t* pipe_status_dev; // the status block those copies come from
   int64_t prof_read;   // pairs already reported by moe_stage_times
+  // expert parallelism (moe_ep_* calls): this rank of ep_world ranks owns experts [ep_rank * E / ep_world, ...);
+  // `own` is the context of the owner side (shape with E / ep_world experts), sized for ep_rows_cap received rows
+  int ep_world, ep_rank;
+  int64_t ep_rows_cap;
+  moe_ctx_impl* own;
 };
 
+// binds the context to the current device on first use (api.cu)
+moe_status ensure_device(moe_ctx_impl* c);
 // ---- launchers (route.cu)
 // first kernel of a forward call: zero row gates, initialise the status block of a workspace seen for the first time
 void launch_prepare(const WsLayout& L, char* ws, cudaStream_t st);
@@ -107,7 +126,7 @@ void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t*
                    const float* logits_in, float* logits, int32_t* idx, float* gates, int32_t* idx_out,
                    float* gates_out, float* logits_out, float* psum_part, cudaStream_t st);
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
-                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st);
+                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only = false);
 // ---- launchers (combine.cu)
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
                     uint16_t* y, cudaStream_t st);
@@ -119,6 +138,7 @@ void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int
                        const float* dg_part, int dg_tiles, int64_t rows_max, const int32_t* inv, float* dg,
                        const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi, uint16_t* dl_lo,
                        cudaStream_t st);
+// dg_tiles == 0: dg[t,j] has been filled by the caller (expert-parallel path) and is read instead of the partials
 // SIMT dW_r (any E) and the shared partial reduction / db_r
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
                 float* db_r, bool partials_ready, cudaStream_t st, bool accumulate = false);

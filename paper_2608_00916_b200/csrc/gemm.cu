@@ -86,9 +86,9 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
           break;
         }
         t_wait += clock64() - w0;
+        const uint32_t sA = smem_base + s * STAGE_BYTES;
         if (lane == 0) {
           mbar_expect_tx(full_bar(s), p.stage_tx);
-          const uint32_t sA = smem_base + s * STAGE_BYTES;
           issue_loads<KIND>(p, tl, kb, sA, sA + A_BYTES, full_bar(s));
         }
         __syncwarp();
@@ -300,8 +300,11 @@ static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
-moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
-                               const GemmIO& io, cudaStream_t st) {
+// One launch of an expert / router contraction.  `pair`: CTA-pair kernel.  `part`: 0 = the whole tile list; row GEMMs
+// of the mixed schedule: 1 = the pair kernel over complete pairs of row blocks only, 2 = the one-CTA kernel over the
+// leftover blocks.
+static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
+                                      const GemmIO& io, cudaStream_t st, bool pair, int part) {
   const uint16_t *W_gate = io.W_gate, *W_up = io.W_up, *W_down = io.W_down;
   uint16_t *dW_gate = io.dW_gate, *dW_up = io.dW_up, *dW_down = io.dW_down;
   const Shape& s = ctx->s;
@@ -325,17 +328,13 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.pair_tab);
   p.expert_order = reinterpret_cast<const int32_t*>(ws + L.expert_order);
   p.timers = ctx->gemm_timers ? reinterpret_cast<unsigned long long*>(ws + L.timers) + 8 * kind : nullptr;
-  // CTA pairs (256 x 256 tiles, half of B per SM) or one-CTA tiles (128 x 256)?  Pairs move a third less operand
-  // data per flop, which under the power cap is worth ~10 % on long-K tiles.  Row GEMMs pay for them with the dummy
-  // half-tile of every expert that has an odd number of 128-row blocks, so they pair only when that expected waste
-  // (64 rows per expert) stays under 3 % of the routed rows.  Weight gradients pair along the weight dimension
-  // without waste, but their K loop is the expert's row count: below ~768 rows per expert the epilogue (two coupled
-  // CTAs draining one tile) bounds them and one-CTA tiles are faster (measured: 512 rows/expert 232 vs 247 us,
-  // 1024 rows/expert 392 vs 350 us for the down-projection gradient at the Qwen3-30B-A3B shape).
-  const bool wgrad_kind = kind == GEMM_B3 || kind == GEMM_B5;
-  const double rows_per_expert = static_cast<double>(T) * s.k / E;
-  const bool pair = ctx->tile_mode == 1 ||
-                    (ctx->tile_mode == 0 && (wgrad_kind ? rows_per_expert >= 768.0 : 64.0 < 0.03 * rows_per_expert));
+  if (part == 1) {
+    p.pair_tab = reinterpret_cast<const int32_t*>(ws + L.fpair_tab);
+    p.pair_count_slot = 3;
+  } else {
+    p.pair_count_slot = 2;
+  }
+  p.tile_list = part == 2 ? reinterpret_cast<const int32_t*>(ws + L.single_tab) : nullptr;
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
   p.b_chunks = 4;
@@ -483,6 +482,36 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   }
   (void)T;
   return MOE_ERR_INVALID_ARG;
+}
+
+// Tile shape per GEMM.  A CTA pair (256 x 256 tile, each CTA staging its rows of A and half of B) moves a third
+// less operand data from L2 per flop than a one-CTA 128 x 256 tile, and the L2 -> SM feed is what limits these
+// kernels: at the Qwen3-30B-A3B shape the pair kernel needs 14 - 18 % fewer cycles per useful flop.  In the
+// power-capped steady state the step is bound by energy rather than cycles and the gain shrinks to 1 - 3 %.
+// Row GEMMs pair two 128-row blocks of ONE expert, so an expert with an odd block count has a block left over.
+// Two ways to deal with it were built and measured in steady state (Qwen shape, ms per step): half-empty pairs
+// (the empty half loads no A rows) 4.17; complete pairs on the pair kernel plus the leftover blocks on one-CTA tiles
+// in a second launch (MOE_FLAG_HYBRID_TILES) 4.22 - the second launch's ramp and ragged last round cost what the
+// empty halves cost; one-CTA tiles throughout 4.39.  Default: half-empty pairs from 512 rows per expert upwards; below
+// that there are few complete pairs and the layer is bound by streaming the weights from HBM anyway.
+// Weight gradients pair along the weight dimension without leftovers, but their K loop is the expert's row count:
+// below ~768 rows per expert the two coupled epilogues bound them and one-CTA tiles are faster.
+moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, const WsLayout& L, char* ws,
+                               const GemmIO& io, cudaStream_t st) {
+  const bool row_kind = kind == GEMM_F3 || kind == GEMM_F4 || kind == GEMM_B2 || kind == GEMM_B4;
+  const bool wgrad_kind = kind == GEMM_B3 || kind == GEMM_B5;
+  const double rows_per_expert = static_cast<double>(T) * ctx->s.k / ctx->s.E;
+  if (wgrad_kind) {
+    const bool pair = ctx->tile_mode == 1 || ctx->tile_mode == 3 || (ctx->tile_mode == 0 && rows_per_expert >= 768.0);
+    return launch_gemm_variant(ctx, kind, T, L, ws, io, st, pair, 0);
+  }
+  if (!row_kind) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 0);
+  if (ctx->tile_mode == 1) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
+  if (ctx->tile_mode == 0 && rows_per_expert >= 512.0) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
+  if (ctx->tile_mode != 3) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 0);
+  const moe_status rc = launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 1);
+  if (rc != MOE_OK) return rc;
+  return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 2);
 }
 
 // Backward operations of the expert-LoRA variant (see launch_lora_gemm below, which prepares `p`).

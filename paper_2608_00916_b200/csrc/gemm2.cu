@@ -14,26 +14,28 @@
 // leaves while its partner may still touch its shared memory, barriers or tensor memory.
 //
 // Row GEMMs pair two consecutive 128-row blocks of ONE expert; an expert with an odd number of blocks gets a pair
-// whose second half is a dummy (it loads whatever follows and stores nothing).  Weight gradients pair along M.
+// whose second half is empty: that CTA stages its half of B only, the MMA runs over whatever its A stage holds, and
+// nothing of its accumulator half is read or stored.  Weight gradients pair along M.
 #include "gemm_common.cuh"
 
 namespace moe {
 
 constexpr int STAGES2 = 6;
-constexpr int GEMM2_THREADS = 192;  // warps: 0 TMA producer, 1 MMA issuer, 2..5 epilogue
+constexpr int GEMM2_THREADS = 320;  // warps: 0 TMA producer, 1 MMA issuer, 2..9 epilogue (two per TMEM lane quadrant)
 constexpr int BH_BYTES = 128 * BK * 2;              // this CTA's half of B: 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;    // 32 KB
 constexpr size_t GEMM2_SMEM = static_cast<size_t>(STAGES2) * STAGE2_BYTES + EPI_BYTES + 1024;
 
 struct Tile2 {
   int e, row0, m0, n0, nkb;
-  bool write;
+  bool write;   // this CTA's 128 rows exist (false: the empty half of an odd expert's last pair)
+  bool full;    // both halves of the pair exist
 };
 
 template <int KIND>
 __device__ __forceinline__ int total_tiles2(const GemmParams& p) {
   if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;  // m_tiles = 256-row pairs of the output
-  return p.sched[2] * p.n_tiles;                                // sched[2] = number of row-block pairs
+  return p.sched[p.pair_count_slot] * p.n_tiles;                // number of row-block pairs in the table in use
 }
 
 template <int KIND>
@@ -49,12 +51,14 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
     tl.row0 = p.pad_offsets[tl.e];
     tl.nkb = (p.counts[tl.e] + BK - 1) / BK;  // the rest of the 128-row padding is zeros
     tl.write = true;
+    tl.full = true;
   } else {
     const int pr = t / p.n_tiles;
     const int4 info = *reinterpret_cast<const int4*>(p.pair_tab + 4 * pr);  // expert, first row, blocks (1 or 2)
     tl.e = info.x;
     tl.row0 = info.y + rank * BM;
     tl.write = rank < info.z;
+    tl.full = info.z == 2;
     tl.m0 = 0;
     tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
     tl.nkb = p.k_blocks * p.nseg;
@@ -67,21 +71,21 @@ template <int KIND>
 __device__ __forceinline__ void issue_loads2(const GemmParams& p, const Tile2& tl, int kb, int rank, uint32_t sA,
                                              uint32_t sB, uint32_t bar) {
   if (KIND == GEMM_F3) {
-    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (tl.write) tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
     const CUtensorMap* mb = rank ? &p.mapB1 : &p.mapB0;  // leader: gate columns, partner: the matching up columns
 #pragma unroll
     for (int c = 0; c < 2; ++c) tma_load_3d_pair(sB + c * CHUNK_BYTES, mb, bar, tl.n0 + c * 64, kb * BK, tl.e);
   } else if (KIND == GEMM_F4) {
-    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (tl.write) tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
 #pragma unroll
     for (int c = 0; c < 2; ++c)
       tma_load_3d_pair(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + rank * 128 + c * 64, kb * BK, tl.e);
   } else if (KIND == GEMM_B2) {
-    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    if (tl.write) tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
     tma_load_3d_pair(sB, &p.mapB0, bar, kb * BK, tl.n0 + rank * 128, tl.e);
   } else if (KIND == GEMM_B4) {
     const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
-    tma_load_2d_pair(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
+    if (tl.write) tma_load_2d_pair(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
     tma_load_3d_pair(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0 + rank * 128, tl.e);
   } else if (KIND == GEMM_B3) {
     const int row = tl.row0 + kb * BK;
@@ -126,7 +130,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);   // one commit from the leader's MMA thread
-      mbar_init(tempty_bar(a), 8);  // used in the leader only: 4 epilogue warps of each CTA
+      mbar_init(tempty_bar(a), 16);  // used in the leader only: 8 epilogue warps of each CTA
     }
     fence_mbar_init();
     tma_prefetch_desc(&p.mapA0);
@@ -162,7 +166,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
         }
         t_wait += clock64() - w0;
         if (lane == 0) {
-          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
+          // the empty half of an odd expert's last pair loads no rows of A (its accumulator half is never read)
+          if (leader) mbar_expect_tx(full_bar(s), tl.full ? 2 * STAGE2_BYTES : 2 * STAGE2_BYTES - A_BYTES);
           const uint32_t sA = smem_base + s * STAGE2_BYTES;
           issue_loads2<KIND>(p, tl, kb, rank, sA, sA + A_BYTES, mapa_shared(full_bar(s), 0));
         }
@@ -240,9 +245,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (4 warps per CTA, own 128 rows)
+    // ------------------------------------------------------------------ epilogue (8 warps per CTA, own 128 rows:
+    // two warps per TMEM lane quadrant, each draining half of the tile's columns)
     const int ew = warp & 3;
-    EpiStage es{smem_base + STAGES2 * STAGE2_BYTES + ew * (EPI_UNITS * EPI_UNIT_BYTES), 0u};
+    const int half = (warp - 2) >> 2;
+    EpiStage es{smem_base + STAGES2 * STAGE2_BYTES + (warp - 2) * (EPI_UNITS * EPI_UNIT_BYTES), 0u};
     uint32_t tc = 0;
     bool ok = true;
     long long t_idle = 0, t_begin = clock64();
@@ -252,13 +259,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       const Tile2 tl = get_tile2<KIND>(p, t, rank);
       const int rin = ew * 32 + lane;
       if (tl.nkb == 0) {
-        if (TR::WGRAD) wgrad_zero_fill<KIND>(p, tl.e, tl.m0 + rin, tl.n0);
+        if (TR::WGRAD && half == 0) wgrad_zero_fill<KIND>(p, tl.e, tl.m0 + rin, tl.n0);
         continue;
       }
       const int acc = tc & 1;
       const uint32_t aph = (tc >> 1) & 1u;
       ++tc;
-      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, tl.write, tl.e, tl.m0 + rin);
+      epilogue_prefetch<KIND>(p, static_cast<int64_t>(tl.row0) + rin, tl.n0, tl.write && half == 0, tl.e, tl.m0 + rin);
       const long long w0 = clock64();
       if (!mbar_wait(tfull_bar(acc), aph)) {
         ok = false;
@@ -268,12 +275,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + acc * ACC_COLS;
       expert_epilogue<KIND>(p, tl.e, static_cast<int64_t>(tl.row0) + rin, (TR::WGRAD ? tl.m0 : tl.row0) + ew * 32, tl.n0, taddr,
-                            tl.write, TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : 32, es, lane);
+                            tl.write, TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : 32, es, lane, half, 2);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
     }
-    if (p.timers && lane == 0 && ew == 0 && leader) {
+    if (p.timers && lane == 0 && ew == 0 && half == 0 && leader) {
       atomicAdd(p.timers + 5, static_cast<unsigned long long>(clock64() - t_begin));
       atomicAdd(p.timers + 6, static_cast<unsigned long long>(t_idle));
       atomicAdd(p.timers + 7, 1ull);

@@ -32,6 +32,8 @@ struct GemmParams {
   const int32_t* counts;       // rows per expert (weight gradients stop their K loop at the last 64-row block with data)
   const int32_t* expert_order; // weight gradients: experts by row count, largest first
   const int32_t* pair_tab;     // CTA-pair kernels: per pair of row blocks {expert, first row, blocks (1|2), 0}
+  int pair_count_slot;         // which entry of sched holds the number of entries of pair_tab
+  const int32_t* tile_list;    // one-CTA row GEMMs: null = every 128-row tile, else the tiles to compute (sched[4] entries)
   int32_t* status;
   unsigned long long* timers;  // null, or 8 counters of this kind: summed over CTAs (see gemm.cu)
   int n_tiles;   // output tiles along N
@@ -102,7 +104,7 @@ template <int KIND>
 __device__ __forceinline__ int total_tiles(const GemmParams& p) {
   if (Traits<KIND>::WGRAD) return p.E * p.m_tiles * p.n_tiles;
   if (Traits<KIND>::STATIC_M) return p.static_m_tiles * p.n_tiles;
-  return p.sched[0] * p.n_tiles;
+  return (p.tile_list ? p.sched[4] : p.sched[0]) * p.n_tiles;
 }
 
 template <int KIND>
@@ -130,7 +132,7 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
     tl.nkb = p.k_blocks * p.nseg + p.k_blocks1;
   } else {
-    const int mt = t / p.n_tiles;
+    const int mt = p.tile_list ? p.tile_list[t / p.n_tiles] : t / p.n_tiles;
     tl.e = p.tile_expert[mt];
     tl.row0 = mt * BM;
     tl.m0 = 0;
@@ -323,42 +325,53 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
       }
     }
   } else if (KIND == GEMM_B2) {
-    // hg, hu of the thread's row are read straight from global memory, one 32-column chunk ahead of their use
+    // hg, hu of the warp's 32 rows x 32 columns arrive one chunk ahead of their use as coalesced pieces (four lanes
+    // per 64-byte row segment, eight rows per load instruction) and are transposed through the warp's two staging
+    // units so that every thread ends up with its own row.  (A thread fetching its own row directly costs one memory
+    // wavefront per lane and load: 256 wavefronts per chunk instead of 64.)
     uint4 nh[4], nu[4];
     const float gate = write ? p.row_gate[row] : 0.f;
     float dgp = 0.f;  // this row's share of dg = <dy, o> = <da, silu(hg) hu> over the tile's columns
-    const bool rd0 = write && n0 + c8_lo * 32 < p.N_total;
-    if (rd0) {
-      const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + n0 + c8_lo * 32);
-      const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + n0 + c8_lo * 32);
+    const int pr = lane >> 2, pc = (lane & 3) * 8;  // piece: rows pr + 8 i of the slab, 8 columns from pc
+    auto fetch = [&](int col) {
+      const uint16_t* qh = p.in0 + (static_cast<int64_t>(slab) + pr) * p.ld_out + col + pc;
+      const uint16_t* qu = p.in1 + (static_cast<int64_t>(slab) + pr) * p.ld_out + col + pc;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        nh[i] = __ldg(qh + i);
-        nu[i] = __ldg(qu + i);
+        nh[i] = __ldg(reinterpret_cast<const uint4*>(qh + static_cast<int64_t>(8 * i) * p.ld_out));
+        nu[i] = __ldg(reinterpret_cast<const uint4*>(qu + static_cast<int64_t>(8 * i) * p.ld_out));
       }
-    }
+    };
+    if (write && n0 + c8_lo * 32 < p.N_total) fetch(n0 + c8_lo * 32);
+    const uint32_t unit_h = es.base, unit_u = es.base + EPI_UNIT_BYTES;
 #pragma unroll 1
     for (int c = c8_lo; c < c8_hi; ++c) {
-      uint4 ch[4], cu[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        ch[i] = nh[i];
-        cu[i] = nu[i];
-      }
       const int col = n0 + c * 32;
-      if (write && c + 1 < c8_hi && col + 32 < p.N_total) {
-        const uint4* qh = reinterpret_cast<const uint4*>(p.in0 + row * p.ld_out + col + 32);
-        const uint4* qu = reinterpret_cast<const uint4*>(p.in1 + row * p.ld_out + col + 32);
+      const bool live = write && col < p.N_total;
+      uint4 ch[4], cu[4];
+      if (live) {
+        __syncwarp();  // the previous chunk's output reads of both units are done
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          nh[i] = __ldg(qh + i);
-          nu[i] = __ldg(qu + i);
+          const int r = pr + 8 * i;
+          const uint32_t a = r * 64 + (((lane & 3) ^ ((r >> 1) & 3)) << 4);
+          st_shared_v4(unit_h + a, nh[i].x, nh[i].y, nh[i].z, nh[i].w);
+          st_shared_v4(unit_u + a, nu[i].x, nu[i].y, nu[i].z, nu[i].w);
         }
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t a = lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4);
+          ch[j] = ld_shared_v4(unit_h + a);
+          cu[j] = ld_shared_v4(unit_u + a);
+        }
+        __syncwarp();  // both units are free for the output staging below
       }
+      if (write && c + 1 < c8_hi && col + 32 < p.N_total) fetch(col + 32);
       uint32_t rd[32];
       tmem_ld32(taddr + c * 32, rd);
       tmem_ld_wait();
-      if (write && col < p.N_total) {
+      if (live) {
         float hg[32], hu[32], t[32];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -380,6 +393,7 @@ __device__ __forceinline__ void expert_epilogue(const GemmParams& p, int e, int6
           hu[i] = dag * hu[i] * sg * (1.f + hg[i] * (1.f - sg));  // dhg
           t[i] = dag * hg[i] * sg;                                 // dhu
         }
+        es.n = 0;  // outputs go through unit 0, then unit 1
         stage_store32(es, p.out0 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, hu, lane);
         stage_store32(es, p.out1 + static_cast<int64_t>(slab) * p.ld_out + col, p.ld_out, rows_valid, t, lane);
       }

@@ -5,6 +5,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "tables.cuh"
 
 namespace moe {
 
@@ -235,18 +236,12 @@ __global__ void __launch_bounds__(TOK_TILE) hist_kernel(int64_t T, int E, int k,
 // (summed in a fixed order: reproducible).
 constexpr int SCAN_THREADS = 1024;
 __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, int k, int tok_tiles, int psum_rows,
-                                                            int32_t* __restrict__ tile_counts,
-                                                            int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-                                                            int32_t* __restrict__ pad_offsets,
-                                                            int32_t* __restrict__ sched, int32_t* __restrict__ tile_expert,
-                                                            int32_t* __restrict__ pair_tab,
-                                                            int32_t* __restrict__ expert_order,
+                                                            int32_t* __restrict__ tile_counts, const TableOut tabs,
                                                             const float* __restrict__ psum_part,
                                                             float* __restrict__ psum, int32_t* __restrict__ counts_out,
                                                             float* __restrict__ aux_out) {
   __shared__ int s_cnt[MAX_E];
-  __shared__ int s_pad[MAX_E + 1];
-  __shared__ int s_pair[MAX_E + 1];
+  __shared__ TableScratch s_tab;
   __shared__ float s_term[MAX_E];
   __shared__ float s_ps[SCAN_THREADS];
   const int tid = threadIdx.x;
@@ -292,83 +287,24 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
   __syncthreads();
   for (int e = tid; e < E; e += SCAN_THREADS) {
     const int run = s_cnt[e];
-    counts[e] = run;
     counts_out[e] = run;
     float ps = 0.f;
     for (int g = 0; g < G; ++g) ps += s_ps[g * E + e];
     psum[e] = ps;
     // aux term: (c_e / (T k)) * (Psum_e / T)
     s_term[e] = (T > 0) ? (static_cast<float>(run) / static_cast<float>(T * k)) * (ps / static_cast<float>(T)) : 0.f;
-    // position of e in the order "most rows first" (ties by index): the weight-gradient kernels start with the
-    // experts whose K loops are longest so that a skewed load does not leave a long tail
-    int rank = 0;
-    for (int o = 0; o < E; ++o) rank += (s_cnt[o] > run || (s_cnt[o] == run && o < e)) ? 1 : 0;
-    expert_order[rank] = e;
   }
   __syncthreads();
-  if (tid < 32) {
-    // exclusive scans of counts, padded counts and block pairs over the experts: lane L owns experts 8L .. 8L+7
-    const int lane = tid;
-    int cn[8], pd[8], pr[8];
-    int scn = 0, spd = 0, spr = 0;
+  if (tid >= 32 && tid < 64) {  // the second warp sums the aux terms in a fixed order while the first one scans
+    const int lane = tid - 32;
     float sterm = 0.f;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int e = lane * 8 + u;
-      const int cnt = e < E ? s_cnt[e] : 0;
-      const int blocks = (cnt + ROW_PAD - 1) / ROW_PAD;
-      cn[u] = scn;
-      pd[u] = spd;
-      pr[u] = spr;
-      scn += cnt;
-      spd += blocks * ROW_PAD;
-      spr += (blocks + 1) / 2;
-      sterm += e < E ? s_term[e] : 0.f;
-    }
-    int icn = scn, ipd = spd, ipr = spr;
+    for (int u = 0; u < 8; ++u) sterm += (lane * 8 + u < E) ? s_term[lane * 8 + u] : 0.f;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const int a = __shfl_up_sync(0xFFFFFFFFu, icn, off), b = __shfl_up_sync(0xFFFFFFFFu, ipd, off),
-                c = __shfl_up_sync(0xFFFFFFFFu, ipr, off);
-      if (lane >= off) {
-        icn += a;
-        ipd += b;
-        ipr += c;
-      }
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sterm += __shfl_xor_sync(0xFFFFFFFFu, sterm, off);  // fixed tree
-    const int bcn = icn - scn, bpd = ipd - spd, bpr = ipr - spr;  // exclusive bases of this lane
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int e = lane * 8 + u;
-      if (e < E) {
-        offsets[e] = bcn + cn[u];
-        pad_offsets[e] = bpd + pd[u];
-        s_pad[e] = bpd + pd[u];
-        s_pair[e] = bpr + pr[u];
-      }
-    }
-    if (lane == 31) {
-      offsets[E] = icn;
-      pad_offsets[E] = ipd;
-      s_pad[E] = ipd;
-      s_pair[E] = ipr;
-      sched[0] = ipd / ROW_PAD;
-      sched[1] = ipd;
-      sched[2] = ipr;
-      aux_out[0] = sterm * static_cast<float>(E);
-    }
+    for (int off = 16; off > 0; off >>= 1) sterm += __shfl_xor_sync(0xFFFFFFFFu, sterm, off);
+    if (lane == 0) aux_out[0] = sterm * static_cast<float>(E);
   }
-  __syncthreads();
-  for (int e = tid; e < E; e += SCAN_THREADS) {
-    for (int m = s_pad[e] / ROW_PAD; m < s_pad[e + 1] / ROW_PAD; ++m) tile_expert[m] = e;
-    // pairs of consecutive 128-row blocks of this expert; the last pair of an odd count has one block
-    const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_PAD;
-    for (int q = 0; q < s_pair[e + 1] - s_pair[e]; ++q)
-      *reinterpret_cast<int4*>(pair_tab + 4 * (s_pair[e] + q)) =
-          make_int4(e, s_pad[e] + 2 * q * ROW_PAD, min(2, blocks - 2 * q), 0);
-  }
+  build_expert_tables(E, s_cnt, s_tab, tabs);
 }
 
 __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int k, const int32_t* __restrict__ idx,
@@ -460,14 +396,16 @@ __global__ void __launch_bounds__(256) prepare_kernel(int32_t* __restrict__ stat
 }
 
 void launch_prepare(const WsLayout& L, char* ws, cudaStream_t st) {
-  const int blocks = static_cast<int>(std::min<int64_t>(296, std::max<int64_t>(1, (L.rows_max + 255) / 256)));
+  const int blocks = static_cast<int>(std::min<int64_t>(296, std::max<int64_t>(1, (L.rows_alloc + 255) / 256)));
   prepare_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + L.status),
-                                         reinterpret_cast<float*>(ws + L.row_gate), L.rows_max);
+                                         reinterpret_cast<float*>(ws + L.row_gate), L.rows_alloc);
   note_launch();
 }
 
+// tables_only: stop after the histogram and the scan (per-tile prefixes, counts, tables, aux loss); the expert-parallel
+// path places the rows itself
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
-                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st) {
+                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only) {
   int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
   int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
   const int tiles = static_cast<int>(L.tok_tiles);
@@ -476,17 +414,11 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
     hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
     note_launch();
   }
-  scan_kernel<<<1, SCAN_THREADS, 0, st>>>(T, s.E, s.k, tiles, psum_rows, tile_counts,
-                                 reinterpret_cast<int32_t*>(ws + L.counts), reinterpret_cast<int32_t*>(ws + L.offsets),
-                                 reinterpret_cast<int32_t*>(ws + L.pad_offsets),
-                                 reinterpret_cast<int32_t*>(ws + L.sched),
-                                 reinterpret_cast<int32_t*>(ws + L.tile_expert),
-                                 reinterpret_cast<int32_t*>(ws + L.pair_tab),
-                                 reinterpret_cast<int32_t*>(ws + L.expert_order),
+  scan_kernel<<<1, SCAN_THREADS, 0, st>>>(T, s.E, s.k, tiles, psum_rows, tile_counts, table_pointers(L, ws),
                                  reinterpret_cast<const float*>(ws + L.psum_part),
                                  reinterpret_cast<float*>(ws + L.psum), counts_out, aux_out);
   note_launch();
-  if (tiles > 0) {
+  if (tiles > 0 && !tables_only) {
     scatter_kernel<<<tiles, TOK_TILE, msm, st>>>(
         T, s.E, s.k, idx, tile_counts, reinterpret_cast<const int32_t*>(ws + L.offsets),
         reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const float*>(ws + L.gates),

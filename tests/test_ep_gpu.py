@@ -1,0 +1,111 @@
+"""Expert parallelism (EP > 1): the ranks of a group, run inside one process on one GPU (ep.LocalGroup: the same
+kernels a multi-GPU group runs, phases enqueued rank after rank), must reproduce the oracle applied to the
+concatenation of the ranks' token batches: routing bit-exact per rank, the owners' row buffers in the oracle's
+expert-major order, y and dx per token, the owned experts' weight gradients, and the sum over ranks of dW_r."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_00916_b200 import ep, synth
+from gpu_util import from_dev_bf16, oracle_run, rel_fro, to_dev_bf16
+from oracle import moe_oracle as orc
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+@pytest.mark.parametrize("d,E,k,f,tokens,seed,flags", [
+    (256, 16, 4, 256, [300, 517], 31, 0),            # two ranks, uneven batches
+    (128, 32, 8, 128, [100, 0, 333, 64], 32, 0),     # four ranks, one of them without tokens
+    (128, 8, 4, 192, [260, 130, 50, 90], 33, 2),     # fewer owned experts (2) than top_k (4); one-CTA tiles
+    (192, 64, 6, 64, [1500, 1100], 34, 1),           # 32 owned experts each, CTA-pair tiles
+])
+def test_local_group_matches_the_oracle_on_the_concatenated_batch(d, E, k, f, tokens, seed, flags):
+    world = len(tokens)
+    T = sum(tokens)
+    shape = synth.MoEShape(T, d, E, k, f)
+    inp = synth.make_inputs(shape, seed, x_std=1.0)
+    ofw, obw = oracle_run(inp, k, 0.0)
+    bounds = np.concatenate([[0], np.cumsum(tokens)])
+    dev = {n: to_dev_bf16(inp[n]) for n in ("x", "W_r", "W_gate", "W_up", "W_down", "dy")}
+    xs = [dev["x"][bounds[r]:bounds[r + 1]].contiguous() for r in range(world)]
+    dys = [dev["dy"][bounds[r]:bounds[r + 1]].contiguous() for r in range(world)]
+    grp = ep.LocalGroup(d, E, f, k, world, ep.rows_cap_bound(tokens, k, E, world), flags)
+    fw, all_counts = grp.forward(xs, dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
+    grp.poll()
+    e_loc = E // world
+    ac = all_counts.cpu().numpy()
+    assert np.array_equal(ac.sum(axis=0), ofw["counts"])
+    for r in range(world):
+        sl = slice(bounds[r], bounds[r + 1])
+        # routing of the rank's tokens: bit-exact; its own counts; aux over its own tokens
+        assert np.array_equal(fw[r]["idx"].cpu().numpy(), ofw["idx"][sl])
+        if tokens[r] > 0:
+            assert np.abs(fw[r]["gates"].cpu().numpy() - ofw["gates"][sl]).max() <= 1e-5
+        assert np.array_equal(ac[r], np.bincount(ofw["idx"][sl].ravel(), minlength=E))
+        if tokens[r] > 0:
+            local = orc.route_only(inp["x"][sl], inp["W_r"], k, E)
+            assert float(fw[r]["aux"].cpu()[0]) == pytest.approx(local["aux"], rel=1e-4)
+            assert rel_fro(from_dev_bf16(fw[r]["y"]), ofw["y"][sl]) <= TOL
+        # placement: the device tables equal the host restatement
+        plan = ep.plan_host(ac, r, world)
+        rk = grp.ranks[r]
+        assert np.array_equal(rk.buffer("ep_dest", torch.int32, False).cpu().numpy(), plan["dest_base"])
+        assert np.array_equal(rk.buffer("counts", torch.int32, True).cpu().numpy(), plan["own_counts"])
+        assert np.array_equal(rk.buffer("pad_offsets", torch.int32, True).cpu().numpy(), plan["own_pad_offsets"])
+        if tokens[r] > 0:
+            inv = rk.buffer("inv", torch.int32, False).view(tokens[r], k).cpu().numpy()
+            assert np.array_equal(inv, ep.rows_of_rank(ofw["idx"][sl], plan["dest_base"]))
+        # the owner's xp rows: expert by expert the oracle's rows of the concatenated batch, in its order; pad rows zero
+        xp = rk.buffer("xp", torch.bfloat16, True).view(-1, d)
+        for el in range(e_loc):
+            e = r * e_loc + el
+            n = int(plan["own_counts"][el])
+            p0, p1 = int(plan["own_pad_offsets"][el]), int(plan["own_pad_offsets"][el + 1])
+            got = xp[p0:p1].float().cpu().numpy()
+            ref = ofw["xp"][ofw["offsets"][e]:ofw["offsets"][e + 1]]
+            assert np.array_equal(got[:n], ref), (r, e)
+            assert not got[n:].any(), (r, e)
+    sender, owner = grp.backward(dys, 0.0, want_db=True)
+    grp.poll()
+    dW_r = np.zeros((d, E))
+    db_r = np.zeros(E)
+    for r in range(world):
+        sl = slice(bounds[r], bounds[r + 1])
+        if tokens[r] > 0:
+            assert rel_fro(from_dev_bf16(sender[r]["dx"]), obw["dx"][sl]) <= TOL
+            dl = grp.ranks[r].buffer("dl", torch.float32, False).view(tokens[r], E).cpu().numpy()
+            assert rel_fro(dl, obw["dl"][sl]) <= TOL
+        dW_r += sender[r]["dW_r"].cpu().numpy().astype(np.float64)
+        db_r += sender[r]["db_r"].cpu().numpy().astype(np.float64)
+        own = slice(r * e_loc, (r + 1) * e_loc)
+        for n in ("dW_gate", "dW_up", "dW_down"):
+            got = from_dev_bf16(owner[r][n])
+            assert rel_fro(got, obw[n][own]) <= TOL, (r, n)
+            for el in range(e_loc):
+                if ofw["counts"][r * e_loc + el] == 0:
+                    assert not got[el].any()
+                else:
+                    assert rel_fro(got[el], obw[n][r * e_loc + el]) <= 2e-2, (r, n, el)
+    assert rel_fro(dW_r, obw["dW_r"]) <= TOL
+    assert rel_fro(db_r, obw["db_r"]) <= TOL
+
+
+def test_ep_with_one_rank_equals_the_plain_layer():
+    """world = 1 degenerates to the one-GPU layer: same routing, y and gradients as moe_forward / moe_backward."""
+    from gpu_util import Run
+    shape = synth.MoEShape(700, 256, 16, 4, 128)
+    inp = synth.make_inputs(shape, 35)
+    r = Run(inp, shape.k)
+    fw = r.forward()
+    bw = r.backward(0.03)
+    grp = ep.LocalGroup(shape.d, shape.E, shape.f, shape.k, 1, shape.T * shape.k)
+    v = r.dev
+    efw, _ = grp.forward([v["x"]], v["W_r"], v["W_gate"], v["W_up"], v["W_down"])
+    sender, owner = grp.backward([v["dy"]], 0.03)
+    grp.poll()
+    assert torch.equal(efw[0]["idx"], fw["idx"]) and torch.equal(efw[0]["gates"], fw["gates"])
+    assert torch.equal(efw[0]["y"], fw["y"]) and torch.equal(efw[0]["aux"], fw["aux"])
+    assert torch.equal(sender[0]["dx"], bw["dx"]) and torch.equal(sender[0]["dW_r"], bw["dW_r"])
+    for n in ("dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(owner[0][n], bw[n]), n

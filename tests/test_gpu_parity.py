@@ -10,6 +10,7 @@ import torch
 
 from paper_2608_00916_b200 import synth
 from gpu_util import Run, from_dev_bf16, oracle_run, rel_fro
+from paper_2608_00916_b200.binding import MoELayer
 from oracle import moe_oracle as orc
 
 pytestmark = pytest.mark.gpu
@@ -88,11 +89,14 @@ def test_odd_shapes(T, d, E, k, f, seed):
     check_all(Run(inp, k), ofw, obw, 0.05)
 
 
-@pytest.mark.parametrize("flag", [1, 2])
-@pytest.mark.parametrize("T,d,E,k,f,seed", [(1000, 512, 16, 4, 384, 14), (333, 192, 5, 5, 320, 15), (2049, 256, 32, 8, 128, 17)])
+@pytest.mark.parametrize("flag", [1, 2, 16, 16 | 8])
+@pytest.mark.parametrize("T,d,E,k,f,seed", [(1000, 512, 16, 4, 384, 14), (333, 192, 5, 5, 320, 15), (2049, 256, 32, 8, 128, 17),
+                                            (3000, 256, 8, 2, 256, 21)])
 def test_forced_tile_shapes(T, d, E, k, f, seed, flag):
-    """Forcing CTA pairs (cta_group::2, 256-row tiles; flag 1) or one-CTA tiles (flag 2) for every expert GEMM gives
-    the same results as the default per-GEMM choice."""
+    """Forcing CTA pairs (cta_group::2, 256-row tiles; flag 1), one-CTA tiles (flag 2) or the mixed schedule (complete
+    pairs of row blocks on CTA pairs, leftover blocks on one-CTA tiles; flag 16, also with the router's gradient chain
+    kept on the caller's stream, flag 8) for every expert GEMM gives the same results as the default per-GEMM
+    choice.  The last shape has experts with one, an even and an odd number of row blocks."""
     shape = synth.MoEShape(T, d, E, k, f)
     inp = synth.make_inputs(shape, seed, x_std=1.0)
     ofw, obw = oracle_run(inp, k, 0.05)
@@ -126,7 +130,7 @@ def test_random_shapes(T, d, E, k, f, seed):
             pytest.skip("no guarded token in this draw")
         inp["x"], inp["dy"] = inp["x"][keep], inp["dy"][keep]
     ofw, obw = oracle_run(inp, k, 0.03)
-    check_all(Run(inp, k, flags=seed % 3), ofw, obw, 0.03)
+    check_all(Run(inp, k, flags=(0, 1, 2, 16)[seed % 4]), ofw, obw, 0.03)
 
 
 @pytest.mark.parametrize("T,d,E,k,f", [(1, 64, 8, 2, 64), (47, 128, 256, 3, 64), (300, 192, 24, 4, 320), (1029, 256, 16, 8, 128)])
@@ -261,7 +265,7 @@ def test_forward_inference_entry(T, d, E, k, f, seed):
     assert torch.equal(train["y"], fw["y"])  # bitwise the same outputs as the training forward
 
 
-@pytest.mark.parametrize("flag", [0, 1, 2])
+@pytest.mark.parametrize("flag", [0, 1, 2, 16])
 def test_backward_accumulate_over_micro_batches(flag):
     """moe_backward_accumulate adds the weight gradients of successive micro-batches into fp32 buffers: after
     three micro-batches (one of them leaving experts empty) the buffers hold the sum of the oracle's gradients."""

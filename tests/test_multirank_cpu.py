@@ -121,3 +121,128 @@ def test_launcher_starts_gloo_ranks(tmp_path):
     assert got == ["0 2 0 20.0", "1 2 1 20.0"]
     # a rank that fails makes the launcher report it
     assert pdist.launch_ranks(2, script, [str(tmp_path), "fail-on-1"], timeout=180) != 0
+
+
+# ------------------------------------------------------------------------------------------ expert parallelism
+def _ep_worker(rank, world, port, q):
+    """One CPU rank of an expert-parallel group.  The exchange logic under test is the host restatement of the
+    placement (ep.plan_host / ep.rows_of_rank): counts all-gather, per-rank expert ownership, destination rows inside
+    the owner's expert-major buffers, the inverse map used by the combine.  The per-expert arithmetic is the oracle's
+    (test infrastructure); rows travel between the ranks through the gloo group."""
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    import torch
+    import torch.distributed as dist
+    from oracle import moe_oracle as orc
+    from paper_2608_00916_b200 import dist as pdist
+    from paper_2608_00916_b200 import ep, synth
+    pdist.init(world, rank, backend="gloo")
+    d, E, k, f = 64, 8, 3, 64
+    tokens = [37, 0, 52, 21][:world] if world == 4 else [45, 30]
+    T = sum(tokens)
+    inp = synth.make_inputs(synth.MoEShape(T, d, E, k, f), 900 + world, threads=1)  # the concatenated batch
+    b = np.concatenate([[0], np.cumsum(tokens)])
+    sl = slice(b[rank], b[rank + 1])
+    e_loc = E // world
+    x = orc.widen_bf16(inp["x"][sl])
+    dy = orc.widen_bf16(inp["dy"][sl])
+    Wg, Wu, Wd = (orc.widen_bf16(inp[n][rank * e_loc:(rank + 1) * e_loc]) for n in ("W_gate", "W_up", "W_down"))
+    route = orc.route_only(inp["x"][sl], inp["W_r"], k, E) if tokens[rank] else {"idx": np.zeros((0, k), np.int64),
+                                                                                    "gates": np.zeros((0, k))}
+    idx, gates = route["idx"], route["gates"]
+    # --- counts all-gather
+    mine = torch.from_numpy(np.bincount(idx.ravel(), minlength=E).astype(np.int64))
+    gathered = [torch.zeros(E, dtype=torch.int64) for _ in range(world)]
+    dist.all_gather(gathered, mine)
+    all_counts = torch.stack(gathered).numpy()
+    plan = ep.plan_host(all_counts, rank, world)
+    inv = ep.rows_of_rank(idx, plan["dest_base"])
+
+    def exchange(payload_of_pair):
+        """Sends payload(t, j) of every pair to the owner of its expert, addressed by its destination row."""
+        out = [[] for _ in range(world)]
+        for t in range(idx.shape[0]):
+            for j in range(k):
+                out[int(idx[t, j]) // e_loc].append((int(inv[t, j]), payload_of_pair(t, j)))
+        box = [None] * world
+        dist.all_gather_object(box, out)
+        return [item for src in range(world) for item in box[src][rank]]
+
+    # --- dispatch x rows (with their gates) into the owner's padded expert-major buffer
+    rows_pad = int(plan["own_pad_offsets"][-1])
+    xp = np.zeros((rows_pad, d))
+    filled = np.zeros(rows_pad, dtype=bool)
+    for r, (row, g) in exchange(lambda t, j: (x[t], float(gates[t, j]))):
+        assert not filled[r]
+        xp[r], filled[r] = row, True
+    # every real row of every owned segment was written exactly once, pad rows never
+    for el in range(e_loc):
+        p0 = int(plan["own_pad_offsets"][el])
+        n = int(plan["own_counts"][el])
+        assert filled[p0:p0 + n].all() and not filled[p0 + n:int(plan["own_pad_offsets"][el + 1])].any()
+    # --- experts (oracle arithmetic), outputs pulled back by destination row
+    o = np.zeros((rows_pad, d))
+    hg, hu = np.zeros((rows_pad, f)), np.zeros((rows_pad, f))
+    for el in range(e_loc):
+        p0, n = int(plan["own_pad_offsets"][el]), int(plan["own_counts"][el])
+        hg[p0:p0 + n], hu[p0:p0 + n], _, o[p0:p0 + n] = orc.expert_ffn(xp[p0:p0 + n], Wg[el], Wu[el], Wd[el])
+    box = [None] * world
+    dist.all_gather_object(box, o)
+    y = np.zeros((idx.shape[0], d))
+    for t in range(idx.shape[0]):
+        for j in range(k):
+            y[t] += gates[t, j] * box[int(idx[t, j]) // e_loc][int(inv[t, j])]
+    # --- backward of the expert path: g dy rows to the owners, dxp rows back
+    d_o = np.zeros((rows_pad, d))
+    for r, row in exchange(lambda t, j: gates[t, j] * dy[t]):
+        d_o[r] = row
+    dxp = np.zeros((rows_pad, d))
+    for el in range(e_loc):
+        p0, n = int(plan["own_pad_offsets"][el]), int(plan["own_counts"][el])
+        s_ = slice(p0, p0 + n)
+        da = d_o[s_] @ Wd[el].T
+        sg = 1.0 / (1.0 + np.exp(-hg[s_]))
+        dhg = da * hu[s_] * sg * (1.0 + hg[s_] * (1.0 - sg))
+        dhu = da * hg[s_] * sg
+        dxp[s_] = dhg @ Wg[el].T + dhu @ Wu[el].T
+    dist.all_gather_object(box, dxp)
+    dx_experts = np.zeros((idx.shape[0], d))
+    for t in range(idx.shape[0]):
+        for j in range(k):
+            dx_experts[t] += box[int(idx[t, j]) // e_loc][int(inv[t, j])]
+    # --- reference: the oracle on the concatenated batch (every rank can afford it at this size)
+    fw = orc.forward(inp["x"], inp["W_r"], inp["W_gate"], inp["W_up"], inp["W_down"], k)
+    bw = orc.backward(fw, inp["dy"], 0.0, inp["x"], inp["W_r"], inp["W_gate"], inp["W_up"], inp["W_down"])
+    dx_router = bw["dl"][sl] @ orc.widen_bf16(inp["W_r"]).T
+    ok_rows = all(np.array_equal(xp[int(plan["own_pad_offsets"][el]):int(plan["own_pad_offsets"][el]) + int(plan["own_counts"][el])],
+                                 fw["xp"][fw["offsets"][rank * e_loc + el]:fw["offsets"][rank * e_loc + el + 1]])
+                  for el in range(e_loc))
+    q.put((rank, bool(np.array_equal(idx, fw["idx"][sl])), ok_rows,
+           float(np.abs(y - fw["y"][sl]).max()) if tokens[rank] else 0.0,
+           float(np.abs(dx_experts + dx_router - bw["dx"][sl]).max()) if tokens[rank] else 0.0,
+           float(np.abs(fw["y"]).max())))
+    pdist.finish()
+
+
+import pytest  # noqa: E402
+
+
+@pytest.mark.parametrize("world", [2, 4])
+def test_expert_parallel_exchange_over_gloo_ranks(world):
+    """EP group on CPU ranks: after the counts all-gather every rank places its rows inside the owners' buffers; the
+    owners' segments come out in the order of the concatenated batch, and y / dx of every rank's tokens equal the
+    oracle's on the concatenated batch (routing bit-exact, values to rounding)."""
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29950 + os.getpid() % 40 + 3 * world
+    procs = [ctx.Process(target=_ep_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, routing_same, rows_in_order, y_err, dx_err, scale in res:
+        assert routing_same and rows_in_order, rank
+        assert y_err <= 1e-9 * max(scale, 1.0) and dx_err <= 1e-9, (rank, y_err, dx_err)
