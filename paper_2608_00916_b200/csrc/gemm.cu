@@ -30,6 +30,10 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
     grouped_gemm_kernel(const __grid_constant__ GemmParams p) {
   using TR = Traits<KIND>;
   constexpr int EPI_WARPS = (KIND == GEMM_RT) ? 4 : 8;
+  // the routing kind runs a three-stage ring (it streams x once, 16 KB per stage) and uses the rest of the dynamic
+  // shared memory (the fourth stage and the staging units: 80 KB) as scratch of its routing epilogue
+  constexpr int NST = (KIND == GEMM_RT) ? 3 : STAGES;
+  static_assert(STAGE_BYTES + EPI_BYTES >= ROUTE_SCRATCH_BYTES, "routing scratch does not fit");
   extern __shared__ unsigned char gemm_smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
   __shared__ uint32_t tmem_base_slot;
@@ -46,7 +50,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < NST; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
@@ -78,8 +82,8 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       if (t >= ntiles) continue;
       const Tile tl = get_tile<KIND>(p, t);
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1u;
+        const int s = it % NST;
+        const uint32_t ph = (it / NST) & 1u;
         const long long w0 = clock64();
         if (!mbar_wait(empty_bar(s), ph ^ 1u)) {
           ok = false;
@@ -126,8 +130,8 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
       for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1u;
+        const int s = it % NST;
+        const uint32_t ph = (it / NST) & 1u;
         const long long w1 = clock64();
         if (!mbar_wait(full_bar(s), ph)) {
           ok = false;
@@ -206,8 +210,9 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
                               TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
                               es, lane, half, NHALF);
       } else if (KIND == GEMM_RT) {
-        if (p.N_total <= 128)
-          routing_epilogue_regs(p, s_bias, row, tl.row0 / BM, ew, taddr, lane);
+        if (p.N_total <= 128 && p.top_k <= ROUTE_SMEM_MAX_K)  // picks live in the unused tail of stage 0 (B is <= 16 KB)
+          routing_epilogue_smem(p, s_bias, smem_base + NST * STAGE_BYTES, smem_base + A_BYTES + 2 * CHUNK_BYTES, row,
+                                tl.row0 / BM, ew, taddr, lane);
         else
           routing_epilogue_tmem(p, s_bias, row, tl.row0 / BM, ew, taddr, lane);
       } else if (KIND == GEMM_DWR) {

@@ -601,91 +601,142 @@ __device__ __forceinline__ void routing_epilogue_tmem(const GemmParams& p, const
         }
 }
 
-// E <= 128: the whole row of logits stays in registers (one TMEM read), exponentials use the fast intrinsic.
-__device__ __forceinline__ void routing_epilogue_regs(const GemmParams& p, const float* s_bias, int64_t row, int tile,
-                                                      int ew, uint32_t taddr, int lane) {
+// E <= 128, top_k <= 16.  Top-k is a three-level tournament per token: the 128 logits in groups of four, the group
+// maxima in "supers" of four groups, the eight super maxima in registers.  A round takes the largest super maximum
+// (lowest super among equals), then the group and the column inside it (lowest index among equals at every level,
+// which is the lowest-index rule overall because the levels partition the index range in order), removes the column
+// and repairs the three maxima above it.  The group of four values and the four group maxima sit in shared memory
+// because the group that wins a round is only known at run time; each level is one 16-byte access.
+// The code is written as rolled loops on purpose.  A CTA runs this epilogue once (one 128-token tile per CTA), so
+// every instruction is fetched cold: the earlier fully unrolled versions (thousands of straight-line instructions)
+// were bound by instruction fetch, not by execution - unrolling the k rounds made the epilogue twice as slow.
+// Shared-memory layout (per CTA): vals[g][thread] float4 for g < 32 (64 KB), gmax[s][thread] float4 for s < 8 (16 KB),
+// picks[j][thread] {value, column} for j < 16 (16 KB, in the unused tail of the first pipeline stage); consecutive
+// threads touch consecutive words, so accesses are conflict-free whichever group a thread picks.
+constexpr uint32_t ROUTE_SCRATCH_BYTES = 128 * 128 * 4 + 128 * 32 * 4;
+constexpr int ROUTE_SMEM_MAX_K = 16;
+
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts_f4(uint32_t addr, float4 v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ float max4(float4 v) { return fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)); }
+// index (0..3) of the first component equal to m
+__device__ __forceinline__ int first_eq4(float4 v, float m) { return v.x == m ? 0 : (v.y == m ? 1 : (v.z == m ? 2 : 3)); }
+
+__device__ __forceinline__ void routing_epilogue_smem(const GemmParams& p, const float* s_bias, uint32_t scratch,
+                                                      uint32_t picks_base, int64_t row, int tile, int ew, uint32_t taddr,
+                                                      int lane) {
   const int64_t tok = row;
   const bool valid = tok < p.T;
   const int E = p.N_total, k = p.top_k;
-  float v[128];
-  {
-    uint32_t r0[32], r1[32], r2[32], r3[32];
-    tmem_ld32(taddr, r0);
-    tmem_ld32(taddr + 32, r1);
-    tmem_ld32(taddr + 64, r2);
-    tmem_ld32(taddr + 96, r3);
+  const int tid = ew * 32 + lane;  // token of the tile
+  const uint32_t vals = scratch + tid * 16, gmx = scratch + 128 * 128 * 4 + tid * 16, picks = picks_base + tid * 8;
+  constexpr uint32_t PITCH = 128 * 16;  // bytes between consecutive groups / supers of one thread
+  float sm[8];
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    uint32_t r[32];
+    tmem_ld32(taddr + c * 32, r);
     tmem_ld_wait();
+    float v[32];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      v[i] = __uint_as_float(r0[i]) + s_bias[i];
-      v[32 + i] = __uint_as_float(r1[i]) + s_bias[32 + i];
-      v[64 + i] = __uint_as_float(r2[i]) + s_bias[64 + i];
-      v[96 + i] = __uint_as_float(r3[i]) + s_bias[96 + i];
+    for (int i = 0; i < 32; ++i) v[i] = (c * 32 + i < E) ? __uint_as_float(r[i]) + s_bias[c * 32 + i] : -INFINITY;
+    if (valid) {
+#pragma unroll
+      for (int i = 0; i < 32; i += 4) {
+        if (c * 32 + i < E) {
+          const float4 w = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          *reinterpret_cast<float4*>(p.logits + tok * E + c * 32 + i) = w;
+          if (p.logits_out) *reinterpret_cast<float4*>(p.logits_out + tok * E + c * 32 + i) = w;
+        }
+      }
     }
-  }
-  if (valid) {
+    float gm[8];
 #pragma unroll
-    for (int i = 0; i < 128; i += 4) {
-      if (i < E) {
-        const float4 w = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-        *reinterpret_cast<float4*>(p.logits + tok * E + i) = w;
-        if (p.logits_out) *reinterpret_cast<float4*>(p.logits_out + tok * E + i) = w;
+    for (int q = 0; q < 8; ++q) {
+      const float4 w = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      sts_f4(vals + (c * 8 + q) * PITCH, w);
+      gm[q] = max4(w);
+    }
+    const float4 w0 = make_float4(gm[0], gm[1], gm[2], gm[3]), w1 = make_float4(gm[4], gm[5], gm[6], gm[7]);
+    sts_f4(gmx + (c * 2) * PITCH, w0);
+    sts_f4(gmx + (c * 2 + 1) * PITCH, w1);
+    const float m0 = max4(w0), m1 = max4(w1);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) sm[q] = (q == 2 * c) ? m0 : ((q == 2 * c + 1) ? m1 : sm[q]);
+  }
+  float vmax = 0.f, zs = 0.f;
+#pragma unroll 1
+  for (int j = 0; j < k; ++j) {
+    const float best = fmaxf(fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3])), fmaxf(fmaxf(sm[4], sm[5]), fmaxf(sm[6], sm[7])));
+    int s = 7;
+#pragma unroll
+    for (int q = 6; q >= 0; --q) s = (sm[q] == best) ? q : s;
+    float4 g4 = lds_f4(gmx + s * PITCH);
+    const int gi = first_eq4(g4, best);
+    const int g = s * 4 + gi;
+    float4 v4 = lds_f4(vals + g * PITCH);
+    const int ci = first_eq4(v4, best);
+    if (j == 0) vmax = best;
+    const float ex = __expf(best - vmax);
+    zs += ex;
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(picks + j * (128 * 8)), "r"(__float_as_uint(ex)), "r"(g * 4 + ci)
+                 : "memory");
+    v4.x = ci == 0 ? -INFINITY : v4.x;
+    v4.y = ci == 1 ? -INFINITY : v4.y;
+    v4.z = ci == 2 ? -INFINITY : v4.z;
+    v4.w = ci == 3 ? -INFINITY : v4.w;
+    sts_f4(vals + g * PITCH, v4);
+    const float ng = max4(v4);
+    g4.x = gi == 0 ? ng : g4.x;
+    g4.y = gi == 1 ? ng : g4.y;
+    g4.z = gi == 2 ? ng : g4.z;
+    g4.w = gi == 3 ? ng : g4.w;
+    sts_f4(gmx + s * PITCH, g4);
+    const float ns = max4(g4);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) sm[q] = (q == s) ? ns : sm[q];
+  }
+  // softmax over all E logits (read again from tensor memory: the shared copy has lost the picks); the exponentials
+  // are parked in the shared copy until their sum is known
+  float z = 0.f;
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    if (c * 32 < E) {
+      uint32_t r[32];
+      tmem_ld32(taddr + c * 32, r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        float4 w;
+        w.x = (c * 32 + 4 * q + 0 < E) ? __expf(__uint_as_float(r[4 * q + 0]) + s_bias[c * 32 + 4 * q + 0] - vmax) : 0.f;
+        w.y = (c * 32 + 4 * q + 1 < E) ? __expf(__uint_as_float(r[4 * q + 1]) + s_bias[c * 32 + 4 * q + 1] - vmax) : 0.f;
+        w.z = (c * 32 + 4 * q + 2 < E) ? __expf(__uint_as_float(r[4 * q + 2]) + s_bias[c * 32 + 4 * q + 2] - vmax) : 0.f;
+        w.w = (c * 32 + 4 * q + 3 < E) ? __expf(__uint_as_float(r[4 * q + 3]) + s_bias[c * 32 + 4 * q + 3] - vmax) : 0.f;
+        z += (w.x + w.y) + (w.z + w.w);
+        sts_f4(vals + (c * 8 + q) * PITCH, w);
       }
     }
   }
-  // Top-k by k rounds of (max value, lowest index attaining it, remove it).  Only one warp per scheduler runs this
-  // code, so it is written for instruction-level parallelism: the value maximum and the index minimum are
-  // FMNMX / IMNMX chains split four ways, everything else is independent per column; no predicate feeds a
-  // loop-carried dependency (a compare-and-select chain took 56 cycles per column here).
-#pragma unroll
-  for (int i = 0; i < 128; ++i)
-    if (i >= E) v[i] = -INFINITY;  // columns beyond E can never be picked
-  float selv[MAX_K];
-  int seli[MAX_K];
-  for (int j = 0; j < k; ++j) {
-    float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-    for (int i = 0; i < 128; ++i) m[i & 3] = fmaxf(m[i & 3], v[i]);
-    const float best = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
-    int q[4] = {0x7FFFFFFF, 0x7FFFFFFF, 0x7FFFFFFF, 0x7FFFFFFF};
-#pragma unroll
-    for (int i = 0; i < 128; ++i) q[i & 3] = min(q[i & 3], v[i] == best ? i : 0x7FFFFFFF);
-    const int bi = min(min(q[0], q[1]), min(q[2], q[3]));
-#pragma unroll
-    for (int i = 0; i < 128; ++i) v[i] = (i == bi) ? -INFINITY : v[i];
-    selv[j] = best;
-    seli[j] = bi;
-  }
-  // the picks were removed from the register copy: read the row again for the softmax statistics
-  {
-    uint32_t r0[32], r1[32], r2[32], r3[32];
-    tmem_ld32(taddr, r0);
-    tmem_ld32(taddr + 32, r1);
-    tmem_ld32(taddr + 64, r2);
-    tmem_ld32(taddr + 96, r3);
-    tmem_ld_wait();
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      v[i] = __uint_as_float(r0[i]) + s_bias[i];
-      v[32 + i] = __uint_as_float(r1[i]) + s_bias[32 + i];
-      v[64 + i] = __uint_as_float(r2[i]) + s_bias[64 + i];
-      v[96 + i] = __uint_as_float(r3[i]) + s_bias[96 + i];
-    }
-  }
-  const float vmax = selv[0];
-  float z = 0.f;
-#pragma unroll
-  for (int i = 0; i < 128; ++i) {
-    v[i] = (i < E) ? __expf(v[i] - vmax) : 0.f;
-    z += v[i];
-  }
   const float rz = valid ? 1.f / z : 0.f;
-#pragma unroll
+#pragma unroll 1
   for (int c = 0; c < 4; ++c) {
     if (c * 32 < E) {
       float pc[32];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) pc[i] = v[c * 32 + i] * rz;
+      for (int q = 0; q < 8; ++q) {
+        const float4 w = lds_f4(vals + (c * 8 + q) * PITCH);
+        pc[4 * q + 0] = w.x * rz;
+        pc[4 * q + 1] = w.y * rz;
+        pc[4 * q + 2] = w.z * rz;
+        pc[4 * q + 3] = w.w * rz;
+      }
+      // column sums over the 32 tokens of this warp: butterfly transpose-reduce, lane L ends with column L
 #pragma unroll
       for (int off = 16, cnt = 16; off >= 1; off >>= 1, cnt >>= 1) {
 #pragma unroll
@@ -702,14 +753,15 @@ __device__ __forceinline__ void routing_epilogue_regs(const GemmParams& p, const
     }
   }
   if (valid) {
-    float zs = 0.f;
-    for (int j = 0; j < k; ++j) zs += __expf(selv[j] - vmax);
     const float rzs = 1.f / zs;
+#pragma unroll 1
     for (int j = 0; j < k; ++j) {
-      const float g = __expf(selv[j] - vmax) * rzs;
-      p.idx[tok * k + j] = seli[j];
+      uint32_t exb, col;
+      asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(exb), "=r"(col) : "r"(picks + j * (128 * 8)));
+      const float g = __uint_as_float(exb) * rzs;
+      p.idx[tok * k + j] = static_cast<int32_t>(col);
       p.gates[tok * k + j] = g;
-      p.idx_out[tok * k + j] = seli[j];
+      p.idx_out[tok * k + j] = static_cast<int32_t>(col);
       p.gates_out[tok * k + j] = g;
     }
   }

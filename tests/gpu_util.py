@@ -22,6 +22,27 @@ def rel_fro(got: np.ndarray, ref: np.ndarray) -> float:
     return float(num / den) if den > 0 else float(num)
 
 
+def rows_max_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """Largest error of any single row: max_r |got_r - ref_r| / max(|ref_r|, rms_r' |ref_r'|) (2-norms over the last
+    axis).  A whole-tensor norm hides a wrong row among thousands; this does not.  Each row is measured against its own
+    size, except that rows much smaller than the typical row are measured against the typical row (their rounding
+    errors are set by the operands, not by their own cancelled sum)."""
+    got = got.astype(np.float64).reshape(-1, got.shape[-1])
+    ref = ref.astype(np.float64).reshape(-1, ref.shape[-1])
+    if ref.shape[0] == 0:
+        return 0.0
+    num = np.linalg.norm(got - ref, axis=1)
+    own = np.linalg.norm(ref, axis=1)
+    rms = np.sqrt(np.mean(own * own))
+    den = np.maximum(own, rms)
+    if rms == 0:
+        return float(num.max())
+    return float((num / den).max())
+
+
+ROW_TOL = 3e-2  # bound on rows_max_err: about ten bf16 roundings' worth, far below the O(1) of a wrong row
+
+
 class Run:
     """Runs the CUDA layer on an instance from synth.make_inputs and keeps the device tensors."""
 

@@ -9,7 +9,7 @@ import pytest
 import torch
 
 from paper_2608_00916_b200 import synth
-from gpu_util import Run, from_dev_bf16, oracle_run, rel_fro
+from gpu_util import ROW_TOL, Run, from_dev_bf16, oracle_run, rel_fro, rows_max_err
 from paper_2608_00916_b200.binding import MoELayer
 from oracle import moe_oracle as orc
 
@@ -38,8 +38,10 @@ def check_all(r: Run, ofw, obw, d_aux, stages=True):
             got, pad = r.rows(nm, w)
             ref = ofw[nm] * g_row if nm in ("act", "o") else ofw[nm]
             assert rel_fro(got, ref) <= (0.0 if nm == "xp" else TOL), nm
+            assert rows_max_err(got, ref) <= ROW_TOL, nm
             assert not pad.any(), f"pad rows of {nm} are not zero"
     assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+    assert rows_max_err(from_dev_bf16(fw["y"]), ofw["y"]) <= ROW_TOL  # no single token row is wrong
     bw = r.backward(d_aux)
     if stages:
         assert rel_fro(r.layer.buffer("dg", torch.float32).cpu().numpy().reshape(-1, k), obw["dg"]) <= TOL
@@ -48,11 +50,17 @@ def check_all(r: Run, ofw, obw, d_aux, stages=True):
         for nm, w, ref in (("o", d, dy_rows), ("dhg", f, obw["dhg"]), ("dhu", f, obw["dhu"]), ("dxp", d, obw["dxp"])):
             got, pad = r.rows(nm, w)
             assert rel_fro(got, ref) <= (0.0 if nm == "o" else TOL), nm
+            assert rows_max_err(got, ref) <= ROW_TOL, nm
             assert not pad.any(), f"pad rows of {nm} (backward) are not zero"
         assert rel_fro(r.layer.buffer("dl", torch.float32).cpu().numpy().reshape(-1, E), obw["dl"]) <= TOL
     for nm in ("dx", "dW_gate", "dW_up", "dW_down"):
         assert rel_fro(from_dev_bf16(bw[nm]), obw[nm]) <= TOL, nm
+        assert rows_max_err(from_dev_bf16(bw[nm]), obw[nm]) <= ROW_TOL, nm
     assert rel_fro(bw["dW_r"].cpu().numpy(), obw["dW_r"]) <= TOL
+    assert rows_max_err(bw["dW_r"].cpu().numpy(), obw["dW_r"]) <= ROW_TOL
+    # dW_r against the float64 host contraction of x with the ORACLE's dl (not with the library's own dl)
+    ref_dwr = synth.bf16_bits_to_f64(r.inp["x"]).T @ obw["dl"]
+    assert rel_fro(bw["dW_r"].cpu().numpy(), ref_dwr) <= TOL
     assert rel_fro(bw["db_r"].cpu().numpy(), obw["db_r"]) <= TOL
     # per-expert slabs
     for nm in ("dW_gate", "dW_up", "dW_down"):
