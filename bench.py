@@ -394,10 +394,14 @@ def main():
                     reducer.wait()
                 for t in acc.values():
                     t.zero_()
-            layer.backward_accumulate(tens["dy"], inp["d_aux"], acc)
+            last = (step_no[0] + 1) % window == 0
+            # the window's last micro-batch runs its weight gradients in ranges of experts and signals each range, so
+            # that the sum over the ranks of a finished range overlaps the rest of this backward pass
+            layer.backward_accumulate(tens["dy"], inp["d_aux"], acc,
+                                      group_events=reducer.events() if (reducer is not None and last) else None)
             step_no[0] += 1
-            if reducer is not None and step_no[0] % window == 0:
-                reducer.start([acc["dW_gate"], acc["dW_up"], acc["dW_down"], acc["dW_r"]])
+            if reducer is not None and last:
+                reducer.start_grouped(acc)
         else:
             layer.backward(tens["dy"], inp["d_aux"], grads=grads)
 
@@ -553,7 +557,8 @@ def main():
             "config": {"workload": args.workload, "mode": args.mode, "T_per_gpu": T, "d": shape.d, "E": shape.E, "top_k": shape.k,
                        "f": shape.f,
                        "parallelism": f"dp{world} over tokens, experts replicated (EP=1), "
-                                      + ("weight gradients all-reduced once per accumulation window"
+                                      + ("weight gradients all-reduced once per accumulation window, range by range "
+                                         "of experts while the backward pass still runs"
                                          if reducer is not None else "no data-path collective"),
                        "conditioning": f"{cond_steps} untimed steps (>= {args.condition_seconds} s) before the timed region",
                        "l2": l2_note,

@@ -198,6 +198,24 @@ MOE_API moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16
                                            float* db_r, float* dW_gate, float* dW_up, float* dW_down,
                                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* moe_backward_accumulate for data-parallel training, where the weight gradients must be summed over the ranks (the
+ * paper's Megatron backend: DP = world / (TP x PP), gradients reduced into the distributed optimizer's buffers; Section
+ * "Megatron backend").  The two weight-gradient GEMMs run as n_groups launches over consecutive ranges of
+ * ceil(E / n_groups) experts, and the library records, on cuda_stream, the caller's events
+ *     group_events[g]             when dW_down[range g] is complete           (g = 0 .. n_groups - 1)
+ *     group_events[n_groups + g]  when dW_gate[range g] and dW_up[range g] are complete
+ * (host array of 2 * n_groups cudaEvent_t handles).  A caller makes its communication stream wait for an event and
+ * all-reduces that range's slab while the remaining weight-gradient launches, the dgrad GEMM between them and the
+ * router's chain still run: the reduction overlaps the backward pass instead of following it.  Results are those of
+ * moe_backward_accumulate (within a range the experts run in index order, not largest first). */
+MOE_API moe_status moe_backward_accumulate_grouped(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux,
+                                                   const uint16_t* x, const uint16_t* W_r, const uint16_t* W_gate,
+                                                   const uint16_t* W_up, const uint16_t* W_down, uint16_t* dx,
+                                                   float* dW_r, float* db_r, float* dW_gate, float* dW_up,
+                                                   float* dW_down, int32_t n_groups,
+                                                   void* const* group_events /* host */, void* workspace,
+                                                   size_t workspace_bytes, void* cuda_stream);
+
 /* Expert LoRA: the same layer with frozen expert weights and trainable rank-r adapters on the experts' fc1 (gate | up)
  * and fc2 (down) - the paper's "moe_experts" LoRA target group (experts.*.linear_fc1, experts.*.linear_fc2; Section
  * "LoRA target groups for MoE").  Effective weights:

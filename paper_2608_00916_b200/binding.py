@@ -24,7 +24,8 @@ EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_fi
            "moe_step_host_begin", "moe_step_host_end", "moe_kernel_launches", "moe_ctx_device",
            "moe_e2e_workspace_offset", "moe_ep_create", "moe_ep_send_workspace_bytes", "moe_ep_own_workspace_bytes",
            "moe_ep_workspace_find", "moe_ep_route", "moe_ep_plan", "moe_ep_dispatch", "moe_ep_expert_forward",
-           "moe_ep_combine", "moe_ep_expert_backward", "moe_ep_router_backward"]
+           "moe_ep_combine", "moe_ep_expert_backward", "moe_ep_router_backward",
+           "moe_backward_accumulate_grouped"]
 EP_MAX_RANKS = 16  # MOE_EP_MAX_RANKS of include/moe.h
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
@@ -75,6 +76,8 @@ def load_library() -> C.CDLL:
     lib.moe_backward.restype = C.c_int
     lib.moe_backward_accumulate.argtypes = lib.moe_backward.argtypes
     lib.moe_backward_accumulate.restype = C.c_int
+    lib.moe_backward_accumulate_grouped.argtypes = [vp, i64, vp, C.c_float] + [vp] * 11 + [C.c_int32, C.POINTER(vp), vp, sz, vp]
+    lib.moe_backward_accumulate_grouped.restype = C.c_int
     lib.moe_step_host_begin.argtypes = [vp, C.c_int, i64, vp, vp, C.c_float, vp, vp, vp, vp, sz, vp]
     lib.moe_step_host_begin.restype = C.c_int
     lib.moe_step_host_end.argtypes = [vp, C.c_int]
@@ -272,9 +275,11 @@ class MoELayer:
         _check(self.lib, rc, "moe_backward")
         return out
 
-    def backward_accumulate(self, dy, d_aux: float, acc):
+    def backward_accumulate(self, dy, d_aux: float, acc, group_events=None):
         """Backward of the last forward() that adds the weight gradients into the fp32 tensors of `acc`
-        (keys dW_r [d,E], dW_gate, dW_up [E,d,f], dW_down [E,f,d], optional db_r [E]); returns dx."""
+        (keys dW_r [d,E], dW_gate, dW_up [E,d,f], dW_down [E,f,d], optional db_r [E]); returns dx.
+        group_events: 2 n torch.cuda.Event objects; the weight gradients then run in n ranges of experts and event g
+        (n + g) is recorded when dW_down (dW_gate and dW_up) of range g is complete."""
         import torch
         if self._saved is None:
             raise MoEError("backward_accumulate() needs a preceding training forward()")
@@ -284,6 +289,19 @@ class MoELayer:
                        ("dW_down", (self.E, self.f, self.d))):
             assert acc[n].dtype == torch.float32 and tuple(acc[n].shape) == shp and acc[n].is_contiguous(), n
         dx = torch.empty(T, self.d, dtype=torch.bfloat16, device=x.device)
+        if group_events is not None:
+            n = len(group_events) // 2
+            assert len(group_events) == 2 * n and n >= 1
+            for ev in group_events:
+                if ev.cuda_event == 0:  # torch creates the CUDA event lazily, at the first record
+                    ev.record(torch.cuda.current_stream())
+            evs = (C.c_void_p * (2 * n))(*[C.c_void_p(ev.cuda_event) for ev in group_events])
+            rc = self.lib.moe_backward_accumulate_grouped(
+                self.h, T, _ptr(dy), C.c_float(d_aux), _ptr(x), _ptr(W_r), _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(dx),
+                _ptr(acc["dW_r"]), _ptr(acc.get("db_r")), _ptr(acc["dW_gate"]), _ptr(acc["dW_up"]), _ptr(acc["dW_down"]), n,
+                evs, _ptr(self.ws), self.ws.numel(), self._stream())
+            _check(self.lib, rc, "moe_backward_accumulate_grouped")
+            return dx
         rc = self.lib.moe_backward_accumulate(self.h, T, _ptr(dy), C.c_float(d_aux), _ptr(x), _ptr(W_r), _ptr(W_gate),
                                               _ptr(W_up), _ptr(W_down), _ptr(dx), _ptr(acc["dW_r"]), _ptr(acc.get("db_r")),
                                               _ptr(acc["dW_gate"]), _ptr(acc["dW_up"]), _ptr(acc["dW_down"]),

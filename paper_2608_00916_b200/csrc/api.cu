@@ -441,12 +441,15 @@ size_t moe_inference_workspace_bytes(const moe_ctx* ctx, int64_t T) {
 }
 
 // acc_* non-null: accumulate mode (fp32 weight-gradient buffers are added to; dW_r / db_r are added to as well)
+// n_groups > 0 (accumulate mode): the weight gradients are computed in n_groups launches over consecutive ranges of
+// experts and group_events[g] / group_events[n_groups + g] are recorded on the stream when the dW_down / the dW_gate and
+// dW_up slabs of range g are complete.
 static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
                                 const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
                                 const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,
                                 uint16_t* dW_up, uint16_t* dW_down, float* acc_gate, float* acc_up, float* acc_down,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream,
-                                const LoraArgs* lora = nullptr) {
+                                const LoraArgs* lora = nullptr, int n_groups = 0, void* const* group_events = nullptr) {
   const bool accumulate = acc_gate != nullptr;
   if (!ctx || T < 0) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
@@ -534,9 +537,25 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     if (rc != MOE_OK) return rc;
     rc = router_chain();
     if (rc != MOE_OK) return rc;
+    // weight gradients: one launch, or one per range of experts with an event after each
+    auto wgrad = [&](GemmKind kind, int ev_base) -> moe_status {
+      if (n_groups <= 0) return launch_grouped_gemm(c, kind, T, L, ws, io, st);
+      const int per = (s.E + n_groups - 1) / n_groups;
+      for (int g = 0; g < n_groups; ++g) {
+        GemmIO gio = io;
+        gio.e_first = g * per;
+        gio.e_count = s.E - gio.e_first < per ? s.E - gio.e_first : per;
+        if (gio.e_count > 0) {
+          const moe_status r2 = launch_grouped_gemm(c, kind, T, L, ws, gio, st);
+          if (r2 != MOE_OK) return r2;
+        }
+        if (cudaEventRecord(static_cast<cudaEvent_t>(group_events[ev_base + g]), st) != cudaSuccess) return MOE_ERR_CUDA;
+      }
+      return MOE_OK;
+    };
     {
       StageTimer tm(c, st, 7);
-      rc = launch_grouped_gemm(c, GEMM_B3, T, L, ws, io, st);
+      rc = wgrad(GEMM_B3, 0);
     }
     if (rc != MOE_OK) return rc;
     if (T > 0) {
@@ -546,7 +565,7 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     if (rc != MOE_OK) return rc;
     {
       StageTimer tm(c, st, 9);
-      rc = launch_grouped_gemm(c, GEMM_B5, T, L, ws, io, st);
+      rc = wgrad(GEMM_B5, n_groups);
     }
     if (rc != MOE_OK) return rc;
   }
@@ -581,6 +600,20 @@ moe_status moe_backward_accumulate(moe_ctx* ctx, int64_t T, const uint16_t* dy, 
   if (!dW_gate || !dW_up || !dW_down) return MOE_ERR_INVALID_ARG;
   return backward_impl(ctx, T, dy, d_aux, x, W_r, W_gate, W_up, W_down, dx, dW_r, db_r, nullptr, nullptr, nullptr, dW_gate,
                        dW_up, dW_down, workspace, workspace_bytes, cuda_stream);
+}
+
+moe_status moe_backward_accumulate_grouped(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
+                                           const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
+                                           const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r,
+                                           float* dW_gate, float* dW_up, float* dW_down, int32_t n_groups,
+                                           void* const* group_events, void* workspace, size_t workspace_bytes,
+                                           void* cuda_stream) {
+  if (!dW_gate || !dW_up || !dW_down || !ctx || n_groups < 1 || !group_events) return MOE_ERR_INVALID_ARG;
+  if (n_groups > reinterpret_cast<moe_ctx_impl*>(ctx)->s.E) return MOE_ERR_INVALID_ARG;
+  for (int g = 0; g < 2 * n_groups; ++g)
+    if (!group_events[g]) return MOE_ERR_INVALID_ARG;
+  return backward_impl(ctx, T, dy, d_aux, x, W_r, W_gate, W_up, W_down, dx, dW_r, db_r, nullptr, nullptr, nullptr, dW_gate,
+                       dW_up, dW_down, workspace, workspace_bytes, cuda_stream, nullptr, n_groups, group_events);
 }
 
 // ------------------------------------------------------------------------------------------ expert LoRA

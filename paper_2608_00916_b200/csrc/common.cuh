@@ -162,6 +162,7 @@ struct GemmIO {
   uint16_t* dW_up = nullptr;
   uint16_t* dW_down = nullptr;
   uint16_t* dx = nullptr;
+  int e_first = 0, e_count = 0;  // weight gradients: e_count > 0 restricts the launch to experts [e_first, e_first + e_count)
   float* dW_gate_acc = nullptr;  // accumulate mode: fp32 buffers the weight gradients are added to
   float* dW_up_acc = nullptr;
   float* dW_down_acc = nullptr;

@@ -30,12 +30,14 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
     grouped_gemm_kernel(const __grid_constant__ GemmParams p) {
   using TR = Traits<KIND>;
   constexpr int EPI_WARPS = (KIND == GEMM_RT) ? 4 : 8;
-  // the routing kind runs a three-stage ring (it streams x once, 16 KB per stage) and uses the rest of the dynamic
-  // shared memory (the fourth stage and the staging units: 80 KB) as scratch of its routing epilogue
-  constexpr int NST = (KIND == GEMM_RT) ? 3 : STAGES;
-  static_assert(STAGE_BYTES + EPI_BYTES >= ROUTE_SCRATCH_BYTES, "routing scratch does not fit");
+  constexpr int NST = STAGES;
+  // The routing kind with E <= 128 stages only 32 KB per K block (16 KB of x, 16 KB of W_r): its stages are packed at
+  // that stride and the 96 KB this frees hold the scratch of its routing epilogue (80 KB) and the picks (16 KB).
+  constexpr uint32_t RT_STAGE_BYTES = A_BYTES + 2 * CHUNK_BYTES;
+  static_assert(STAGES * RT_STAGE_BYTES + ROUTE_SCRATCH_BYTES + 128 * ROUTE_SMEM_MAX_K * 8 <= STAGES * STAGE_BYTES + EPI_BYTES,
+                "routing scratch does not fit");
   extern __shared__ unsigned char gemm_smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];  // full, empty, accumulator full / empty, drain (failure path)
   __shared__ uint32_t tmem_base_slot;
   __shared__ float s_bias[KIND == GEMM_RT ? MAX_E : 1];  // router bias (zero beyond E)
   if (KIND == GEMM_RT)
@@ -43,6 +45,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(gemm_smem_raw) + 1023u) & ~1023u;
+  const uint32_t stage_stride = (KIND == GEMM_RT && p.b_chunks <= 2) ? RT_STAGE_BYTES : STAGE_BYTES;
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -58,6 +61,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       mbar_init(tfull_bar(a), 1);
       mbar_init(tempty_bar(a), 32 * EPI_WARPS);
     }
+    mbar_init(bar0 + 8u * (2 * STAGES + 4), 1);
     fence_mbar_init();
     tma_prefetch_desc(&p.mapA0);
     tma_prefetch_desc(&p.mapB0);
@@ -90,7 +94,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
           break;
         }
         t_wait += clock64() - w0;
-        const uint32_t sA = smem_base + s * STAGE_BYTES;
+        const uint32_t sA = smem_base + s * stage_stride;
         if (lane == 0) {
           mbar_expect_tx(full_bar(s), p.stage_tx);
           issue_loads<KIND>(p, tl, kb, sA, sA + A_BYTES, full_bar(s));
@@ -102,8 +106,11 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       atomicAdd(p.timers + 0, static_cast<unsigned long long>(clock64() - t_begin));  // producer: total
       atomicAdd(p.timers + 1, static_cast<unsigned long long>(t_wait));               // producer: waiting for a free stage
     }
-    if (!ok && lane == 0) {
-      record_status(p.status, DEV_TIMEOUT, 100 + KIND);
+    if (!ok) {
+      // gave up: the copies already issued still land in this CTA's shared memory - wait for them (bounded again)
+      // before the CTA may exit
+      if (lane == 0) record_status(p.status, DEV_TIMEOUT, 100 + KIND);
+      for (uint32_t i = it > static_cast<uint32_t>(NST) ? it - NST : 0; i < it; ++i) mbar_wait(full_bar(i % NST), (i / NST) & 1u);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -140,7 +147,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
         t_full += clock64() - w1;
         tc_fence_after();
         if (lane == 0) {
-          const uint32_t sA = smem_base + s * STAGE_BYTES;
+          const uint32_t sA = smem_base + s * stage_stride;
           const uint32_t sB = sA + A_BYTES;
 #pragma unroll
           for (int ks = 0; ks < BK / 16; ++ks) {
@@ -160,8 +167,14 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
       atomicAdd(p.timers + 3, static_cast<unsigned long long>(t_acc));                // waiting for a drained accumulator
       atomicAdd(p.timers + 4, static_cast<unsigned long long>(t_full));               // waiting for operands
     }
-    if (!ok && lane == 0) {
-      record_status(p.status, DEV_TIMEOUT, 200 + KIND);
+    if (!ok) {
+      // gave up: let every MMA issued so far finish (bounded) before the tensor memory is freed
+      if (lane == 0) {
+        record_status(p.status, DEV_TIMEOUT, 200 + KIND);
+        umma_commit(bar0 + 8u * (2 * STAGES + 4));
+      }
+      __syncwarp();
+      mbar_wait(bar0 + 8u * (2 * STAGES + 4), 0u);
     }
   } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------------------------ epilogue (128 TMEM lanes; two warps per
@@ -210,9 +223,10 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
                               TR::WGRAD ? p.M_total - (tl.m0 + ew * 32) : (KIND == GEMM_DX ? static_cast<int>(p.T - tl.row0 - ew * 32) : 32),
                               es, lane, half, NHALF);
       } else if (KIND == GEMM_RT) {
-        if (p.N_total <= 128 && p.top_k <= ROUTE_SMEM_MAX_K)  // picks live in the unused tail of stage 0 (B is <= 16 KB)
-          routing_epilogue_smem(p, s_bias, smem_base + NST * STAGE_BYTES, smem_base + A_BYTES + 2 * CHUNK_BYTES, row,
-                                tl.row0 / BM, ew, taddr, lane);
+        if (p.N_total <= 128 && p.top_k <= ROUTE_SMEM_MAX_K)
+          routing_epilogue_smem(p, s_bias, smem_base + STAGES * RT_STAGE_BYTES,
+                                smem_base + STAGES * RT_STAGE_BYTES + ROUTE_SCRATCH_BYTES, row, tl.row0 / BM, ew, taddr,
+                                lane);
         else
           routing_epilogue_tmem(p, s_bias, row, tl.row0 / BM, ew, taddr, lane);
       } else if (KIND == GEMM_DWR) {
@@ -342,6 +356,11 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
   p.tile_list = part == 2 ? reinterpret_cast<const int32_t*>(ws + L.single_tab) : nullptr;
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
+  if ((kind == GEMM_B3 || kind == GEMM_B5) && io.e_count > 0) {  // one group of experts, in index order
+    p.E = io.e_count;
+    p.e_first = io.e_first;
+    p.expert_grouped = 1;
+  }
   p.b_chunks = 4;
   p.mma_n = BN;
   p.stage_tx = STAGE_BYTES;

@@ -44,7 +44,7 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
   if (Traits<KIND>::WGRAD) {
     const int per = p.m_tiles * p.n_tiles;
     const int slot = t / per;
-    tl.e = p.expert_order[slot];  // longest K loops first
+    tl.e = p.expert_grouped ? p.e_first + slot : p.expert_order[slot];  // else: longest K loops first
     const int rem = t - slot * per;
     tl.m0 = (rem / p.n_tiles) * 2 * BM + rank * BM;
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
@@ -110,7 +110,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
     grouped_gemm_pair_kernel(const __grid_constant__ GemmParams p) {
   using TR = Traits<KIND>;
   extern __shared__ unsigned char gemm2_smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES2 + 4];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES2 + 5];  // full, empty, accumulator full / empty, drain (failure path)
   __shared__ uint32_t tmem_base_slot;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -132,6 +132,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       mbar_init(tfull_bar(a), 1);   // one commit from the leader's MMA thread
       mbar_init(tempty_bar(a), 16);  // used in the leader only: 8 epilogue warps of each CTA
     }
+    mbar_init(bar0 + 8u * (2 * STAGES2 + 4), 1);
     fence_mbar_init();
     tma_prefetch_desc(&p.mapA0);
     tma_prefetch_desc(&p.mapB0);
@@ -178,8 +179,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
       atomicAdd(p.timers + 0, static_cast<unsigned long long>(clock64() - t_begin));
       atomicAdd(p.timers + 1, static_cast<unsigned long long>(t_wait));
     }
-    if (!ok && lane == 0) {
-      record_status(p.status, DEV_TIMEOUT, 1100 + KIND);
+    if (!ok) {
+      // gave up: the leader waits (bounded) for the copies of BOTH CTAs that were already issued - they are all credited
+      // to its full barriers - so that neither CTA exits with copies in flight (the cluster barrier below holds the
+      // partner until then)
+      if (lane == 0) record_status(p.status, DEV_TIMEOUT, 1100 + KIND);
+      if (leader)
+        for (uint32_t i = it > static_cast<uint32_t>(STAGES2) ? it - STAGES2 : 0; i < it; ++i)
+          mbar_wait(full_bar(i % STAGES2), (i / STAGES2) & 1u);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
@@ -240,8 +247,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
         atomicAdd(p.timers + 3, static_cast<unsigned long long>(t_acc));
         atomicAdd(p.timers + 4, static_cast<unsigned long long>(t_full));
       }
-      if (!ok && lane == 0) {
-        record_status(p.status, DEV_TIMEOUT, 1200 + KIND);
+      if (!ok) {
+        // gave up: let every MMA issued so far finish (bounded) before the pair's tensor memory is freed
+        if (lane == 0) {
+          record_status(p.status, DEV_TIMEOUT, 1200 + KIND);
+          umma_commit_pair_both(bar0 + 8u * (2 * STAGES2 + 4));
+        }
+        __syncwarp();
+        mbar_wait(bar0 + 8u * (2 * STAGES2 + 4), 0u);
       }
     }
   } else {

@@ -38,7 +38,9 @@ struct GemmParams {
   unsigned long long* timers;  // null, or 8 counters of this kind: summed over CTAs (see gemm.cu)
   int n_tiles;   // output tiles along N
   int m_tiles;   // weight gradients: output tiles along M per expert
-  int E;
+  int E;         // weight gradients: number of experts this launch covers
+  int e_first;   // weight gradients: first expert of the launch when it covers a range (expert_grouped), else unused
+  int expert_grouped;  // weight gradients: 1 = experts e_first .. e_first + E - 1 in index order, 0 = all, largest first
   int k_blocks;  // row GEMMs: K blocks per segment
   int nseg;      // row GEMMs: K segments of k_blocks blocks (B4, DX: up to 2)
   int k_blocks1; // row GEMMs: K blocks of the extra segment that follows them (0: none)
@@ -116,7 +118,7 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     const int rem = t - tl.e * per;
     tl.m0 = (rem / p.n_tiles) * BM;
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
-    if (KIND != GEMM_DWR) tl.e = p.expert_order[tl.e];  // longest K loops first
+    if (KIND != GEMM_DWR) tl.e = p.expert_grouped ? p.e_first + tl.e : p.expert_order[tl.e];  // else: longest K loops first
     if (KIND == GEMM_DWR) {  // "expert" = token slice
       tl.row0 = tl.e * p.split_rows;
       tl.nkb = max(0, min(p.split_rows, p.rows_total - tl.row0)) / BK;

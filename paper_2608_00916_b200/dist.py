@@ -103,17 +103,36 @@ class GradAllReducer:
     """Sums the weight-gradient buffers of the data-parallel ranks (the one exchange step of the sharded layer: tokens
     are split over the ranks, experts are replicated, so dW_gate / dW_up / dW_down / dW_r must be added up).
 
-    The buffers (fp32, as filled by MoELayer.backward_accumulate) are cut along the expert axis into buckets; each
-    bucket is all-reduced asynchronously on the process group (NCCL over NVLink on GPUs, gloo on CPU).  start() may be
-    called as soon as the kernels that write the buffers have been enqueued: on CUDA it makes a side stream wait for an
-    event recorded on the compute stream, so the reduction overlaps whatever the compute stream runs next (the router
-    gradient and the unpermute); wait() joins before the optimizer reads the buffers.  With one rank both are no-ops."""
+    Two ways to start the reduction of the fp32 buffers filled by MoELayer.backward_accumulate:
 
-    def __init__(self, experts_per_bucket: int = 16):
+    * start_grouped(acc, events): for a backward pass that ran with `group_events=events` (see events()).  The library
+      records an event as soon as a range of experts has its final dW_down (then dW_gate / dW_up); the communication
+      stream waits for exactly that event and all-reduces the range's slab, so the reduction of the first ranges runs
+      while the later weight-gradient launches, the dgrad GEMM between them and the router's chain are still
+      computing.  dW_r, which is complete only at the end of the pass, goes last.
+    * start(tensors): whole buffers, cut along the expert axis into buckets, after everything has been enqueued (the
+      reduction then overlaps only what follows the backward pass).  Also the form for CPU tensors (gloo).
+
+    wait() joins before the optimizer reads the buffers.  With one rank both are no-ops unless a `reduce_fn` is given
+    (tests inject one to watch the stream plumbing on a single GPU)."""
+
+    def __init__(self, experts_per_bucket: int = 16, n_groups: int = 4, reduce_fn=None):
         self.experts_per_bucket = max(1, int(experts_per_bucket))
+        self.n_groups = max(1, int(n_groups))
+        self.reduce_fn = reduce_fn
         self._work = []
         self._side = None
         self._done = None
+        self._events = None
+
+    def _active(self) -> bool:
+        return _state["world"] > 1 or self.reduce_fn is not None
+
+    def _reduce(self, t):
+        if self.reduce_fn is not None:
+            return self.reduce_fn(t)
+        import torch.distributed as dist
+        return dist.all_reduce(t, op=dist.ReduceOp.SUM, async_op=True)
 
     def buckets(self, tensors):
         """(tensor, first expert, last expert + 1) slices in launch order; tensors without an expert axis (dW_r) last."""
@@ -127,11 +146,50 @@ class GradAllReducer:
                 out.append((t, 0, t.shape[0]))
         return out
 
-    def start(self, tensors) -> None:
-        if _state["world"] <= 1:
+    def group_ranges(self, E: int):
+        """Expert ranges of the grouped backward pass: n_groups ranges of ceil(E / n_groups) experts (the last may be
+        shorter or empty), the split moe_backward_accumulate_grouped uses."""
+        per = (E + self.n_groups - 1) // self.n_groups
+        return [(min(E, g * per), min(E, (g + 1) * per)) for g in range(self.n_groups)]
+
+    def events(self):
+        """The 2 n_groups CUDA events to hand to MoELayer.backward_accumulate(..., group_events=...)."""
+        import torch
+        if self._events is None:
+            self._events = [torch.cuda.Event() for _ in range(2 * self.n_groups)]
+        return self._events
+
+    def start_grouped(self, acc: dict) -> None:
+        """acc: the dict given to backward_accumulate (dW_gate, dW_up, dW_down, dW_r)."""
+        if not self._active():
             return
         import torch
-        import torch.distributed as dist
+        if self._side is None:
+            self._side = torch.cuda.Stream()
+        ev = self.events()
+        n = self.n_groups
+        ranges = self.group_ranges(acc["dW_down"].shape[0])
+        tail = torch.cuda.Event()
+        tail.record(torch.cuda.current_stream())  # everything of the pass, dW_r included, has been enqueued
+        with torch.cuda.stream(self._side):
+            for g, (e0, e1) in enumerate(ranges):
+                self._side.wait_event(ev[g])
+                if e1 > e0:
+                    self._work.append(self._reduce(acc["dW_down"][e0:e1]))
+            for g, (e0, e1) in enumerate(ranges):
+                self._side.wait_event(ev[n + g])
+                if e1 > e0:
+                    self._work.append(self._reduce(acc["dW_gate"][e0:e1]))
+                    self._work.append(self._reduce(acc["dW_up"][e0:e1]))
+            self._side.wait_event(tail)
+            self._work.append(self._reduce(acc["dW_r"]))
+            self._done = torch.cuda.Event()
+            self._done.record(self._side)
+
+    def start(self, tensors) -> None:
+        if not self._active():
+            return
+        import torch
         on_cuda = tensors[0].is_cuda
         if on_cuda:
             if self._side is None:
@@ -142,7 +200,7 @@ class GradAllReducer:
         ctx = torch.cuda.stream(self._side) if on_cuda else _NullCtx()
         with ctx:
             for t, e0, e1 in self.buckets(tensors):
-                self._work.append(dist.all_reduce(t[e0:e1], op=dist.ReduceOp.SUM, async_op=True))
+                self._work.append(self._reduce(t[e0:e1]))
             if on_cuda:
                 self._done = torch.cuda.Event()
                 self._done.record(self._side)
@@ -150,7 +208,8 @@ class GradAllReducer:
     def wait(self) -> None:
         import torch
         for w in self._work:
-            w.wait()
+            if w is not None:
+                w.wait()
         self._work = []
         if self._done is not None:
             torch.cuda.current_stream().wait_event(self._done)

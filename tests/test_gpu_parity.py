@@ -567,3 +567,41 @@ def test_full_coarse_config_sampled():
 @pytest.mark.parametrize("name", ["sweep_T1000", "sweep_T4096", "sweep_T8191", "sweep_T32768", "sweep_T65536"])
 def test_sweep_sampled(name):
     sampled_parity(name, n_tokens=24)
+
+
+def test_grouped_weight_gradients_signal_ranges_of_experts():
+    """moe_backward_accumulate_grouped: the weight gradients run range by range of experts, an event fires after each
+    range, and the buffers end up bitwise as moe_backward_accumulate leaves them.  The reducer's side-stream plumbing
+    is watched on one GPU through an injected stand-in for the all-reduce (it doubles a slab once its event has fired):
+    every range must have been final before it was touched."""
+    from paper_2608_00916_b200 import dist as pdist
+    d, E, k, f = 256, 24, 4, 192
+    inp = synth.make_inputs(synth.MoEShape(1800, d, E, k, f), 71)
+    r = Run(inp, k)
+    r.forward()
+
+    def zeros():
+        return {"dW_r": torch.zeros(d, E, device="cuda"), "dW_gate": torch.zeros(E, d, f, device="cuda"),
+                "dW_up": torch.zeros(E, d, f, device="cuda"), "dW_down": torch.zeros(E, f, d, device="cuda")}
+    plain = zeros()
+    dx0 = r.layer.backward_accumulate(r.dev["dy"], 0.02, plain)
+    touched = []
+
+    def fake_all_reduce(t):
+        touched.append(tuple(t.shape))
+        t.mul_(2.0)  # on the communication stream, after the range's event
+        return None
+    red = pdist.GradAllReducer(n_groups=5, reduce_fn=fake_all_reduce)  # 24 experts -> ranges of 5, 5, 5, 5, 4
+    assert red.group_ranges(E) == [(0, 5), (5, 10), (10, 15), (15, 20), (20, 24)]
+    grouped = zeros()
+    r.forward()
+    dx1 = r.layer.backward_accumulate(r.dev["dy"], 0.02, grouped, group_events=red.events())
+    red.start_grouped(grouped)
+    red.wait()
+    torch.cuda.synchronize()
+    r.layer.poll()
+    assert all(ev.query() for ev in red.events())
+    assert torch.equal(dx0, dx1)
+    for n in plain:
+        assert torch.equal(grouped[n], 2.0 * plain[n]), n  # doubled exactly once, after the final value was there
+    assert touched == [(5, f, d)] * 4 + [(4, f, d)] + [(5, d, f)] * 8 + [(4, d, f)] * 2 + [(d, E)]
