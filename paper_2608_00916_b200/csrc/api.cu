@@ -385,7 +385,8 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
   {
     StageTimer tm(c, st, 1);
     launch_permute(s, T, L, ws, x, expert_counts, perm, aux_loss,
-                   static_cast<int>(router_psum_rows(s, T, logits_in != nullptr)), st);
+                   static_cast<int>(router_psum_rows(s, T, logits_in != nullptr)), st, /*tables_only=*/false,
+                   /*histogram_done=*/tc_router && T > 0 && router_writes_histogram(s));
   }
   if (T > 0) {
     {

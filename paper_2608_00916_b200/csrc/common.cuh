@@ -11,7 +11,9 @@
 namespace moe {
 
 constexpr int ROW_PAD = 128;     // every expert's row segment starts and ends on a multiple of this
-constexpr int TOK_TILE = 256;    // tokens per block in the histogram / scatter kernels (8 warps x 32)
+constexpr int TOK_TILE = 128;    // tokens per tile of the permutation (histogram / scatter blocks: 4 warps x 32); equal to
+                                 // the token tile of the tensor-core router, whose epilogue writes the tile histograms
+constexpr int TOK_WARPS = TOK_TILE / 32;
 constexpr int ROUTER_TOK = 16;   // tokens per block in the router kernel
 constexpr int MAX_E = 256;
 constexpr int MAX_K = 32;
@@ -126,7 +128,8 @@ void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t*
                    const float* logits_in, float* logits, int32_t* idx, float* gates, int32_t* idx_out,
                    float* gates_out, float* logits_out, float* psum_part, cudaStream_t st);
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
-                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only = false);
+                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only = false,
+                    bool histogram_done = false);
 // ---- launchers (combine.cu)
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
                     uint16_t* y, cudaStream_t st);
@@ -201,6 +204,8 @@ moe_status launch_lora_gemm(moe_ctx_impl* ctx, LoraOp op, int64_t T, const WsLay
 
 // true when the tensor-core router / dW_r / dx kernels apply (their TMA maps need E % 8 == 0)
 inline bool router_on_tensor_cores(const Shape& s) { return s.E % 8 == 0; }
+// true when that router's epilogue also writes the per-tile histograms of the permutation (its shared-memory form)
+inline bool router_writes_histogram(const Shape& s) { return router_on_tensor_cores(s) && s.E <= 128 && s.k <= 16; }
 // psum_part rows written by the router: one per warp of a 128-token tile (tensor cores) or per ROUTER_TOK tokens (SIMT)
 inline int64_t router_psum_rows(const Shape& s, int64_t T, bool logits_given) {
   return (router_on_tensor_cores(s) && !logits_given) ? 4 * ((T + 127) / 128) : (T + ROUTER_TOK - 1) / ROUTER_TOK;

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(256) ep_zero_pad_kernel(int d, const int32_t* 
 
 // ---------------------------------------------------------------------------------------------- dispatch
 // Destination row of every (token, slot) pair of this rank and its gate, stored next to that row on the owner.
-// Ranks inside a 256-token tile come from per-warp expert masks and population counts, as in the one-GPU scatter.
+// Ranks inside a token tile come from per-warp expert masks and population counts, as in the one-GPU scatter.
 __global__ void __launch_bounds__(TOK_TILE) ep_scatter_kernel(int64_t T, int E, int k, int E_loc,
                                                               const int32_t* __restrict__ idx,
                                                               const int32_t* __restrict__ tile_base,
@@ -87,10 +87,10 @@ __global__ void __launch_bounds__(TOK_TILE) ep_scatter_kernel(int64_t T, int E, 
                                                               const float* __restrict__ gates,
                                                               int32_t* __restrict__ inv, const EpPeers peers,
                                                               size_t row_gate_off) {
-  extern __shared__ uint32_t ep_masks[];  // [8][E]
+  extern __shared__ uint32_t ep_masks[];  // [TOK_WARPS][E]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t t = static_cast<int64_t>(blockIdx.x) * TOK_TILE + tid;
-  for (int i = tid; i < 8 * E; i += TOK_TILE) ep_masks[i] = 0u;
+  for (int i = tid; i < TOK_WARPS * E; i += TOK_TILE) ep_masks[i] = 0u;
   __syncthreads();
   if (t < T)
     for (int j = 0; j < k; ++j) atomicOr(&ep_masks[warp * E + idx[t * k + j]], 1u << lane);
@@ -311,7 +311,7 @@ moe_status moe_ep_route(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16
     if (rc != MOE_OK) return rc;
   }
   launch_permute(s, T, L, ws, x, counts_local, nullptr, aux_loss, static_cast<int>(router_psum_rows(s, T, false)), st,
-                 /*tables_only=*/true);
+                 /*tables_only=*/true, /*histogram_done=*/T > 0 && router_writes_histogram(s));
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -357,7 +357,7 @@ moe_status moe_ep_dispatch(moe_ctx* ctx, int64_t T, const uint16_t* src, int bac
   const int32_t* idx = reinterpret_cast<const int32_t*>(ws + l.send.idx);
   int32_t* inv = reinterpret_cast<int32_t*>(ws + l.send.inv);
   if (!backward) {
-    ep_scatter_kernel<<<static_cast<unsigned>(l.send.tok_tiles), TOK_TILE, sizeof(uint32_t) * 8 * s.E, st>>>(
+    ep_scatter_kernel<<<static_cast<unsigned>(l.send.tok_tiles), TOK_TILE, sizeof(uint32_t) * TOK_WARPS * s.E, st>>>(
         T, s.E, s.k, E_loc, idx, reinterpret_cast<const int32_t*>(ws + l.send.tile_counts),
         reinterpret_cast<const int32_t*>(ws + l.send.ep_dest), reinterpret_cast<const float*>(ws + l.send.gates), inv,
         peers, l.own.row_gate);

@@ -40,8 +40,12 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
   __shared__ __align__(8) uint64_t bars[2 * STAGES + 5];  // full, empty, accumulator full / empty, drain (failure path)
   __shared__ uint32_t tmem_base_slot;
   __shared__ float s_bias[KIND == GEMM_RT ? MAX_E : 1];  // router bias (zero beyond E)
+  __shared__ int s_hist[KIND == GEMM_RT ? 128 : 1];      // picks per expert of the tile (routing epilogue for E <= 128)
   if (KIND == GEMM_RT)
-    for (int i = threadIdx.x; i < MAX_E; i += blockDim.x) s_bias[i] = (p.bias && i < p.N_total) ? p.bias[i] : 0.f;
+    for (int i = threadIdx.x; i < MAX_E; i += blockDim.x) {
+      s_bias[i] = (p.bias && i < p.N_total) ? p.bias[i] : 0.f;
+      if (i < 128) s_hist[i] = 0;
+    }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(gemm_smem_raw) + 1023u) & ~1023u;
@@ -224,7 +228,7 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
                               es, lane, half, NHALF);
       } else if (KIND == GEMM_RT) {
         if (p.N_total <= 128 && p.top_k <= ROUTE_SMEM_MAX_K)
-          routing_epilogue_smem(p, s_bias, smem_base + STAGES * RT_STAGE_BYTES,
+          routing_epilogue_smem(p, s_bias, s_hist, smem_base + STAGES * RT_STAGE_BYTES,
                                 smem_base + STAGES * RT_STAGE_BYTES + ROUTE_SCRATCH_BYTES, row, tl.row0 / BM, ew, taddr,
                                 lane);
         else
@@ -353,6 +357,7 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
   } else {
     p.pair_count_slot = 2;
   }
+  p.oob_row = static_cast<int>(R);
   p.tile_list = part == 2 ? reinterpret_cast<const int32_t*>(ws + L.single_tab) : nullptr;
   p.status = reinterpret_cast<int32_t*>(ws + L.status);
   p.E = E;
@@ -467,6 +472,7 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       p.idx_out = io.idx_out;
       p.gates_out = io.gates_out;
       p.psum_part = reinterpret_cast<float*>(ws + L.psum_part);
+      p.tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);  // written by the shared-memory routing epilogue
       if (!ok) return MOE_ERR_CUDA;
       return launch_kind<GEMM_RT>(ctx, p, st);
     case GEMM_DX:
@@ -531,7 +537,11 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   }
   if (!row_kind) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 0);
   if (ctx->tile_mode == 1) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
-  if (ctx->tile_mode == 0 && rows_per_expert >= 512.0) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
+  // dgrad gate/up is the exception at short K: with 2 f / 64 < 64 K blocks per tile its pair form needs fewer cycles
+  // but more time under the power cap than its one-CTA form (Qwen3-30B-A3B shape: 842 vs 811 us in steady state)
+  const bool long_k = kind != GEMM_B4 || 2 * ctx->s.f / BK >= 64;
+  if (ctx->tile_mode == 0 && rows_per_expert >= 512.0 && long_k)
+    return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
   if (ctx->tile_mode != 3) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 0);
   const moe_status rc = launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 1);
   if (rc != MOE_OK) return rc;

@@ -14,8 +14,10 @@
 // leaves while its partner may still touch its shared memory, barriers or tensor memory.
 //
 // Row GEMMs pair two consecutive 128-row blocks of ONE expert; an expert with an odd number of blocks gets a pair
-// whose second half is empty: that CTA stages its half of B only, the MMA runs over whatever its A stage holds, and
-// nothing of its accumulator half is read or stored.  Weight gradients pair along M.
+// whose second half is empty: that CTA stages its half of B, and for A it issues the same TMA copy at a row beyond
+// the end of the row buffer, which the copy engine fills with zeros without touching memory - so the unavoidable MMA
+// over the empty half multiplies zeros (its power draw depends on the operand data, and the step is power-bound) -
+// and nothing of its accumulator half is read or stored.  Weight gradients pair along M.
 #include "gemm_common.cuh"
 
 namespace moe {
@@ -71,21 +73,21 @@ template <int KIND>
 __device__ __forceinline__ void issue_loads2(const GemmParams& p, const Tile2& tl, int kb, int rank, uint32_t sA,
                                              uint32_t sB, uint32_t bar) {
   if (KIND == GEMM_F3) {
-    if (tl.write) tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.write ? tl.row0 : p.oob_row);
     const CUtensorMap* mb = rank ? &p.mapB1 : &p.mapB0;  // leader: gate columns, partner: the matching up columns
 #pragma unroll
     for (int c = 0; c < 2; ++c) tma_load_3d_pair(sB + c * CHUNK_BYTES, mb, bar, tl.n0 + c * 64, kb * BK, tl.e);
   } else if (KIND == GEMM_F4) {
-    if (tl.write) tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.write ? tl.row0 : p.oob_row);
 #pragma unroll
     for (int c = 0; c < 2; ++c)
       tma_load_3d_pair(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + rank * 128 + c * 64, kb * BK, tl.e);
   } else if (KIND == GEMM_B2) {
-    if (tl.write) tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.row0);
+    tma_load_2d_pair(sA, &p.mapA0, bar, kb * BK, tl.write ? tl.row0 : p.oob_row);
     tma_load_3d_pair(sB, &p.mapB0, bar, kb * BK, tl.n0 + rank * 128, tl.e);
   } else if (KIND == GEMM_B4) {
     const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
-    if (tl.write) tma_load_2d_pair(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
+    tma_load_2d_pair(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.write ? tl.row0 : p.oob_row);
     tma_load_3d_pair(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0 + rank * 128, tl.e);
   } else if (KIND == GEMM_B3) {
     const int row = tl.row0 + kb * BK;
@@ -167,8 +169,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
         }
         t_wait += clock64() - w0;
         if (lane == 0) {
-          // the empty half of an odd expert's last pair loads no rows of A (its accumulator half is never read)
-          if (leader) mbar_expect_tx(full_bar(s), tl.full ? 2 * STAGE2_BYTES : 2 * STAGE2_BYTES - A_BYTES);
+          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
           const uint32_t sA = smem_base + s * STAGE2_BYTES;
           issue_loads2<KIND>(p, tl, kb, rank, sA, sA + A_BYTES, mapa_shared(full_bar(s), 0));
         }

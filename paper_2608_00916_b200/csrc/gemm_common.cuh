@@ -33,6 +33,7 @@ struct GemmParams {
   const int32_t* expert_order; // weight gradients: experts by row count, largest first
   const int32_t* pair_tab;     // CTA-pair kernels: per pair of row blocks {expert, first row, blocks (1|2), 0}
   int pair_count_slot;         // which entry of sched holds the number of entries of pair_tab
+  int oob_row;                 // a row index beyond the row buffers: TMA copies from there deliver zeros
   const int32_t* tile_list;    // one-CTA row GEMMs: null = every 128-row tile, else the tiles to compute (sched[4] entries)
   int32_t* status;
   unsigned long long* timers;  // null, or 8 counters of this kind: summed over CTAs (see gemm.cu)
@@ -71,6 +72,7 @@ struct GemmParams {
   float* gates;
   float* gates_out;
   float* psum_part;     // RT: [4 * tiles, E] per-warp column sums of p
+  int32_t* tile_counts; // RT: [tiles, E] histogram of the picks of every 128-token tile (null: not produced here)
   float* outf;          // DWR: [slices, d, E] fp32 partials; B2: [column tiles, rows_max] partial sums of dg
   float* accf0;         // B3, B5 in accumulate mode: fp32 weight-gradient buffers that the tile is ADDED to
   float* accf1;
@@ -630,9 +632,9 @@ __device__ __forceinline__ float max4(float4 v) { return fmaxf(fmaxf(v.x, v.y), 
 // index (0..3) of the first component equal to m
 __device__ __forceinline__ int first_eq4(float4 v, float m) { return v.x == m ? 0 : (v.y == m ? 1 : (v.z == m ? 2 : 3)); }
 
-__device__ __forceinline__ void routing_epilogue_smem(const GemmParams& p, const float* s_bias, uint32_t scratch,
-                                                      uint32_t picks_base, int64_t row, int tile, int ew, uint32_t taddr,
-                                                      int lane) {
+__device__ __forceinline__ void routing_epilogue_smem(const GemmParams& p, const float* s_bias, int* s_hist,
+                                                      uint32_t scratch, uint32_t picks_base, int64_t row, int tile,
+                                                      int ew, uint32_t taddr, int lane) {
   const int64_t tok = row;
   const bool valid = tok < p.T;
   const int E = p.N_total, k = p.top_k;
@@ -689,6 +691,7 @@ __device__ __forceinline__ void routing_epilogue_smem(const GemmParams& p, const
     zs += ex;
     asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(picks + j * (128 * 8)), "r"(__float_as_uint(ex)), "r"(g * 4 + ci)
                  : "memory");
+    if (valid) atomicAdd(&s_hist[g * 4 + ci], 1);  // the tile's histogram (integer adds: order-free, deterministic)
     v4.x = ci == 0 ? -INFINITY : v4.x;
     v4.y = ci == 1 ? -INFINITY : v4.y;
     v4.z = ci == 2 ? -INFINITY : v4.z;
@@ -704,6 +707,13 @@ __device__ __forceinline__ void routing_epilogue_smem(const GemmParams& p, const
 #pragma unroll
     for (int q = 0; q < 8; ++q) sm[q] = (q == s) ? ns : sm[q];
   }
+  // the four epilogue warps (128 tokens) have counted their picks: the tile's row of the permutation's histogram
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+  if (tid < E) {
+    p.tile_counts[static_cast<int64_t>(tile) * E + tid] = s_hist[tid];
+    s_hist[tid] = 0;  // ready for this CTA's next tile
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
   // softmax over all E logits (read again from tensor memory: the shared copy has lost the picks); the exponentials
   // are parked in the shared copy until their sum is known
   float z = 0.f;

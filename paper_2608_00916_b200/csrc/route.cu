@@ -204,10 +204,10 @@ void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t*
 // the order inside an expert is the token order.  Each warp covers 32 consecutive tokens and records, per
 // expert, the 32-bit mask of its tokens that chose it (atomicOr: order-free, hence deterministic); ranks
 // are population counts of mask prefixes.  Tiles of TOK_TILE tokens are combined by a column scan.
-__device__ __forceinline__ void build_masks(uint32_t* masks /* [8][E] */, const int32_t* __restrict__ idx, int64_t T,
+__device__ __forceinline__ void build_masks(uint32_t* masks /* [TOK_WARPS][E] */, const int32_t* __restrict__ idx, int64_t T,
                                             int E, int k, int64_t tile_t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int i = tid; i < 8 * E; i += TOK_TILE) masks[i] = 0u;
+  for (int i = tid; i < TOK_WARPS * E; i += TOK_TILE) masks[i] = 0u;
   __syncthreads();
   const int64_t t = tile_t0 + tid;
   if (t < T) {
@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(TOK_TILE) hist_kernel(int64_t T, int E, int k,
   for (int e = threadIdx.x; e < E; e += TOK_TILE) {
     int c = 0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) c += __popc(hist_masks[w * E + e]);
+    for (int w = 0; w < TOK_WARPS; ++w) c += __popc(hist_masks[w * E + e]);
     tile_counts[static_cast<int64_t>(blockIdx.x) * E + e] = c;
   }
 }
@@ -244,6 +244,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
   __shared__ TableScratch s_tab;
   __shared__ float s_term[MAX_E];
   __shared__ float s_ps[SCAN_THREADS];
+  __shared__ int s_seg[SCAN_THREADS];
   const int tid = threadIdx.x;
   // column sums of p: G groups of threads stride over the partial rows
   const int G = SCAN_THREADS / E;
@@ -267,22 +268,43 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(int64_t T, int E, in
     s_ps[tid] = acc[0];
   }
   __syncthreads();
-  // exclusive prefix of every expert's column of tile_counts along the tiles.  One thread per expert, so that the
-  // lanes of a warp touch consecutive addresses (a warp per column with a lane per tile costs one memory wavefront per
-  // lane - 16 k cycles of this one-block kernel went there); 32 loads are in flight before the first dependent store.
-  for (int e = tid; e < E; e += SCAN_THREADS) {
-    int run = 0;
-    for (int t0 = 0; t0 < tok_tiles; t0 += 32) {
-      int c[32];
+  // exclusive prefix of every expert's column of tile_counts along the tiles.  The G thread groups cut the tiles into G
+  // consecutive segments; thread (g, e) sums its segment of column e (lanes of a warp touch consecutive experts, so the
+  // accesses are coalesced, sixteen loads in flight), the segment totals are combined through shared memory, and a
+  // second sweep over the segment writes the prefixes.  One thread per expert walking all tiles took 4 - 8 dependent
+  // rounds of global loads; this takes two.
+  {
+    const int seg = (tok_tiles + G - 1) / G;
+    const int g = tid / E, e = tid - g * E;
+    const bool mine = tid < G * E;
+    const int t_lo = min(tok_tiles, g * seg), t_hi = min(tok_tiles, t_lo + seg);
+    int total = 0;
+    if (mine) {
+      for (int t0 = t_lo; t0 < t_hi; t0 += 16) {
+        int c[16];
 #pragma unroll
-      for (int u = 0; u < 32; ++u) c[u] = (t0 + u < tok_tiles) ? tile_counts[static_cast<int64_t>(t0 + u) * E + e] : 0;
+        for (int u = 0; u < 16; ++u) c[u] = (t0 + u < t_hi) ? tile_counts[static_cast<int64_t>(t0 + u) * E + e] : 0;
 #pragma unroll
-      for (int u = 0; u < 32; ++u) {
-        if (t0 + u < tok_tiles) tile_counts[static_cast<int64_t>(t0 + u) * E + e] = run;
-        run += c[u];
+        for (int u = 0; u < 16; ++u) total += c[u];
       }
+      s_seg[tid] = total;
     }
-    s_cnt[e] = run;
+    __syncthreads();
+    if (mine) {
+      int run = 0;
+      for (int q = 0; q < g; ++q) run += s_seg[q * E + e];
+      for (int t0 = t_lo; t0 < t_hi; t0 += 16) {
+        int c[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) c[u] = (t0 + u < t_hi) ? tile_counts[static_cast<int64_t>(t0 + u) * E + e] : 0;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          if (t0 + u < t_hi) tile_counts[static_cast<int64_t>(t0 + u) * E + e] = run;
+          run += c[u];
+        }
+      }
+      if (g == G - 1) s_cnt[e] = run;  // the last segment ends with the column total (empty segments pass it on)
+    }
   }
   __syncthreads();
   for (int e = tid; e < E; e += SCAN_THREADS) {
@@ -405,12 +427,13 @@ void launch_prepare(const WsLayout& L, char* ws, cudaStream_t st) {
 // tables_only: stop after the histogram and the scan (per-tile prefixes, counts, tables, aux loss); the expert-parallel
 // path places the rows itself
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
-                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only) {
+                    int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only,
+                    bool histogram_done) {
   int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
   int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
   const int tiles = static_cast<int>(L.tok_tiles);
-  const size_t msm = sizeof(uint32_t) * 8 * s.E;
-  if (tiles > 0) {
+  const size_t msm = sizeof(uint32_t) * TOK_WARPS * s.E;
+  if (tiles > 0 && !histogram_done) {
     hist_kernel<<<tiles, TOK_TILE, msm, st>>>(T, s.E, s.k, idx, tile_counts);
     note_launch();
   }
