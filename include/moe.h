@@ -68,6 +68,16 @@ typedef struct {
  * the context, forked and joined inside the call (the caller's stream sees one ordered call; the pattern is legal
  * inside a stream capture).  This flag keeps everything on the caller's stream. */
 #define MOE_FLAG_NO_SIDE_STREAM 8
+/* The router weight W_r is passed as fp32 [d,E] instead of bf16 (moe_forward / moe_backward only; E must be a multiple
+ * of 8).  Every fp32 value is the exact sum of three bf16 values, so the logits are still an fp32 contraction of exact
+ * products: the library splits W_r on the device at every forward call and runs three tensor-core passes. */
+#define MOE_FLAG_ROUTER_FP32 32
+/* Debug build of the index-driven kernels (permutation scatter, row copies, combine, unpermute, router gradient): every
+ * expert index and row index read from the routing tables is checked against its range before it is used; a violation
+ * is recorded in the status word (moe_poll_status then returns MOE_ERR_DEVICE_BOUNDS) and the access is skipped or
+ * redirected to row 0, so nothing out of range is touched.  For hunting corrupted tables where a memory checker is not
+ * available; costs a few percent in those kernels. */
+#define MOE_FLAG_DEBUG_CHECKS 64
 
 typedef struct moe_ctx moe_ctx; /* opaque, lives in host memory */
 
@@ -139,7 +149,7 @@ MOE_API moe_status moe_stage_times(moe_ctx* ctx, float* ms /* host */, int32_t* 
 
 /* Forward pass over T tokens (T >= 0).
  *   x          [T,d]   bf16
- *   W_r        [d,E]   bf16 router weight; the contraction accumulates in fp32
+ *   W_r        [d,E]   bf16 router weight (fp32 with MOE_FLAG_ROUTER_FP32); the contraction accumulates in fp32
  *   b_r        [E]     fp32 additive logit bias, or NULL
  *   logits_in  [T,E]   fp32, or NULL.  When given, routing starts from these logits and the router
  *                      contraction is skipped (test hook: lets a caller construct exact ties).

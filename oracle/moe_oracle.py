@@ -38,7 +38,10 @@ import numpy as np
 
 # --------------------------------------------------------------------------------------------- inputs
 def widen_bf16(bits: np.ndarray, dtype=np.float64) -> np.ndarray:
-    """bf16 bit patterns (uint16) -> ``dtype`` (exact)."""
+    """bf16 bit patterns (uint16) -> ``dtype`` (exact).  A floating-point array is taken as values, not bit patterns,
+    and only converted to ``dtype`` (the router weight may be given in fp32)."""
+    if np.issubdtype(np.asarray(bits).dtype, np.floating):
+        return np.asarray(bits).astype(dtype)
     u = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
     return u.view(np.float32).astype(dtype)
 

@@ -13,6 +13,8 @@ FLAG_CTA_PAIR_TILES = 1    # MOE_FLAG_CTA_PAIR_TILES of include/moe.h
 FLAG_SINGLE_CTA_TILES = 2  # MOE_FLAG_SINGLE_CTA_TILES
 FLAG_NO_SIDE_STREAM = 8    # MOE_FLAG_NO_SIDE_STREAM
 FLAG_HYBRID_TILES = 16     # MOE_FLAG_HYBRID_TILES
+FLAG_ROUTER_FP32 = 32      # MOE_FLAG_ROUTER_FP32
+FLAG_DEBUG_CHECKS = 64     # MOE_FLAG_DEBUG_CHECKS
 STAGE_NAMES = ["router", "permute", "gemm_gateup_swiglu", "gemm_down", "combine", "combine_bwd",
                "dgrad_down_swiglu_bwd", "wgrad_down", "dgrad_gateup", "wgrad_gateup", "router_bwd", "dW_r",
                "unpermute_bwd", "dx_router_term"]
@@ -170,6 +172,7 @@ class MoELayer:
     def __init__(self, d: int, E: int, f: int, top_k: int, flags: int = 0):
         self.lib = load_library()
         self.d, self.E, self.f, self.k = d, E, f, top_k
+        self.flags = flags
         cfg = MoEConfig(d, E, f, top_k, flags)
         h = C.c_void_p()
         _check(self.lib, self.lib.moe_create(C.byref(cfg), C.byref(h)), "moe_create")
@@ -223,7 +226,8 @@ class MoELayer:
         T = x.shape[0]
         d, E, f, k = self.d, self.E, self.f, self.k
         assert x.dtype == torch.bfloat16 and tuple(x.shape) == (T, d) and x.is_contiguous()
-        assert tuple(W_r.shape) == (d, E) and W_r.dtype == torch.bfloat16 and W_r.is_contiguous()
+        wr_dtype = torch.float32 if (self.flags & FLAG_ROUTER_FP32) else torch.bfloat16
+        assert tuple(W_r.shape) == (d, E) and W_r.dtype == wr_dtype and W_r.is_contiguous()
         for w, shp in ((W_gate, (E, d, f)), (W_up, (E, d, f)), (W_down, (E, f, d))):
             assert tuple(w.shape) == shp and w.dtype == torch.bfloat16 and w.is_contiguous()
         self._ensure_ws(T, inference)

@@ -63,6 +63,7 @@ WsLayout make_layout(const Shape& s, int64_t T, bool row_buffers) {
   L.dl_hi = take(sizeof(uint16_t) * (T * s.E + 64));
   L.dl_lo = take(sizeof(uint16_t) * (T * s.E + 64));
   L.dwr_part = take(sizeof(float) * DWR_SPLIT * s.d * s.E);
+  L.wr_split = take(sizeof(uint16_t) * 3 * (static_cast<size_t>(s.d) * s.E + 64));
   L.dhg = take(rows_f);
   L.dhu = take(rows_f);
   L.dxp = take(rows_d);
@@ -144,12 +145,15 @@ moe_status moe_create(const moe_config* cfg, moe_ctx** out) {
   if (cfg->d <= 0 || cfg->f <= 0 || cfg->d % 64 != 0 || cfg->f % 64 != 0) return MOE_ERR_INVALID_ARG;
   if (cfg->E < 1 || cfg->E > MAX_E) return MOE_ERR_INVALID_ARG;
   if (cfg->top_k < 1 || cfg->top_k > cfg->E || cfg->top_k > MAX_K) return MOE_ERR_INVALID_ARG;
+  if ((cfg->flags & MOE_FLAG_ROUTER_FP32) && cfg->E % 8 != 0) return MOE_ERR_UNSUPPORTED;  // tensor-core router only
   moe_ctx_impl* c = new (std::nothrow) moe_ctx_impl;
   if (!c) return MOE_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
   c->s = Shape{cfg->d, cfg->E, cfg->f, cfg->top_k};
   c->device = -1;  // bound by the first call that launches work
   c->use_side_stream = (cfg->flags & MOE_FLAG_NO_SIDE_STREAM) ? 0 : 1;
+  c->router_fp32 = (cfg->flags & MOE_FLAG_ROUTER_FP32) ? 1 : 0;
+  c->debug_checks = (cfg->flags & MOE_FLAG_DEBUG_CHECKS) ? 1 : 0;
   c->tile_mode = (cfg->flags & MOE_FLAG_CTA_PAIR_TILES) ? 1
                  : (cfg->flags & MOE_FLAG_SINGLE_CTA_TILES) ? 2
                  : (cfg->flags & MOE_FLAG_HYBRID_TILES) ? 3 : 0;
@@ -370,7 +374,17 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
   io.x = x; io.W_r = W_r; io.b_r = b_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
   io.idx_out = topk_idx; io.gates_out = topk_w; io.logits_out = logits_out;
   const bool tc_router = router_on_tensor_cores(s) && logits_in == nullptr;
+  if (c->router_fp32 && (lora || !training)) return MOE_ERR_UNSUPPORTED;  // fp32 router weight: moe_forward / moe_backward
   launch_prepare(L, ws, st);  // before any kernel that may record a status
+  if (c->router_fp32 && W_r) {
+    // W_r points at fp32 values: split them into three exact bf16 terms, kept in the workspace for the backward pass
+    const int64_t n = static_cast<int64_t>(s.d) * s.E, stride = n + 64;
+    uint16_t* sp = reinterpret_cast<uint16_t*>(ws + L.wr_split);
+    launch_split_fp32(reinterpret_cast<const float*>(W_r), sp, sp + stride, sp + 2 * stride, n, st);
+    io.W_r = sp;
+    io.W_r_mid = sp + stride;
+    io.W_r_lo = sp + 2 * stride;
+  }
   {
     StageTimer tm(c, st, 0);
     if (T > 0 && tc_router) {
@@ -386,7 +400,7 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
     StageTimer tm(c, st, 1);
     launch_permute(s, T, L, ws, x, expert_counts, perm, aux_loss,
                    static_cast<int>(router_psum_rows(s, T, logits_in != nullptr)), st, /*tables_only=*/false,
-                   /*histogram_done=*/tc_router && T > 0 && router_writes_histogram(s));
+                   /*histogram_done=*/tc_router && T > 0 && router_writes_histogram(s), c->debug_checks != 0);
   }
   if (T > 0) {
     {
@@ -412,7 +426,8 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
     {
       StageTimer tm(c, st, 4);
       launch_combine(s, T, reinterpret_cast<const uint16_t*>(ws + L.o), reinterpret_cast<const float*>(ws + L.gates),
-                     reinterpret_cast<const int32_t*>(ws + L.inv), y, st);  // o already carries the gates
+                     reinterpret_cast<const int32_t*>(ws + L.inv), y, st,  // o already carries the gates
+                     c->debug_checks ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr, L.rows_max);
     }
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
@@ -474,12 +489,20 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
   const float* gates = reinterpret_cast<const float*>(ws + L.gates);
   GemmIO io;
   io.x = x; io.W_r = W_r; io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
+  if (c->router_fp32) {  // the three bf16 terms the forward call left in the workspace
+    if (lora) return MOE_ERR_UNSUPPORTED;
+    const int64_t stride = static_cast<int64_t>(s.d) * s.E + 64;
+    uint16_t* sp = reinterpret_cast<uint16_t*>(static_cast<char*>(workspace) + L.wr_split);
+    io.W_r = sp;
+    io.W_r_mid = sp + stride;
+    io.W_r_lo = sp + 2 * stride;
+  }
   io.dW_gate = dW_gate; io.dW_up = dW_up; io.dW_down = dW_down; io.dx = dx;
   io.dW_gate_acc = acc_gate; io.dW_up_acc = acc_up; io.dW_down_acc = acc_down;
   const bool tc_router = router_on_tensor_cores(s);
   if (T > 0) {
     StageTimer tm(c, st, 5);
-    launch_gather_rows(s, T, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st);
+    launch_gather_rows(s, T, L, ws, dy, reinterpret_cast<uint16_t*>(ws + L.o), st, c->debug_checks != 0);
   }
   // The router's gradient chain (dl, dW_r, db_r and the router term of dx) needs only the dg partials that the
   // dgrad-down GEMM leaves behind.  It is small and latency-bound, so it runs on a second stream of the context, forked
@@ -499,7 +522,8 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
       launch_router_bwd(s, T, reinterpret_cast<const float*>(ws + L.logits), reinterpret_cast<const int32_t*>(ws + L.idx),
                         gates, reinterpret_cast<const float*>(ws + L.dg_part), 2 * ((s.f + 255) / 256), L.rows_max, inv,
                         reinterpret_cast<float*>(ws + L.dg), reinterpret_cast<const int32_t*>(ws + L.counts), d_aux, dl,
-                        reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo), rs);
+                        reinterpret_cast<uint16_t*>(ws + L.dl_hi), reinterpret_cast<uint16_t*>(ws + L.dl_lo), rs,
+                        c->debug_checks ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr);
     }
     {
       StageTimer tm(c, rs, 11);
@@ -575,7 +599,8 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     StageTimer tm(c, st, 12);
     if (tc_router && T > 0) {
       launch_unpermute_sum(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv,
-                           reinterpret_cast<const uint16_t*>(ws + L.dxr), dx, st);
+                           reinterpret_cast<const uint16_t*>(ws + L.dxr), dx, st,
+                           c->debug_checks ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr, L.rows_max);
     } else {
       launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, st);
     }
@@ -730,6 +755,7 @@ moe_status moe_step_host(moe_ctx* ctx, int64_t T, int copy_weights, const uint16
   if (copy_weights && (!W_r || !W_gate || !W_up || !W_down || !dW_r || !dW_gate || !dW_up || !dW_down))
     return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  if (c->router_fp32) return MOE_ERR_UNSUPPORTED;  // the host-buffer steps carry a bf16 router weight
   const Shape& s = c->s;
   const E2ELayout L = e2e_layout(s, T);
   if (dev_bytes < L.total) return MOE_ERR_WORKSPACE;
@@ -800,6 +826,7 @@ moe_status moe_step_host_begin(moe_ctx* ctx, int slot, int64_t T, const uint16_t
                                void* cuda_stream) {
   if (!ctx || T < 0 || (slot != 0 && slot != 1) || !dev || !x || !dy || !y || !dx || !aux_loss) return MOE_ERR_INVALID_ARG;
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
+  if (c->router_fp32) return MOE_ERR_UNSUPPORTED;
   const Shape& s = c->s;
   const E2ELayout L = e2e_layout(s, T);
   if (dev_bytes < L.total) return MOE_ERR_WORKSPACE;

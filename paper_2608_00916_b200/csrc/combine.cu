@@ -10,11 +10,18 @@ namespace moe {
 // One block per token; a thread owns 8 consecutive columns (16 bytes) and issues the k row loads back to back.
 __global__ void __launch_bounds__(256) combine_kernel(int d, int k, const uint16_t* __restrict__ o,
                                                       const float* __restrict__ gates, const int32_t* __restrict__ inv,
-                                                      uint16_t* __restrict__ y) {
+                                                      uint16_t* __restrict__ y, int32_t* dbg_status, int64_t rows_max) {
   const int64_t t = blockIdx.x;
   __shared__ int sr[MAX_K];
   (void)gates;
-  if (threadIdx.x < k) sr[threadIdx.x] = inv[t * k + threadIdx.x];
+  if (threadIdx.x < k) {
+    int r = inv[t * k + threadIdx.x];
+    if (dbg_status && (r < 0 || r >= rows_max)) {  // debug checks: record, and read row 0 instead of out of range
+      record_status(dbg_status, DEV_BOUNDS, 504);
+      r = 0;
+    }
+    sr[threadIdx.x] = r;
+  }
   __syncthreads();
   for (int c = threadIdx.x * 8; c < d; c += 256 * 8) {
     float acc[8];
@@ -39,9 +46,9 @@ __global__ void __launch_bounds__(256) combine_kernel(int d, int k, const uint16
 }
 
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
-                    uint16_t* y, cudaStream_t st) {
+                    uint16_t* y, cudaStream_t st, int32_t* dbg_status, int64_t rows_max) {
   if (T == 0) return;
-  combine_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, o, gates, inv, y);
+  combine_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, o, gates, inv, y, dbg_status, rows_max);
   note_launch();
 }
 
@@ -58,7 +65,7 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
                                                          float* __restrict__ dg,
                                                          const int32_t* __restrict__ counts, float d_aux,
                                                          float* __restrict__ dl, uint16_t* __restrict__ dl_hi,
-                                                         uint16_t* __restrict__ dl_lo) {
+                                                         uint16_t* __restrict__ dl_lo, int32_t* dbg_status) {
   const int lane = threadIdx.x & 31;
   const int64_t t = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (t >= T) return;
@@ -102,8 +109,16 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
   if (lane < k) {
     g = gates[t * k + lane];
     ej = idx[t * k + lane];
+    if (dbg_status && (ej < 0 || ej >= E)) {  // debug checks
+      record_status(dbg_status, DEV_BOUNDS, 506);
+      ej = 0;
+    }
     if (dg_tiles > 0) {
-      const int r = inv[t * k + lane];
+      int r = inv[t * k + lane];
+      if (dbg_status && (r < 0 || r >= rows_max)) {
+        record_status(dbg_status, DEV_BOUNDS, 507);
+        r = 0;
+      }
       for (int nt = 0; nt < dg_tiles; ++nt) dgj += dg_part[nt * rows_max + r];
       dg[t * k + lane] = dgj;
     } else {
@@ -140,11 +155,11 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(int64_t T, int E, int k
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
                        const float* dg_part, int dg_tiles, int64_t rows_max, const int32_t* inv, float* dg,
                        const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi, uint16_t* dl_lo,
-                       cudaStream_t st) {
+                       cudaStream_t st, int32_t* dbg_status) {
   if (T == 0) return;
   router_bwd_kernel<<<static_cast<unsigned>((T + 7) / 8), 256, 0, st>>>(T, s.E, s.k, logits, idx, gates, dg_part,
                                                                         dg_tiles, rows_max, inv, dg, counts, d_aux, dl,
-                                                                        dl_hi, dl_lo);
+                                                                        dl_hi, dl_lo, dbg_status);
   note_launch();
 }
 
@@ -353,10 +368,18 @@ __global__ void __launch_bounds__(256) unpermute_bwd_kernel(int64_t T, int d, in
 __global__ void __launch_bounds__(256) unpermute_sum_kernel(int d, int k, const uint16_t* __restrict__ dxp,
                                                             const int32_t* __restrict__ inv,
                                                             const uint16_t* __restrict__ dxr,
-                                                            uint16_t* __restrict__ dx) {
+                                                            uint16_t* __restrict__ dx, int32_t* dbg_status,
+                                                            int64_t rows_max) {
   const int64_t t = blockIdx.x;
   __shared__ int sr[MAX_K];
-  if (threadIdx.x < k) sr[threadIdx.x] = inv[t * k + threadIdx.x];
+  if (threadIdx.x < k) {
+    int r = inv[t * k + threadIdx.x];
+    if (dbg_status && (r < 0 || r >= rows_max)) {
+      record_status(dbg_status, DEV_BOUNDS, 505);
+      r = 0;
+    }
+    sr[threadIdx.x] = r;
+  }
   __syncthreads();
   for (int c = threadIdx.x * 8; c < d; c += 256 * 8) {
     float acc[8];
@@ -386,9 +409,9 @@ __global__ void __launch_bounds__(256) unpermute_sum_kernel(int d, int k, const 
 }
 
 void launch_unpermute_sum(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const uint16_t* dxr,
-                          uint16_t* dx, cudaStream_t st) {
+                          uint16_t* dx, cudaStream_t st, int32_t* dbg_status, int64_t rows_max) {
   if (T == 0) return;
-  unpermute_sum_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, dxp, inv, dxr, dx);
+  unpermute_sum_kernel<<<static_cast<unsigned>(T), 256, 0, st>>>(s.d, s.k, dxp, inv, dxr, dx, dbg_status, rows_max);
   note_launch();
 }
 

@@ -59,6 +59,7 @@ struct WsLayout {
   size_t dl;           // float[T*E]
   size_t dl_hi, dl_lo; // bf16[T*E]   dl split into two bf16 terms (hi + lo) for the tensor-core contractions
   size_t dwr_part;     // float[DWR_SPLIT * d * E]
+  size_t wr_split;     // bf16[3 * d * E]  fp32 router weight split into three bf16 terms (MOE_FLAG_ROUTER_FP32)
   size_t xp;           // bf16[rows_max * d]
   size_t hg, hu, act;  // bf16[rows_max * f]
   size_t o;            // bf16[rows_max * d]   gate-scaled o in forward, the gathered dy rows in backward
@@ -88,6 +89,8 @@ struct moe_ctx_impl {
   int sm_count;
   int device;
   void* encode_fn;  // cuTensorMapEncodeTiled, fetched through the runtime
+  int router_fp32;      // W_r is passed as fp32 (MOE_FLAG_ROUTER_FP32)
+  int debug_checks;     // MOE_FLAG_DEBUG_CHECKS: index checks in the permutation / combine / router-gradient kernels
   int use_side_stream;  // backward runs the router's gradient chain on s_side, beside the big GEMMs
   int side_created;
   cudaStream_t s_side;
@@ -129,18 +132,22 @@ void launch_router(const Shape& s, int64_t T, const uint16_t* x, const uint16_t*
                    float* gates_out, float* logits_out, float* psum_part, cudaStream_t st);
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
                     int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only = false,
-                    bool histogram_done = false);
+                    bool histogram_done = false, bool debug = false);
+// fp32 [n] -> three bf16 terms hi, mid, lo with hi + mid + lo == w exactly (route.cu)
+void launch_split_fp32(const float* w, uint16_t* hi, uint16_t* mid, uint16_t* lo, int64_t n, cudaStream_t st);
 // ---- launchers (combine.cu)
+// dbg_status (here and below): null, or the workspace's status word - the kernel then checks every row / expert index
+// it is about to use, records DEV_BOUNDS and skips or redirects the access instead of touching memory out of range
 void launch_combine(const Shape& s, int64_t T, const uint16_t* o, const float* gates, const int32_t* inv,
-                    uint16_t* y, cudaStream_t st);
+                    uint16_t* y, cudaStream_t st, int32_t* dbg_status = nullptr, int64_t rows_max = 0);
 // rows[inv[t,j],:] = src[t,:] for every (token, slot), pad rows zeroed: xp from x, and the dy rows of backward
 void launch_gather_rows(const Shape& s, int64_t T, const WsLayout& L, const char* ws, const uint16_t* src,
-                        uint16_t* rows, cudaStream_t st);
+                        uint16_t* rows, cudaStream_t st, bool debug = false);
 // dg[t,j] = sum over column tiles of dg_part[tile][inv[t,j]], then dl (fp32 and the two-term bf16 split)
 void launch_router_bwd(const Shape& s, int64_t T, const float* logits, const int32_t* idx, const float* gates,
                        const float* dg_part, int dg_tiles, int64_t rows_max, const int32_t* inv, float* dg,
                        const int32_t* counts, float d_aux, float* dl, uint16_t* dl_hi, uint16_t* dl_lo,
-                       cudaStream_t st);
+                       cudaStream_t st, int32_t* dbg_status = nullptr);
 // dg_tiles == 0: dg[t,j] has been filled by the caller (expert-parallel path) and is read instead of the partials
 // SIMT dW_r (any E) and the shared partial reduction / db_r
 void launch_dwr(const Shape& s, int64_t T, const uint16_t* x, const float* dl, float* part, float* dW_r,
@@ -149,14 +156,16 @@ void launch_unpermute_bwd(const Shape& s, int64_t T, const uint16_t* dxp, const 
                           const uint16_t* W_r, uint16_t* dx, cudaStream_t st);
 // dx[t,:] = dxr[t,:] + sum_j dxp[inv[t,j],:]  (router term already contracted on the tensor cores)
 void launch_unpermute_sum(const Shape& s, int64_t T, const uint16_t* dxp, const int32_t* inv, const uint16_t* dxr,
-                          uint16_t* dx, cudaStream_t st);
+                          uint16_t* dx, cudaStream_t st, int32_t* dbg_status = nullptr, int64_t rows_max = 0);
 // ---- launchers (gemm.cu); each returns a CUDA / driver error as moe_status
 enum GemmKind { GEMM_F3 = 0, GEMM_F4, GEMM_B2, GEMM_B3, GEMM_B4, GEMM_B5, GEMM_RT, GEMM_DX, GEMM_DWR, GEMM_KINDS };
 // Caller tensors a grouped-GEMM launch may need besides the workspace.
 struct GemmIO {
   bool save_preactivations = true;  // forward: also write hg, hu (needed by backward only)
   const uint16_t* x = nullptr;
-  const uint16_t* W_r = nullptr;
+  const uint16_t* W_r = nullptr;      // bf16 router weight, or the leading bf16 term of an fp32 one
+  const uint16_t* W_r_mid = nullptr;  // fp32 router weight: the second and third bf16 terms (W = hi + mid + lo exactly)
+  const uint16_t* W_r_lo = nullptr;
   const float* b_r = nullptr;
   const uint16_t* W_gate = nullptr;
   const uint16_t* W_up = nullptr;

@@ -226,6 +226,7 @@ moe_status moe_ep_create(const moe_config* cfg, int32_t world, int32_t rank, int
   *out = nullptr;
   if (world < 1 || world > MOE_EP_MAX_RANKS || rank < 0 || rank >= world || rows_cap < 0) return MOE_ERR_INVALID_ARG;
   if (cfg->E % world != 0 || cfg->E % 8 != 0) return MOE_ERR_INVALID_ARG;
+  if (cfg->flags & MOE_FLAG_ROUTER_FP32) return MOE_ERR_UNSUPPORTED;  // the expert-parallel path takes a bf16 router weight
   if (rows_cap > (int64_t(1) << 30)) return MOE_ERR_UNSUPPORTED;
   moe_ctx* full = nullptr;
   moe_status rc = moe_create(cfg, &full);

@@ -455,6 +455,10 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       // logits[T,E] = x[T,d] W_r[d,E]; W_r is read as a one-slab 3D tensor so the weight loaders apply
       ok = map_2d(fn, &p.mapA0, io.x, T, d, 128) && map_3d(fn, &p.mapB0, io.W_r, 1, d, E, 64);
       p.mapA1 = p.mapA0; p.mapB1 = p.mapB0;
+      if (io.W_r_mid) {  // fp32 router weight: x (hi + mid + lo), each product exact in fp32
+        ok = ok && map_3d(fn, &p.mapB1, io.W_r_mid, 1, d, E, 64) && map_3d(fn, &p.mapB2, io.W_r_lo, 1, d, E, 64);
+        p.nseg = 3;
+      }
       p.static_m_tiles = static_cast<int>((T + BM - 1) / BM);
       p.n_tiles = 1;
       p.k_blocks = d / BK;
@@ -480,6 +484,10 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       ok = map_2d(fn, &p.mapA0, ws + L.dl_hi, T, E, 128) && map_2d(fn, &p.mapA1, ws + L.dl_lo, T, E, 128) &&
            map_3d(fn, &p.mapB0, io.W_r, 1, d, E, 256);
       p.mapB1 = p.mapB0;
+      if (io.W_r_mid) {  // fp32 router weight: dl_hi W_hi^T + dl_lo W_hi^T + dl_hi W_mid^T (the rest is below 2^-17)
+        ok = ok && map_2d(fn, &p.mapA2, ws + L.dl_hi, T, E, 128) && map_3d(fn, &p.mapB2, io.W_r_mid, 1, d, E, 256);
+        p.nseg = 3;
+      }
       p.static_m_tiles = static_cast<int>((T + BM - 1) / BM);
       p.n_tiles = (d + 255) / 256;
       p.k_blocks = (E + BK - 1) / BK;

@@ -178,7 +178,15 @@ __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl,
       tma_load_3d(sB + c * CHUNK_BYTES, &p.mapB0, bar, tl.n0 + c * 64, kb * BK, tl.e);
       tma_load_3d(sB + (2 + c) * CHUNK_BYTES, &p.mapB1, bar, tl.n0 + c * 64, kb * BK, tl.e);
     }
-  } else if (KIND == GEMM_F4 || KIND == GEMM_RT) {
+  } else if (KIND == GEMM_RT) {
+    // one K segment per bf16 term of the router weight (one term for a bf16 weight, three for an fp32 weight)
+    const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
+    const CUtensorMap* mb = seg == 0 ? &p.mapB0 : (seg == 1 ? &p.mapB1 : &p.mapB2);
+    tma_load_2d(sA, &p.mapA0, bar, kk * BK, tl.row0);
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (c < p.b_chunks) tma_load_3d(sB + c * CHUNK_BYTES, mb, bar, tl.n0 + c * 64, kk * BK, tl.e);
+  } else if (KIND == GEMM_F4) {
     tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
 #pragma unroll
     for (int c = 0; c < 4; ++c)
@@ -187,9 +195,9 @@ __device__ __forceinline__ void issue_loads(const GemmParams& p, const Tile& tl,
     tma_load_2d(sA, &p.mapA0, bar, kb * BK, tl.row0);
     tma_load_3d(sB, &p.mapB0, bar, kb * BK, tl.n0, tl.e);
   } else if (KIND == GEMM_B4 || KIND == GEMM_DX) {
-    const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;
-    tma_load_2d(sA, seg ? &p.mapA1 : &p.mapA0, bar, kk * BK, tl.row0);
-    tma_load_3d(sB, seg ? &p.mapB1 : &p.mapB0, bar, kk * BK, tl.n0, tl.e);
+    const int seg = kb / p.k_blocks, kk = kb - seg * p.k_blocks;  // DX: a third segment with an fp32 router weight
+    tma_load_2d(sA, seg == 0 ? &p.mapA0 : (seg == 1 ? &p.mapA1 : &p.mapA2), bar, kk * BK, tl.row0);
+    tma_load_3d(sB, seg == 0 ? &p.mapB0 : (seg == 1 ? &p.mapB1 : &p.mapB2), bar, kk * BK, tl.n0, tl.e);
   } else if (KIND == GEMM_B3) {
     const int row = tl.row0 + kb * BK;
 #pragma unroll

@@ -336,7 +336,8 @@ __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int
                                                            const float* __restrict__ gates,
                                                            int32_t* __restrict__ inv,
                                                            float* __restrict__ row_gate,
-                                                           int32_t* __restrict__ perm_out) {
+                                                           int32_t* __restrict__ perm_out, int32_t* dbg_status,
+                                                           int64_t rows_max) {
   extern __shared__ uint32_t sc_masks[];
   const int64_t tile_t0 = static_cast<int64_t>(blockIdx.x) * TOK_TILE;
   build_masks(sc_masks, idx, T, E, k, tile_t0);
@@ -345,10 +346,18 @@ __global__ void __launch_bounds__(TOK_TILE) scatter_kernel(int64_t T, int E, int
   if (t >= T) return;
   for (int j = 0; j < k; ++j) {
     const int e = idx[t * k + j];
+    if (dbg_status && (e < 0 || e >= E)) {  // debug checks: record and skip instead of touching memory out of range
+      record_status(dbg_status, DEV_BOUNDS, 501);
+      continue;
+    }
     int rank = tile_base[static_cast<int64_t>(blockIdx.x) * E + e];
     for (int w = 0; w < warp; ++w) rank += __popc(sc_masks[w * E + e]);
     rank += __popc(sc_masks[warp * E + e] & ((1u << lane) - 1u));
     const int r = pad_offsets[e] + rank;
+    if (dbg_status && (r < 0 || r >= rows_max)) {
+      record_status(dbg_status, DEV_BOUNDS, 502);
+      continue;
+    }
     inv[t * k + j] = r;
     row_gate[r] = gates[t * k + j];
     if (perm_out) perm_out[offsets[e] + rank] = static_cast<int32_t>(t * k + j);
@@ -365,7 +374,8 @@ __global__ void __launch_bounds__(256) scatter_rows_kernel(int64_t T, int d, int
                                                            const int32_t* __restrict__ inv,
                                                            const int32_t* __restrict__ counts,
                                                            const int32_t* __restrict__ pad_offsets,
-                                                           uint16_t* __restrict__ rows) {
+                                                           uint16_t* __restrict__ rows, int32_t* dbg_status,
+                                                           int64_t rows_max) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n16 = d / 8;
   if (static_cast<int>(blockIdx.x) >= tok_blocks) {
@@ -385,7 +395,12 @@ __global__ void __launch_bounds__(256) scatter_rows_kernel(int64_t T, int d, int
     for (int i = 0; i < 8; ++i)
       if (c0 + lane + 32 * i < n16) v[i] = __ldg(s4 + c0 + lane + 32 * i);
     for (int j = 0; j < k; ++j) {
-      uint4* dst = reinterpret_cast<uint4*>(rows + static_cast<int64_t>(inv[t * k + j]) * d);
+      const int r = inv[t * k + j];
+      if (dbg_status && (r < 0 || r >= rows_max)) {
+        if (lane == 0) record_status(dbg_status, DEV_BOUNDS, 503);
+        continue;
+      }
+      uint4* dst = reinterpret_cast<uint4*>(rows + static_cast<int64_t>(r) * d);
 #pragma unroll
       for (int i = 0; i < 8; ++i)
         if (c0 + lane + 32 * i < n16) dst[c0 + lane + 32 * i] = v[i];
@@ -394,11 +409,12 @@ __global__ void __launch_bounds__(256) scatter_rows_kernel(int64_t T, int d, int
 }
 
 void launch_gather_rows(const Shape& s, int64_t T, const WsLayout& L, const char* ws, const uint16_t* src,
-                        uint16_t* rows, cudaStream_t st) {
+                        uint16_t* rows, cudaStream_t st, bool debug) {
   const int tok_blocks = static_cast<int>((T + 7) / 8);
   scatter_rows_kernel<<<tok_blocks + s.E, 256, 0, st>>>(
       T, s.d, s.k, s.E, tok_blocks, src, reinterpret_cast<const int32_t*>(ws + L.inv),
-      reinterpret_cast<const int32_t*>(ws + L.counts), reinterpret_cast<const int32_t*>(ws + L.pad_offsets), rows);
+      reinterpret_cast<const int32_t*>(ws + L.counts), reinterpret_cast<const int32_t*>(ws + L.pad_offsets), rows,
+      debug ? reinterpret_cast<int32_t*>(const_cast<char*>(ws) + L.status) : nullptr, L.rows_max);
   note_launch();
 }
 
@@ -426,9 +442,32 @@ void launch_prepare(const WsLayout& L, char* ws, cudaStream_t st) {
 
 // tables_only: stop after the histogram and the scan (per-tile prefixes, counts, tables, aux loss); the expert-parallel
 // path places the rows itself
+// An fp32 value is the exact sum of three bf16 values (8 + 8 + 8 significand bits): the router contraction of an
+// fp32 weight runs as three bf16 tensor-core products, each exact in fp32.
+__global__ void __launch_bounds__(256) split_fp32_kernel(const float* __restrict__ w, uint16_t* __restrict__ hi,
+                                                         uint16_t* __restrict__ mid, uint16_t* __restrict__ lo,
+                                                         int64_t n) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (i >= n) return;
+  const float v = w[i];
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(h);
+  const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+  const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+  hi[i] = *reinterpret_cast<const uint16_t*>(&h);
+  mid[i] = *reinterpret_cast<const uint16_t*>(&m);
+  lo[i] = *reinterpret_cast<const uint16_t*>(&l);
+}
+
+void launch_split_fp32(const float* w, uint16_t* hi, uint16_t* mid, uint16_t* lo, int64_t n, cudaStream_t st) {
+  if (n == 0) return;
+  split_fp32_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(w, hi, mid, lo, n);
+  note_launch();
+}
+
 void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, const uint16_t* x, int32_t* counts_out,
                     int32_t* perm_out, float* aux_out, int psum_rows, cudaStream_t st, bool tables_only,
-                    bool histogram_done) {
+                    bool histogram_done, bool debug) {
   int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
   int32_t* tile_counts = reinterpret_cast<int32_t*>(ws + L.tile_counts);
   const int tiles = static_cast<int>(L.tok_tiles);
@@ -445,9 +484,10 @@ void launch_permute(const Shape& s, int64_t T, const WsLayout& L, char* ws, cons
     scatter_kernel<<<tiles, TOK_TILE, msm, st>>>(
         T, s.E, s.k, idx, tile_counts, reinterpret_cast<const int32_t*>(ws + L.offsets),
         reinterpret_cast<const int32_t*>(ws + L.pad_offsets), reinterpret_cast<const float*>(ws + L.gates),
-        reinterpret_cast<int32_t*>(ws + L.inv), reinterpret_cast<float*>(ws + L.row_gate), perm_out);
+        reinterpret_cast<int32_t*>(ws + L.inv), reinterpret_cast<float*>(ws + L.row_gate), perm_out,
+        debug ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr, L.rows_max);
     note_launch();
-    launch_gather_rows(s, T, L, ws, x, reinterpret_cast<uint16_t*>(ws + L.xp), st);
+    launch_gather_rows(s, T, L, ws, x, reinterpret_cast<uint16_t*>(ws + L.xp), st, debug);
   }
 }
 

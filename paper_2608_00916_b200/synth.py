@@ -52,6 +52,9 @@ CONFIGS = {
     "qwen": (MoEShape(16384, 2048, 128, 8, 768), 1001, 1.0, False),
     "skewed": (MoEShape(16384, 2048, 128, 8, 768), 1002, 1.0, True),
     "coarse": (MoEShape(16384, 4096, 8, 2, 14336), 1003, 1.0, False),
+    # the coarse configuration cut down (a quarter of the tokens and of the expert width, same d, E, k and the same
+    # 1024 rows per expert per 4096 tokens) so that a profiler capture holds about 2 GB instead of 12 GB on the device
+    "coarse_reduced": (MoEShape(4096, 4096, 8, 2, 3584), 1003, 1.0, False),
     "sweep_T1000": (MoEShape(1000, 2048, 128, 8, 768), 1004, 1.0, False),
     "sweep_T4096": (MoEShape(4096, 2048, 128, 8, 768), 1005, 1.0, False),
     "sweep_T8191": (MoEShape(8191, 2048, 128, 8, 768), 1006, 1.0, False),

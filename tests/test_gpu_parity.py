@@ -605,3 +605,68 @@ def test_grouped_weight_gradients_signal_ranges_of_experts():
     for n in plain:
         assert torch.equal(grouped[n], 2.0 * plain[n]), n  # doubled exactly once, after the final value was there
     assert touched == [(5, f, d)] * 4 + [(4, f, d)] + [(5, d, f)] * 8 + [(4, d, f)] * 2 + [(d, E)]
+
+
+def test_fp32_router_weight():
+    """MOE_FLAG_ROUTER_FP32: W_r arrives as genuine fp32 values (not representable in bf16); the library splits it into
+    three exact bf16 terms, so logits, routing and gradients follow the oracle evaluated with the fp32 weight."""
+    from paper_2608_00916_b200.binding import FLAG_ROUTER_FP32
+    shape = synth.MoEShape(900, 256, 32, 4, 128)
+    inp = synth.make_inputs(shape, 81)
+    rng = np.random.default_rng(81)
+    W32 = (0.02 * rng.standard_normal((shape.d, shape.E))).astype(np.float32)
+    assert np.any(synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(W32)) != W32)  # needs more than bf16
+    # keep the tokens whose top-k gaps are safe under THIS weight
+    l = synth.bf16_bits_to_f64(inp["x"]) @ W32.astype(np.float64)
+    keep = ~synth._gap_violations(l, shape.k)
+    inp["x"], inp["dy"] = inp["x"][keep], inp["dy"][keep]
+    T = int(keep.sum())
+    ofw = orc.forward(inp["x"], W32, inp["W_gate"], inp["W_up"], inp["W_down"], shape.k)
+    obw = orc.backward(ofw, inp["dy"], 0.02, inp["x"], W32, inp["W_gate"], inp["W_up"], inp["W_down"])
+    layer = MoELayer(shape.d, shape.E, shape.f, shape.k, FLAG_ROUTER_FP32)
+    dev = {n: torch.from_numpy(inp[n].view(np.int16)).cuda().view(torch.bfloat16) for n in ("x", "W_gate", "W_up", "W_down", "dy")}
+    W_r = torch.from_numpy(W32).cuda()
+    fw = layer.forward(dev["x"], W_r, dev["W_gate"], dev["W_up"], dev["W_down"], want_logits=True)
+    bw = layer.backward(dev["dy"], 0.02, want_db=True)
+    layer.poll()
+    check_routing(fw, ofw)
+    # the logits carry the low-order bits of the weight: a bf16-rounded weight would be off by ~1e-3 relative
+    lg = fw["logits"].cpu().numpy()
+    bf = synth.bf16_bits_to_f64(inp["x"]) @ synth.bf16_bits_to_f64(synth.f32_to_bf16_bits(W32))
+    assert np.abs(lg - ofw["logits"]).max() < 0.05 * np.abs(bf - ofw["logits"]).max()
+    assert rel_fro(from_dev_bf16(fw["y"]), ofw["y"]) <= TOL
+    for n in ("dx", "dW_gate", "dW_up", "dW_down"):
+        assert rel_fro(from_dev_bf16(bw[n]), obw[n]) <= TOL, n
+    assert rel_fro(bw["dW_r"].cpu().numpy(), obw["dW_r"]) <= TOL
+    assert rel_fro(bw["db_r"].cpu().numpy(), obw["db_r"]) <= TOL
+    # the router term of dx, isolated: dx minus the oracle's expert part
+    assert T > 800
+
+
+def test_debug_checks_report_a_corrupted_routing_table_without_touching_memory_out_of_range():
+    """MOE_FLAG_DEBUG_CHECKS: a row index of the routing tables is overwritten with a value far outside the row buffers
+    between forward and backward.  The checked kernels record MOE_ERR_DEVICE_BOUNDS and skip / redirect the access (so
+    nothing faults); with an intact table the same context computes the same bits as an unchecked one."""
+    from paper_2608_00916_b200.binding import FLAG_DEBUG_CHECKS, MoEError
+    inp = synth.make_inputs(synth.MoEShape(500, 128, 16, 4, 128), 91)
+    plain = Run(inp, 4)
+    pfw = plain.forward()
+    pbw = plain.backward(0.01)
+    r = Run(inp, 4, flags=FLAG_DEBUG_CHECKS)
+    fw = r.forward()
+    bw = r.backward(0.01)
+    for n in ("y", "idx", "gates"):
+        assert torch.equal(fw[n], pfw[n]), n
+    for n in ("dx", "dW_r", "dW_gate", "dW_down"):
+        assert torch.equal(bw[n], pbw[n]), n
+    # corrupt one entry of inv (the padded row of pair (token 7, slot 1)) and run backward again
+    r.forward()
+    inv = r.layer.buffer("inv", torch.int32)
+    inv[7 * 4 + 1] = 2 ** 30
+    v = r.dev
+    r.layer.backward(v["dy"], 0.01)
+    with pytest.raises(MoEError, match="bounds check"):
+        r.layer.poll()
+    # acknowledged: the context and the workspace work again
+    fw2 = r.forward()
+    assert torch.equal(fw2["y"], pfw["y"])
