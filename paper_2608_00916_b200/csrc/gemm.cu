@@ -323,6 +323,14 @@ static moe_status launch_kind(moe_ctx_impl* ctx, const GemmParams& p, cudaStream
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
+// Row tiles (or pairs) walked together inside a column tile: 1 while the expert's weights are few column tiles wide (they
+// stay in L2 between row tiles: Qwen3-30B-A3B shape), 16 for wide experts (coarse shape: at 112 column tiles an expert's
+// gate and up slabs are 235 MB and were read from DRAM once per row pair).  MOE_ROW_GROUP overrides (measurements).
+static int row_group_for(int n_tiles, const moe_ctx_impl* ctx) {
+  if (ctx->row_group_override > 0) return ctx->row_group_override;
+  return n_tiles > 12 ? 16 : 1;
+}
+
 // One launch of an expert / router contraction.  `pair`: CTA-pair kernel.  `part`: 0 = the whole tile list; row GEMMs
 // of the mixed schedule: 1 = the pair kernel over complete pairs of row blocks only, 2 = the one-CTA kernel over the
 // leftover blocks.
@@ -386,6 +394,7 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       p.row_gate = reinterpret_cast<const float*>(ws + L.row_gate);
       p.save_pre = io.save_preactivations ? 1 : 0;
       if (!ok) return MOE_ERR_CUDA;
+      p.row_group = row_group_for(p.n_tiles, ctx);
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_F3>(ctx, p, st);
     case GEMM_F4:
       ok = map_2d(fn, &p.mapA0, act, R, f, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, 64);
@@ -396,6 +405,7 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       p.out0 = o;
       p.ld_out = d;
       if (!ok) return MOE_ERR_CUDA;
+      p.row_group = row_group_for(p.n_tiles, ctx);
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_F4>(ctx, p, st);
     case GEMM_B2:
       ok = map_2d(fn, &p.mapA0, o, R, d, 128) && map_3d(fn, &p.mapB0, W_down, E, f, d, pair ? 128 : 256);
@@ -410,6 +420,7 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       p.outf = reinterpret_cast<float*>(ws + L.dg_part);
       p.rows_max = L.rows_max;
       if (!ok) return MOE_ERR_CUDA;
+      p.row_group = row_group_for(p.n_tiles, ctx);
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B2>(ctx, p, st);
     case GEMM_B4:
       ok = map_2d(fn, &p.mapA0, dhg, R, f, 128) && map_2d(fn, &p.mapA1, dhu, R, f, 128) &&
@@ -421,6 +432,7 @@ static moe_status launch_gemm_variant(moe_ctx_impl* ctx, GemmKind kind, int64_t 
       p.out0 = dxp;
       p.ld_out = d;
       if (!ok) return MOE_ERR_CUDA;
+      p.row_group = row_group_for(p.n_tiles, ctx);
       return pair ? launch_pair_gemm(ctx, kind, p, st) : launch_kind<GEMM_B4>(ctx, p, st);
     case GEMM_B3:
       ok = map_2d(fn, &p.mapA0, act, R, f, 64) && map_2d(fn, &p.mapB0, o, R, d, 64);

@@ -55,14 +55,15 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
     tl.write = true;
     tl.full = true;
   } else {
-    const int pr = t / p.n_tiles;
+    int pr, nt;
+    row_tile_order(t, p.n_tiles, p.row_group, p.sched[p.pair_count_slot], pr, nt);
     const int4 info = *reinterpret_cast<const int4*>(p.pair_tab + 4 * pr);  // expert, first row, blocks (1 or 2)
     tl.e = info.x;
     tl.row0 = info.y + rank * BM;
     tl.write = rank < info.z;
     tl.full = info.z == 2;
     tl.m0 = 0;
-    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.n0 = nt * Traits<KIND>::N_SPAN;
     tl.nkb = p.k_blocks * p.nseg;
   }
   return tl;

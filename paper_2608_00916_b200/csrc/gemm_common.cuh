@@ -34,6 +34,7 @@ struct GemmParams {
   const int32_t* pair_tab;     // CTA-pair kernels: per pair of row blocks {expert, first row, blocks (1|2), 0}
   int pair_count_slot;         // which entry of sched holds the number of entries of pair_tab
   int oob_row;                 // a row index beyond the row buffers: TMA copies from there deliver zeros
+  int row_group;               // row GEMMs: consecutive row tiles (or pairs) walked together inside one column tile
   const int32_t* tile_list;    // one-CTA row GEMMs: null = every 128-row tile, else the tiles to compute (sched[4] entries)
   int32_t* status;
   unsigned long long* timers;  // null, or 8 counters of this kind: summed over CTAs (see gemm.cu)
@@ -111,6 +112,24 @@ __device__ __forceinline__ int total_tiles(const GemmParams& p) {
   return (p.tile_list ? p.sched[4] : p.sched[0]) * p.n_tiles;
 }
 
+// Order of the tiles of a row GEMM.  group == 1: column tiles fastest (the tiles of one row tile are adjacent; right
+// when an expert's weights stay in L2 anyway).  group > 1: `group` consecutive row tiles are walked together inside
+// one column tile before the next column tile starts, so that a B tile of a wide expert (whose weight slab does not
+// fit in L2) is fetched from DRAM once for the whole group instead of once per row tile.
+__device__ __forceinline__ void row_tile_order(int t, int n_tiles, int group, int n_rows, int& ri, int& nt) {
+  if (group <= 1) {
+    ri = t / n_tiles;
+    nt = t - ri * n_tiles;
+    return;
+  }
+  const int per = group * n_tiles;
+  const int g = t / per, rem = t - g * per;
+  const int base = g * group;
+  const int gsz = min(group, n_rows - base);  // the last group may be short
+  nt = rem / gsz;
+  ri = base + rem - nt * gsz;
+}
+
 template <int KIND>
 __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
   Tile tl;
@@ -136,11 +155,13 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
     tl.nkb = p.k_blocks * p.nseg + p.k_blocks1;
   } else {
-    const int mt = p.tile_list ? p.tile_list[t / p.n_tiles] : t / p.n_tiles;
+    int ri, nt;
+    row_tile_order(t, p.n_tiles, p.row_group, p.tile_list ? p.sched[4] : p.sched[0], ri, nt);
+    const int mt = p.tile_list ? p.tile_list[ri] : ri;
     tl.e = p.tile_expert[mt];
     tl.row0 = mt * BM;
     tl.m0 = 0;
-    tl.n0 = (t % p.n_tiles) * Traits<KIND>::N_SPAN;
+    tl.n0 = nt * Traits<KIND>::N_SPAN;
     tl.nkb = p.k_blocks * p.nseg + p.k_blocks1;
   }
   return tl;
