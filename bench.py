@@ -510,6 +510,11 @@ def main():
                 layer.step_host_end((i - 1) % 2)
             layer.step_host_end((n - 1) % 2)
         run_pipelined(3)
+        # the same untimed conditioning as for the device-resident number (setting up the pinned buffers above took
+        # long enough for the power state to relax)
+        t_c = time.perf_counter()
+        while time.perf_counter() - t_c < args.condition_seconds:
+            run_pipelined(20)
         pdist.barrier()
         torch.cuda.synchronize()
         n_e2e = max(4, min(args.steps, 20))
@@ -575,6 +580,10 @@ def main():
                                f"{mhz} MHz; sustained peak measured at {peaks['sustained_sm_mhz']:.0f} MHz, burst near "
                                f"{peaks['sm_max_mhz']:.0f} MHz)",
                 "frac_of_burst": stages[dom]["frac_of_burst"], "frac_of_sustained": stages[dom]["frac_of_sustained"],
+                # the sustained peak rescaled to the clock this region ran at (that peak was measured at
+                # sustained_sm_mhz; a box that settles at a lower clock under the same cap has a lower ceiling)
+                "frac_of_sustained_at_this_clock": (stages[dom]["TFLOP/s"] / (peaks["bf16_tflops_sustained"] * mhz /
+                                                                             peaks["sustained_sm_mhz"])) if mhz else None,
                 "flop_per_clk_per_sm": stages[dom].get("flop_per_clk_per_sm"),
                 "traffic": NCU_TRAFFIC.get((args.workload, dom))}
     else:

@@ -100,7 +100,8 @@ moe_status ensure_device(moe_ctx_impl* c) {
   if (c->use_side_stream) {
     if (cudaStreamCreateWithFlags(&c->s_side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess)
+        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_b4, cudaEventDisableTiming) != cudaSuccess)
       return MOE_ERR_CUDA;
     c->side_created = 1;
   }
@@ -176,6 +177,7 @@ void moe_destroy(moe_ctx* ctx) {
     cudaStreamDestroy(c->s_side);
     cudaEventDestroy(c->ev_fork);
     cudaEventDestroy(c->ev_join);
+    cudaEventDestroy(c->ev_b4);
   }
   if (c->e2e_created) {
     cudaStreamDestroy(c->s_in);
@@ -539,6 +541,29 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
       const moe_status r2 = launch_grouped_gemm(c, GEMM_DX, T, L, ws, io, rs);
       if (r2 != MOE_OK) return r2;
     }
+    return MOE_OK;
+  };
+  // dx = router term + sum of the dxp rows needs the dgrad gate/up GEMM (dxp) and the router chain (dxr), but not the
+  // last weight-gradient GEMM: with the second stream it runs beside that GEMM (it is bandwidth-bound, fits on the SMs
+  // next to the GEMM's CTAs and uses the DRAM bandwidth the GEMM leaves idle); the call joins the two streams at its end.
+  auto finish_dx = [&](bool after_last_gemm) -> moe_status {
+    if (forked == after_last_gemm) return MOE_OK;  // forked: right after the dgrad GEMM; in line: at the very end
+    cudaStream_t xs = st;
+    if (forked) {
+      if (cudaEventRecord(c->ev_b4, st) != cudaSuccess || cudaStreamWaitEvent(c->s_side, c->ev_b4, 0) != cudaSuccess)
+        return MOE_ERR_CUDA;
+      xs = c->s_side;
+    }
+    {
+      StageTimer tm(c, xs, 12);
+      if (tc_router && T > 0) {
+        launch_unpermute_sum(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv,
+                             reinterpret_cast<const uint16_t*>(ws + L.dxr), dx, xs,
+                             c->debug_checks ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr, L.rows_max);
+      } else {
+        launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, xs);
+      }
+    }
     if (forked && cudaEventRecord(c->ev_join, c->s_side) != cudaSuccess) return MOE_ERR_CUDA;
     return MOE_OK;
   };
@@ -553,6 +578,7 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
         if (rc == MOE_OK) rc = launch_lora_gemm(c, seq[g][1], T, L, ws, io, *lora, st);
       }
       if (g == 0 && rc == MOE_OK) rc = router_chain();
+      if (g == 2 && rc == MOE_OK) rc = finish_dx(false);
     }
     if (rc != MOE_OK) return rc;
   } else {
@@ -589,23 +615,17 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
       rc = launch_grouped_gemm(c, GEMM_B4, T, L, ws, io, st);
     }
     if (rc != MOE_OK) return rc;
+    rc = finish_dx(false);
+    if (rc != MOE_OK) return rc;
     {
       StageTimer tm(c, st, 9);
       rc = wgrad(GEMM_B5, n_groups);
     }
     if (rc != MOE_OK) return rc;
   }
+  rc = finish_dx(true);
+  if (rc != MOE_OK) return rc;
   if (forked && cudaStreamWaitEvent(st, c->ev_join, 0) != cudaSuccess) return MOE_ERR_CUDA;
-  {
-    StageTimer tm(c, st, 12);
-    if (tc_router && T > 0) {
-      launch_unpermute_sum(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv,
-                           reinterpret_cast<const uint16_t*>(ws + L.dxr), dx, st,
-                           c->debug_checks ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr, L.rows_max);
-    } else {
-      launch_unpermute_bwd(s, T, reinterpret_cast<const uint16_t*>(ws + L.dxp), inv, dl, W_r, dx, st);
-    }
-  }
   if (c->profiling) c->prof_step++;
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -94,7 +94,7 @@ struct moe_ctx_impl {
   int use_side_stream;  // backward runs the router's gradient chain on s_side, beside the big GEMMs
   int side_created;
   cudaStream_t s_side;
-  cudaEvent_t ev_fork, ev_join;
+  cudaEvent_t ev_fork, ev_join, ev_b4;
   int tile_mode;    // 0: choose per GEMM, 1: always CTA pairs (odd blocks as half-empty pairs), 2: always one-CTA tiles,
                     // 3: row GEMMs as full pairs + one-CTA tiles for the leftover blocks, weight gradients on pairs
   int gemm_timers;  // MOE_GEMM_TIMERS was set when the context first touched its device
