@@ -450,6 +450,26 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+    # A short look at the burst regime first (informative only, reported under "burst"): min(steps, 20) steps right after
+    # the warm-up, before the power cap has pulled the clocks down.  The headline below is the steady state.
+    burst = None
+    if args.condition_seconds > 0:
+        nb = max(3, min(args.steps, 20))
+        layer.set_profiling(True)
+        torch.cuda.synchronize()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        tb0 = time.perf_counter()
+        b0.record()
+        for _ in range(nb):
+            step()
+        b1.record()
+        torch.cuda.synchronize()
+        tb1 = time.perf_counter()
+        bst, bn = layer.stage_times()
+        layer.set_profiling(False)
+        burst = {"steps": nb, "ms_per_step": b0.elapsed_time(b1) / nb,
+                 "stages_ms": {STAGE_NAMES[i]: bst[i] / max(bn, 1) for i in range(len(STAGE_NAMES))},
+                 "window": (tb0, tb1)}
     # untimed conditioning: the same step back to back until the power state has settled
     cond_steps = 0
     if args.condition_seconds > 0:
@@ -480,6 +500,12 @@ def main():
     if rank == 0:
         sampler.stop()
         clocks = sampler.summary(t_host0, t_host1)
+        if burst is not None:
+            w0, w1 = burst.pop("window")
+            burst["sm_mhz"] = sampler.summary(w0, w1).get("sm_mhz")
+            burst["tokens_per_s"] = world * T / (burst["ms_per_step"] / 1e3)
+            burst["note"] = ("first steps after the warm-up, before the power cap settles the clock; not the headline "
+                             "(the headline value is the conditioned steady state)")
     layer.poll()
     layer.set_profiling(False)
     ms_step = pdist.max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
@@ -619,7 +645,7 @@ def main():
             "grouped_gemm_frac_of_sustained_bf16": gemm_tflops / peaks["bf16_tflops_sustained"],
             "grouped_gemm_frac_of_burst_bf16": gemm_tflops / peaks["bf16_tflops"],
             "grouped_gemm_frac_of_regime_peak": gemm_tflops / tensor_peak, "regime": regime,
-            "roofline": roof, "stages": stages, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+            "roofline": roof, "stages": stages, "burst": burst, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
             "gpu_launches": launches}
     print(json.dumps(line))
     pdist.finish()
