@@ -245,10 +245,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="qwen", choices=list(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--mode", default="train", choices=["train", "inference", "accumulate", "lora", "library-gemm"],
+    ap.add_argument("--ep-world", type=int, default=4, help="--mode ep: ranks of the expert-parallel group")
+    ap.add_argument("--mode", default="train", choices=["train", "inference", "accumulate", "lora", "library-gemm", "ep"],
                     help="train: forward + backward (the headline metric); inference: forward-only entry point; "
                          "accumulate: forward + backward that adds weight gradients into fp32 buffers; "
                          "lora: forward + backward of the expert-LoRA variant (rank 16, frozen expert weights); "
+                         "ep: the expert-parallel path with all ranks of the group run as a local group on ONE GPU (same "
+                         "kernels as a multi-GPU group, phases enqueued rank after rank; the batch is split evenly over the "
+                         "ranks, so the work equals one train step and the difference is the cost of the EP path itself); "
                          "library-gemm: calibration only - the library's batched bf16 GEMM (torch.bmm) at the three "
                          "row-GEMM shapes of the workload with uniform rows per expert, in the same steady state")
     ap.add_argument("--condition-seconds", type=float, default=2.0,
@@ -306,6 +310,48 @@ def main():
     grads = {"dx": torch.empty_like(tens["x"]), "dW_r": torch.empty(shape.d, shape.E, dtype=torch.float32, device="cuda"),
              "dW_gate": torch.empty_like(tens["W_gate"]), "dW_up": torch.empty_like(tens["W_up"]),
              "dW_down": torch.empty_like(tens["W_down"])}
+
+    if args.mode == "ep":
+        from paper_2608_00916_b200 import ep as pep
+        W = args.ep_world
+        assert shape.E % W == 0 and T % W == 0
+        per = T // W
+        xs = [tens["x"][r * per:(r + 1) * per].contiguous() for r in range(W)]
+        dys = [tens["dy"][r * per:(r + 1) * per].contiguous() for r in range(W)]
+        grp = pep.LocalGroup(shape.d, shape.E, shape.f, shape.k, W, pep.rows_cap_bound([per] * W, shape.k, shape.E, W))
+
+        def estep():
+            grp.forward(xs, tens["W_r"], tens["W_gate"], tens["W_up"], tens["W_down"], b_r=b_r)
+            grp.backward(dys, inp["d_aux"])
+        for _ in range(args.warmup):
+            estep()
+        grp.poll()
+        t_c = time.perf_counter()
+        while time.perf_counter() - t_c < args.condition_seconds:
+            for _ in range(5):
+                estep()
+            torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = kernel_launches()
+        f0.record()
+        for _ in range(args.steps):
+            estep()
+        f1.record()
+        torch.cuda.synchronize()
+        grp.poll()
+        ms = f0.elapsed_time(f1) / args.steps
+        print(json.dumps({"metric": "moe_layer_ep_local_group_fwd_bwd_tokens_per_s", "value": T / (ms / 1e3),
+                          "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "none", "vs_baseline": None, "dtype": "bf16",
+                          "data": "synthetic",
+                          "config": {"workload": args.workload, "mode": "ep", "ep_world": W, "tokens_per_rank": per,
+                                     "experts_per_rank": shape.E // W, "d": shape.d, "E": shape.E, "top_k": shape.k,
+                                     "f": shape.f,
+                                     "note": "all ranks of the group on one GPU, phases enqueued rank after rank; not a "
+                                             "multi-GPU measurement"},
+                          "gpu_launches": kernel_launches() - launches0}))
+        pdist.finish()
+        return
 
     if args.mode == "library-gemm":
         # What a plain library GEMM reaches at the expert shapes under the same power-capped steady state: no ragged

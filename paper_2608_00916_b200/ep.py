@@ -216,8 +216,8 @@ class LocalGroup:
         for rk, x in zip(R, xs):
             rk.dispatch(x)
         for r, rk in enumerate(R):
-            sl = slice(r * e_loc, (r + 1) * e_loc)
-            rk.expert_forward(W_gate[sl].contiguous(), W_up[sl].contiguous(), W_down[sl].contiguous())
+            sl = slice(r * e_loc, (r + 1) * e_loc)  # a slice along the leading axis is contiguous: a view, no copy
+            rk.expert_forward(W_gate[sl], W_up[sl], W_down[sl])
         ys = [rk.combine() for rk in R]
         return [dict(o, y=y) for o, y in zip(routed, ys)], all_counts
 
