@@ -237,8 +237,8 @@ class LocalGroup:
 class DistGroup:
     """One rank per process and GPU (torch.distributed initialised with the NCCL backend).  The owner workspace lives in
     symmetric memory so that every rank can map its peers' copies; the per-rank expert counts travel by all_gather; a
-    group barrier (stream synchronise + dist.barrier) separates the phases.  Not exercised in this repository's tests:
-    they have one GPU (LocalGroup runs the same kernels there)."""
+    group barrier (stream synchronise + dist.barrier) separates the phases.  The tests run it on a one-rank group (they
+    have one GPU; LocalGroup runs the same kernels for more ranks there)."""
 
     def __init__(self, d, E, f, top_k, rows_cap, flags: int = 0, group=None):
         import torch

@@ -109,3 +109,19 @@ def test_ep_with_one_rank_equals_the_plain_layer():
     assert torch.equal(sender[0]["dx"], bw["dx"]) and torch.equal(sender[0]["dW_r"], bw["dW_r"])
     for n in ("dW_gate", "dW_up", "dW_down"):
         assert torch.equal(owner[0][n], bw[n]), n
+
+
+def test_dist_group_with_one_rank():
+    """ep.DistGroup - the multi-process form (NCCL all_gather of the counts, owner workspace in symmetric memory and
+    mapped through its rendezvous, group barriers between phases) - on a one-rank group in a child process: bitwise the
+    plain layer.  More ranks need more GPUs than a test run has."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "tests", "ep_dist_probe.py"), str(29741 + os.getpid() % 200)],
+                         capture_output=True, text=True, timeout=600, cwd=root)
+    if "symmetric" in out.stderr.lower() and "not" in out.stderr.lower() and "DIST_GROUP" not in out.stdout:
+        pytest.skip("symmetric memory is not available in this torch build: " + out.stderr[-300:])
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "DIST_GROUP_OK" in out.stdout, out.stdout[-500:] + out.stderr[-1500:]
