@@ -153,11 +153,14 @@ __global__ void __launch_bounds__(KIND == GEMM_RT ? 192 : GEMM_THREADS, 1)
         if (lane == 0) {
           const uint32_t sA = smem_base + s * stage_stride;
           const uint32_t sB = sA + A_BYTES;
+          const int nks = kb == tl.nkb - 1 ? tl.klast : BK / 16;
 #pragma unroll
           for (int ks = 0; ks < BK / 16; ++ks) {
-            const uint64_t da = smem_desc(sA + ks * A_KSTEP, A_LBO, 1024);
-            const uint64_t db = smem_desc(sB + ks * B_KSTEP, B_LBO, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+            if (ks < nks) {
+              const uint64_t da = smem_desc(sA + ks * A_KSTEP, A_LBO, 1024);
+              const uint64_t db = smem_desc(sB + ks * B_KSTEP, B_LBO, 1024);
+              umma_bf16(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+            }
           }
           umma_commit(empty_bar(s));
         }

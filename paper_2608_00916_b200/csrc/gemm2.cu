@@ -30,6 +30,7 @@ constexpr size_t GEMM2_SMEM = static_cast<size_t>(STAGES2) * STAGE2_BYTES + EPI_
 
 struct Tile2 {
   int e, row0, m0, n0, nkb;
+  int klast;    // K = 16 steps issued in the last K block
   bool write;   // this CTA's 128 rows exist (false: the empty half of an odd expert's last pair)
   bool full;    // both halves of the pair exist
 };
@@ -43,6 +44,7 @@ __device__ __forceinline__ int total_tiles2(const GemmParams& p) {
 template <int KIND>
 __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank) {
   Tile2 tl;
+  tl.klast = BK / 16;
   if (Traits<KIND>::WGRAD) {
     const int per = p.m_tiles * p.n_tiles;
     const int slot = t / per;
@@ -52,6 +54,7 @@ __device__ __forceinline__ Tile2 get_tile2(const GemmParams& p, int t, int rank)
     tl.n0 = (rem % p.n_tiles) * Traits<KIND>::N_SPAN;
     tl.row0 = p.pad_offsets[tl.e];
     tl.nkb = (p.counts[tl.e] + BK - 1) / BK;  // the rest of the 128-row padding is zeros
+    tl.klast = last_k_steps(p.counts[tl.e]);
     tl.write = true;
     tl.full = true;
   } else {
@@ -228,11 +231,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM2_THREADS, 1)
           if (lane == 0) {
             const uint32_t sA = smem_base + s * STAGE2_BYTES;
             const uint32_t sB = sA + A_BYTES;
+            const int nks = kb == tl.nkb - 1 ? tl.klast : BK / 16;
 #pragma unroll
             for (int ks = 0; ks < BK / 16; ++ks) {
-              const uint64_t da = smem_desc(sA + ks * A_KSTEP, A_LBO, 1024);
-              const uint64_t db = smem_desc(sB + ks * B_KSTEP, B_LBO, 1024);
-              umma_bf16_pair(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+              if (ks < nks) {
+                const uint64_t da = smem_desc(sA + ks * A_KSTEP, A_LBO, 1024);
+                const uint64_t db = smem_desc(sB + ks * B_KSTEP, B_LBO, 1024);
+                umma_bf16_pair(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+              }
             }
             // the stage is free in both CTAs once these MMAs have read it
             umma_commit_pair_both(empty_bar(s));

@@ -93,8 +93,12 @@ struct Traits {
   static constexpr int N_SPAN = (KIND == GEMM_F3 || KIND == GEMM_B5 || KIND == GEMM_DWR) ? 128 : 256;
 };
 
+// K = 16 steps of the last 64-deep K block that hold any of an expert's `count` rows (the rows after them are zeros).
+__device__ __forceinline__ int last_k_steps(int count) { return count > 0 ? ((count - 1) % BK) / 16 + 1 : BK / 16; }
+
 struct Tile {
   int e, row0, m0, n0, nkb;
+  int klast = BK / 16;  // K = 16 steps issued in the last K block (weight gradients stop at the expert's last row)
 };
 
 // Static tile assignment of the persistent kernels: worker `w` of `nw` takes one tile per round.  Weight-gradient
@@ -146,6 +150,7 @@ __device__ __forceinline__ Tile get_tile(const GemmParams& p, int t) {
     } else {
       tl.row0 = p.pad_offsets[tl.e];
       tl.nkb = (p.counts[tl.e] + BK - 1) / BK;  // the rest of the 128-row padding is zeros
+      tl.klast = last_k_steps(p.counts[tl.e]);
     }
   } else if (Traits<KIND>::STATIC_M) {
     const int mt = t / p.n_tiles;
