@@ -20,8 +20,7 @@ import ctypes as C
 
 import numpy as np
 
-from . import binding
-from .binding import MoEConfig, MoEError, _check, _ptr, load_library
+from .binding import MoEConfig, _check, _ptr, load_library
 
 ROW_PAD = 128
 

@@ -3,7 +3,6 @@ import numpy as np
 import torch
 
 from oracle import moe_oracle as orc
-from paper_2608_00916_b200 import synth
 from paper_2608_00916_b200.binding import MoELayer
 
 

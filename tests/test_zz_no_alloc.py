@@ -8,7 +8,6 @@ dl (read back from the workspace), on two calls in a row with different shapes, 
 left in the shared scratch cannot leak into the second."""
 import ctypes as C
 
-import numpy as np
 import pytest
 import torch
 
