@@ -214,6 +214,19 @@ def host_cores():
         return os.cpu_count() or 1
 
 
+def workload_config(workload, mode, shape, world, parallelism_note="no data-path collective"):
+    """The `config` object of the JSON line: what identifies the workload.  Both arms print the same object for the same
+    command-line arguments; what differs between runs (conditioning steps, redrawn tokens, the reference arm's sample)
+    sits beside it."""
+    w_gb = 3 * shape.E * shape.d * shape.f * 2 / 1e9
+    l2_note = (f"inputs larger than L2 ({w_gb:.2f} GB of expert weights streamed per pass); no explicit flush"
+               if w_gb > 0.2 else f"working set ({w_gb * 1e3:.0f} MB of weights) fits in L2: L2-warm, launch-bound numbers")
+    return {"workload": workload, "mode": mode, "T_per_gpu": shape.T, "d": shape.d, "E": shape.E, "top_k": shape.k,
+            "f": shape.f,
+            "parallelism": f"dp{world} over tokens, experts replicated (EP=1), " + parallelism_note,
+            "l2": l2_note}
+
+
 def run_reference(args, shape, inp, workload):
     """--impl reference: the oracle is the timed arm (bounded sample per step)."""
     sample_T = min(shape.T, 2048)
@@ -229,10 +242,10 @@ def run_reference(args, shape, inp, workload):
     line = {"impl": "reference", "metric": "moe_layer_fwd_bwd_tokens_per_s", "value": val, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": workload, "T": shape.T, "d": shape.d, "E": shape.E, "top_k": shape.k, "f": shape.f,
-                       "sample_tokens_per_step": sample_T},
+            "config": workload_config(workload, "train", shape, args.gpus),
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                             "sample": f"first {sample_T} tokens of the batch, all {shape.E} experts' weights, fp32 numpy"},
+                             "sample": f"each step: the first {sample_T} of the batch's {shape.T} tokens, all {shape.E} "
+                                       f"experts' weights, fp32 numpy, forward + backward"},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -672,21 +685,15 @@ def main():
                "sample": f"first {sample_T} tokens of the batch through the fp32 numpy oracle, forward + backward, "
                          f"all {shape.E} experts' weights"}
 
-    w_gb = 3 * shape.E * shape.d * shape.f * 2 / 1e9
-    l2_note = (f"inputs larger than L2 ({w_gb:.2f} GB of expert weights streamed per pass); no explicit flush"
-               if w_gb > 0.2 else f"working set ({w_gb * 1e3:.0f} MB of weights) fits in L2: L2-warm, launch-bound numbers")
     line = {"metric": "moe_layer_fwd_bwd_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "mode": args.mode, "T_per_gpu": T, "d": shape.d, "E": shape.E, "top_k": shape.k,
-                       "f": shape.f,
-                       "parallelism": f"dp{world} over tokens, experts replicated (EP=1), "
-                                      + ("weight gradients all-reduced once per accumulation window, range by range "
-                                         "of experts while the backward pass still runs"
-                                         if reducer is not None else "no data-path collective"),
-                       "conditioning": f"{cond_steps} untimed steps (>= {args.condition_seconds} s) before the timed region",
-                       "l2": l2_note,
-                       "redrawn_tokens": inp["meta"]["redrawn"]},
+            "config": workload_config(args.workload, args.mode, shape, world,
+                                      "weight gradients all-reduced once per accumulation window, range by range of "
+                                      "experts while the backward pass still runs" if reducer is not None
+                                      else "no data-path collective"),
+            "conditioning": f"{cond_steps} untimed steps (>= {args.condition_seconds} s) before the timed region",
+            "redrawn_tokens": inp["meta"]["redrawn"],
             "grouped_gemm_tflops": gemm_tflops,
             "grouped_gemm_frac_of_sustained_bf16": gemm_tflops / peaks["bf16_tflops_sustained"],
             "grouped_gemm_frac_of_burst_bf16": gemm_tflops / peaks["bf16_tflops"],

@@ -20,6 +20,11 @@ def test_reference_arm_prints_the_contract_line():
     assert d["value"] > 0 and d["ms_per_step"] > 0 and d["config"]["workload"] == "tiny"
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["sample"]
     assert d["e2e"] == {"value": d["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    # the same `config` object as the GPU arm prints for the same arguments
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2608_00916_b200 import synth
+    assert d["config"] == bench.workload_config("tiny", "train", synth.CONFIGS["tiny"][0], 1)
 
 
 def test_reference_arm_on_other_ranks_does_nothing():
