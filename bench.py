@@ -557,7 +557,6 @@ def main():
     pdist.barrier()
     clocks = None
     if rank == 0:
-        sampler.stop()
         clocks = sampler.summary(t_host0, t_host1)
         if burst is not None:
             w0, w1 = burst.pop("window")
@@ -602,12 +601,16 @@ def main():
             run_pipelined(20)
         pdist.barrier()
         torch.cuda.synchronize()
-        n_e2e = max(4, min(args.steps, 20))
+        # as many steps as the device-resident region: the pipeline's fill (the first step's inputs) and drain (the last
+        # step's results) are inside the timed region and weigh 1/n of it
+        n_e2e = max(4, args.steps)
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_e0 = time.perf_counter()
         p0.record()
         run_pipelined(n_e2e)  # returns after the last step's results have reached the host buffers
         p1.record()
         torch.cuda.synchronize()
+        t_e1 = time.perf_counter()
         pdist.barrier()
         e2e_ms = pdist.max_over_ranks(p0.elapsed_time(p1)) / n_e2e
         layer.poll()
@@ -621,11 +624,15 @@ def main():
         blocking_ms = e0.elapsed_time(e1) / 3
         td = 2 * T * shape.d
         e2e = {"value": world * T / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": 2 * td,
-               "d2h_bytes_per_step": 2 * td + 4, "ms_per_step": e2e_ms, "ms_per_step_blocking_call": blocking_ms,
+               "d2h_bytes_per_step": 2 * td + 4, "steps": n_e2e, "ms_per_step": e2e_ms,
+               "ms_per_step_blocking_call": blocking_ms,
+               "sm_mhz": sampler.summary(t_e0, t_e1).get("sm_mhz") if rank == 0 else None,
                "note": "moe_step_host_begin/end with two slots in flight: x, dy in and y, dx, aux out every step; the closing "
                        "CUDA event is recorded after the last step's results reached the host; weights and weight "
                        "gradients stay on the device"}
         del dev_buf
+    if rank == 0:
+        sampler.stop()
 
     if rank != 0:
         pdist.finish()
