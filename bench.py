@@ -227,6 +227,17 @@ def workload_config(workload, mode, shape, world, parallelism_note="no data-path
             "l2": l2_note}
 
 
+def routing_report(counts, meta):
+    """The realised per-expert load of the last timed step (the GPU's own counts) and what the generator did to get it."""
+    c = np.asarray(counts, dtype=np.int64)
+    rows = int(c.sum())
+    padded = int(((c + 127) // 128 * 128).sum())
+    return {"rows_per_expert": {"min": int(c.min()), "max": int(c.max()), "mean": float(c.mean())},
+            "empty_experts": int((c == 0).sum()), "largest_five": sorted((int(v) for v in c), reverse=True)[:5],
+            "padding_rows_fraction": (padded - rows) / rows if rows else 0.0,
+            "zipf_bias_alpha": meta.get("alpha"), "redrawn_tokens": meta.get("redrawn")}
+
+
 def run_reference(args, shape, inp, workload):
     """--impl reference: the oracle is the timed arm (bounded sample per step)."""
     sample_T = min(shape.T, 2048)
@@ -700,7 +711,7 @@ def main():
                                       "experts while the backward pass still runs" if reducer is not None
                                       else "no data-path collective"),
             "conditioning": f"{cond_steps} untimed steps (>= {args.condition_seconds} s) before the timed region",
-            "redrawn_tokens": inp["meta"]["redrawn"],
+            "routing": routing_report(layer.buffer("counts", torch.int32).cpu().numpy(), inp["meta"]),
             "grouped_gemm_tflops": gemm_tflops,
             "grouped_gemm_frac_of_sustained_bf16": gemm_tflops / peaks["bf16_tflops_sustained"],
             "grouped_gemm_frac_of_burst_bf16": gemm_tflops / peaks["bf16_tflops"],
