@@ -30,10 +30,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram bytes per launch of the dominant kernel taken from the committed ncu capture (profiles/), by stage name;
 # None where no capture has been taken for the workload.
 NCU_TRAFFIC = {  # profiles/step_launch_list_and_dram_traffic_qwen.md, profiles/gemm_dram_traffic_skewed_and_coarse.md
-    ("qwen", "gemm_gateup_swiglu"): 2.148e9, ("qwen", "gemm_down"): 1.149e9, ("qwen", "dgrad_down_swiglu_bwd"): 1.912e9,
-    ("qwen", "wgrad_down"): 1.135e9, ("qwen", "dgrad_gateup"): 1.780e9, ("qwen", "wgrad_gateup"): 1.742e9,
-    ("skewed", "gemm_gateup_swiglu"): 2.012e9, ("skewed", "gemm_down"): 1.138e9, ("skewed", "dgrad_down_swiglu_bwd"): 1.885e9,
-    ("skewed", "wgrad_down"): 1.204e9, ("skewed", "dgrad_gateup"): 1.758e9, ("skewed", "wgrad_gateup"): 2.066e9,
+    ("qwen", "gemm_gateup_swiglu"): 2.049e9, ("qwen", "gemm_down"): 1.148e9, ("qwen", "dgrad_down_swiglu_bwd"): 1.885e9,
+    ("qwen", "wgrad_down"): 1.134e9, ("qwen", "dgrad_gateup"): 1.797e9, ("qwen", "wgrad_gateup"): 1.750e9,
+    ("skewed", "gemm_gateup_swiglu"): 1.992e9, ("skewed", "gemm_down"): 1.138e9, ("skewed", "dgrad_down_swiglu_bwd"): 1.878e9,
+    ("skewed", "wgrad_down"): 1.196e9, ("skewed", "dgrad_gateup"): 1.765e9, ("skewed", "wgrad_gateup"): 2.027e9,
 }
 
 

@@ -97,6 +97,7 @@ moe_status ensure_device(moe_ctx_impl* c) {
   c->encode_fn = fn;
   c->gemm_timers = getenv("MOE_GEMM_TIMERS") != nullptr;
   c->row_group_override = getenv("MOE_ROW_GROUP") ? atoi(getenv("MOE_ROW_GROUP")) : 0;
+  c->b4_pair_override = getenv("MOE_B4_PAIR") ? atoi(getenv("MOE_B4_PAIR")) : -1;
   if (c->use_side_stream) {
     if (cudaStreamCreateWithFlags(&c->s_side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||

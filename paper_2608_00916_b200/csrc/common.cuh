@@ -99,6 +99,7 @@ struct moe_ctx_impl {
                     // 3: row GEMMs as full pairs + one-CTA tiles for the leftover blocks, weight gradients on pairs
   int gemm_timers;  // MOE_GEMM_TIMERS was set when the context first touched its device
   int row_group_override;  // MOE_ROW_GROUP, if set (measurements of the tile order)
+  int b4_pair_override;    // MOE_B4_PAIR = 0 / 1, if set (measurements: dgrad gate/up on one-CTA tiles / CTA pairs); else -1
   // cudaFuncSetAttribute (dynamic shared memory opt-in) is per device: remembered here, for the device the context is
   // bound to, per kernel family (0: one-CTA kernels, 1: CTA-pair kernels) and GEMM kind
   unsigned char attr_done[2][16];

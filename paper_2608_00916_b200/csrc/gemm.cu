@@ -560,9 +560,11 @@ moe_status launch_grouped_gemm(moe_ctx_impl* ctx, GemmKind kind, int64_t T, cons
   }
   if (!row_kind) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 0);
   if (ctx->tile_mode == 1) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
-  // dgrad gate/up is the exception at short K: with 2 f / 64 < 64 K blocks per tile its pair form needs fewer cycles
-  // but more time under the power cap than its one-CTA form (Qwen3-30B-A3B shape: 842 vs 811 us in steady state)
-  const bool long_k = kind != GEMM_B4 || 2 * ctx->s.f / BK >= 64;
+  // dgrad gate/up at short K (2 f / 64 < 64 K blocks per tile) gains from pairs only from 768 rows per expert on
+  // (Qwen3-30B-A3B shape, steady state under the power cap: 453 vs 443 us at 512 rows per expert, 838 vs 875 us at
+  // 1024, 1590 vs 1709 us at 2048)
+  bool long_k = kind != GEMM_B4 || 2 * ctx->s.f / BK >= 64 || rows_per_expert >= 768.0;
+  if (kind == GEMM_B4 && ctx->b4_pair_override >= 0) long_k = ctx->b4_pair_override != 0;
   if (ctx->tile_mode == 0 && rows_per_expert >= 512.0 && long_k)
     return launch_gemm_variant(ctx, kind, T, L, ws, io, st, true, 0);
   if (ctx->tile_mode != 3) return launch_gemm_variant(ctx, kind, T, L, ws, io, st, false, 0);
