@@ -251,6 +251,60 @@ def test_repeated_calls_are_bitwise_reproducible():
         assert torch.equal(ga[n], gb[n]), n
 
 
+def test_one_context_across_changing_token_counts():
+    """A training loop feeds a different number of tokens every step: the same context (its workspace grows to the
+    largest) alternates between token counts, each step stage by stage against the oracle and bitwise equal to a fresh
+    context's result - no table, tensor map or count of an earlier step leaks into the next."""
+    d, E, k, f = 256, 16, 4, 192
+    layer = MoELayer(d, E, f, k)
+    weights = synth.make_inputs(synth.MoEShape(8, d, E, k, f), 41)
+    for step, T in enumerate([900, 130, 1411, 1, 900]):
+        tok = synth.make_tokens(synth.MoEShape(T, d, E, k, f), 500 + step, weights["W_r"], None)
+        inp = dict(weights, x=tok["x"], dy=tok["dy"])
+        ofw, obw = oracle_run(inp, k, 0.05)
+        r = Run(inp, k)
+        fresh_fw, fresh_bw = check_all(r, ofw, obw, 0.05)
+        dev = r.dev
+        fw = layer.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
+        bw = layer.backward(dev["dy"], 0.05)
+        layer.poll()
+        for n in ("y", "idx", "gates", "perm", "aux", "counts"):
+            assert torch.equal(fw[n], fresh_fw[n]), (T, n)
+        for n in ("dx", "dW_r", "dW_gate", "dW_up", "dW_down"):
+            assert torch.equal(bw[n], fresh_bw[n]), (T, n)
+
+
+def test_two_contexts_on_two_streams():
+    """One context per stream: two layers of different shapes enqueue their steps interleaved on two streams and give
+    bitwise the results of running alone."""
+    cases = [(synth.MoEShape(1200, 256, 16, 4, 256), 51), (synth.MoEShape(700, 384, 8, 2, 320), 52)]
+    runs = [Run(synth.make_inputs(sh, seed), sh.k) for sh, seed in cases]
+    alone = []
+    for r in runs:
+        fw = r.forward()
+        bw = r.backward(0.03)
+        alone.append(({n: fw[n].clone() for n in ("y", "idx", "gates", "aux")},
+                      {n: bw[n].clone() for n in ("dx", "dW_r", "dW_gate", "dW_up", "dW_down")}))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [None, None]
+    for rep in range(3):
+        for i, r in enumerate(runs):
+            with torch.cuda.stream(streams[i]):
+                fw = r.forward()
+                outs[i] = (fw, None)
+        for i, r in enumerate(runs):
+            with torch.cuda.stream(streams[i]):
+                outs[i] = (outs[i][0], r.backward(0.03))
+    torch.cuda.synchronize()
+    for i, r in enumerate(runs):
+        r.layer.poll()
+        for n, v in alone[i][0].items():
+            assert torch.equal(outs[i][0][n], v), (i, n)
+        for n, v in alone[i][1].items():
+            assert torch.equal(outs[i][1][n], v), (i, n)
+
+
 @pytest.mark.parametrize("T,d,E,k,f,seed", [(1000, 512, 16, 4, 384, 14), (777, 256, 64, 8, 192, 27)])
 def test_forward_inference_entry(T, d, E, k, f, seed):
     """moe_forward_inference: same y and routing as the training forward, from a workspace of only the inference size
