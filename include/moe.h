@@ -56,9 +56,10 @@ typedef struct {
 
 /* Tile shape of the expert GEMMs.  By default the library chooses per GEMM between CTA pairs (256 x 256 tiles,
  * tcgen05 cta_group::2, each CTA staging half of B) and one-CTA 128 x 256 tiles: weight gradients run on pairs when
- * the experts average at least 768 rows, row GEMMs when few experts share many rows (the dummy half-tile of an expert
- * with an odd number of 128-row blocks then costs < 3 %).  The flags force one shape everywhere (same results; for
- * comparison measurements). */
+ * the experts average at least 768 rows, row GEMMs from 512 rows per expert (the dgrad of gate / up with fewer than 64
+ * K blocks per tile from 768); an expert with an odd number of 128-row blocks gets a last pair whose second half is
+ * empty.  Below those sizes the layer is bound by streaming the weights and one-CTA tiles are used.  The flags force
+ * one shape everywhere (same results; for comparison measurements). */
 #define MOE_FLAG_CTA_PAIR_TILES 1
 #define MOE_FLAG_SINGLE_CTA_TILES 2
 /* Row GEMMs run every complete pair of 128-row blocks of an expert on a CTA pair and the leftover block of an odd
