@@ -310,6 +310,13 @@ MOE_API moe_status moe_ep_combine(moe_ctx* ctx, int64_t T, void* const* peer_own
 MOE_API moe_status moe_ep_expert_backward(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up,
                                           const uint16_t* W_down, uint16_t* dW_gate, uint16_t* dW_up,
                                           uint16_t* dW_down, void* own_ws, size_t own_ws_bytes, void* cuda_stream);
+/* The same with the owned experts' weight gradients ADDED into fp32 buffers of the same shapes (the main gradients an
+ * expert-parallel rank keeps for its own experts over an accumulation window: they need no reduction inside the group);
+ * the caller zeroes them at the start of a window.  Slabs of experts without rows are left untouched. */
+MOE_API moe_status moe_ep_expert_backward_accumulate(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up,
+                                                     const uint16_t* W_down, float* dW_gate, float* dW_up,
+                                                     float* dW_down, void* own_ws, size_t own_ws_bytes,
+                                                     void* cuda_stream);
 /* Router gradient and dx of the rank's tokens: dx [T,d] bf16, dW_r [d,E] fp32, db_r [E] fp32 or NULL (overwritten). */
 MOE_API moe_status moe_ep_router_backward(moe_ctx* ctx, int64_t T, float d_aux, const uint16_t* x, const uint16_t* W_r,
                                           void* const* peer_own_ws /* host */, void* send_ws, size_t send_ws_bytes,

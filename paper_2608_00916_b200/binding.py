@@ -26,7 +26,7 @@ EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_fi
            "moe_step_host_begin", "moe_step_host_end", "moe_kernel_launches", "moe_ctx_device",
            "moe_e2e_workspace_offset", "moe_ep_create", "moe_ep_send_workspace_bytes", "moe_ep_own_workspace_bytes",
            "moe_ep_workspace_find", "moe_ep_route", "moe_ep_plan", "moe_ep_dispatch", "moe_ep_expert_forward",
-           "moe_ep_combine", "moe_ep_expert_backward", "moe_ep_router_backward",
+           "moe_ep_combine", "moe_ep_expert_backward", "moe_ep_expert_backward_accumulate", "moe_ep_router_backward",
            "moe_backward_accumulate_grouped"]
 EP_MAX_RANKS = 16  # MOE_EP_MAX_RANKS of include/moe.h
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
@@ -120,6 +120,8 @@ def load_library() -> C.CDLL:
     lib.moe_ep_combine.restype = C.c_int
     lib.moe_ep_expert_backward.argtypes = [vp] + [vp] * 6 + [vp, sz, vp]
     lib.moe_ep_expert_backward.restype = C.c_int
+    lib.moe_ep_expert_backward_accumulate.argtypes = [vp] + [vp] * 6 + [vp, sz, vp]
+    lib.moe_ep_expert_backward_accumulate.restype = C.c_int
     lib.moe_ep_router_backward.argtypes = [vp, i64, C.c_float, vp, vp, C.POINTER(vp), vp, sz, vp, vp, vp, vp]
     lib.moe_ep_router_backward.restype = C.c_int
     lib.moe_selftest_timeout.argtypes = [vp, vp, vp]

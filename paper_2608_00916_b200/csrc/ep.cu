@@ -405,14 +405,16 @@ moe_status moe_ep_combine(moe_ctx* ctx, int64_t T, void* const* peer_own_ws, con
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
-moe_status moe_ep_expert_backward(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
-                                  uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, void* own_ws,
-                                  size_t own_ws_bytes, void* cuda_stream) {
+static moe_status ep_expert_backward_impl(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up,
+                                          const uint16_t* W_down, uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down,
+                                          float* acc_gate, float* acc_up, float* acc_down, void* own_ws,
+                                          size_t own_ws_bytes, void* cuda_stream) {
   moe_ctx_impl* c = reinterpret_cast<moe_ctx_impl*>(ctx);
-  if (!c || !c->own || !W_gate || !W_up || !W_down || !dW_gate || !dW_up || !dW_down || !own_ws)
-    return MOE_ERR_INVALID_ARG;
+  const bool accumulate = acc_gate != nullptr;
+  if (!c || !c->own || !W_gate || !W_up || !W_down || !own_ws) return MOE_ERR_INVALID_ARG;
+  if (accumulate ? (!acc_up || !acc_down) : (!dW_gate || !dW_up || !dW_down)) return MOE_ERR_INVALID_ARG;
   if (!aligned16(W_gate) || !aligned16(W_up) || !aligned16(W_down) || !aligned16(dW_gate) || !aligned16(dW_up) ||
-      !aligned16(dW_down) || !aligned16(own_ws))
+      !aligned16(dW_down) || !aligned16(acc_gate) || !aligned16(acc_up) || !aligned16(acc_down) || !aligned16(own_ws))
     return MOE_ERR_INVALID_ARG;
   const EpLayouts l = ep_layouts(c, 0);
   if (own_ws_bytes < l.own.total) return MOE_ERR_WORKSPACE;
@@ -423,6 +425,7 @@ moe_status moe_ep_expert_backward(moe_ctx* ctx, const uint16_t* W_gate, const ui
   GemmIO io;
   io.W_gate = W_gate; io.W_up = W_up; io.W_down = W_down;
   io.dW_gate = dW_gate; io.dW_up = dW_up; io.dW_down = dW_down;
+  io.dW_gate_acc = acc_gate; io.dW_up_acc = acc_up; io.dW_down_acc = acc_down;
   const bool rows = c->ep_rows_cap > 0;  // row GEMMs have no tiles without rows; the weight gradients zero-fill
   if (rows) rc = launch_grouped_gemm(c->own, GEMM_B2, l.T_equiv, l.own, ws, io, st);
   if (rc == MOE_OK) rc = launch_grouped_gemm(c->own, GEMM_B3, l.T_equiv, l.own, ws, io, st);
@@ -430,6 +433,22 @@ moe_status moe_ep_expert_backward(moe_ctx* ctx, const uint16_t* W_gate, const ui
   if (rc == MOE_OK) rc = launch_grouped_gemm(c->own, GEMM_B5, l.T_equiv, l.own, ws, io, st);
   if (rc != MOE_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+moe_status moe_ep_expert_backward(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up, const uint16_t* W_down,
+                                  uint16_t* dW_gate, uint16_t* dW_up, uint16_t* dW_down, void* own_ws,
+                                  size_t own_ws_bytes, void* cuda_stream) {
+  if (!dW_gate || !dW_up || !dW_down) return MOE_ERR_INVALID_ARG;
+  return ep_expert_backward_impl(ctx, W_gate, W_up, W_down, dW_gate, dW_up, dW_down, nullptr, nullptr, nullptr, own_ws,
+                                 own_ws_bytes, cuda_stream);
+}
+
+moe_status moe_ep_expert_backward_accumulate(moe_ctx* ctx, const uint16_t* W_gate, const uint16_t* W_up,
+                                             const uint16_t* W_down, float* dW_gate, float* dW_up, float* dW_down,
+                                             void* own_ws, size_t own_ws_bytes, void* cuda_stream) {
+  if (!dW_gate || !dW_up || !dW_down) return MOE_ERR_INVALID_ARG;
+  return ep_expert_backward_impl(ctx, W_gate, W_up, W_down, nullptr, nullptr, nullptr, dW_gate, dW_up, dW_down, own_ws,
+                                 own_ws_bytes, cuda_stream);
 }
 
 moe_status moe_ep_router_backward(moe_ctx* ctx, int64_t T, float d_aux, const uint16_t* x, const uint16_t* W_r,

@@ -163,9 +163,18 @@ class EPRank:
                                                  _ptr(y), self._stream()), "moe_ep_combine")
         return y
 
-    def expert_backward(self):
+    def expert_backward(self, acc=None):
+        """acc: dict of fp32 dW_gate / dW_up / dW_down of the owned experts' shapes to ADD the gradients into (the
+        main gradients of an accumulation window); None: new bf16 tensors, overwritten."""
         import torch
         W_gate, W_up, W_down = self._W
+        if acc is not None:
+            for n, w in (("dW_gate", W_gate), ("dW_up", W_up), ("dW_down", W_down)):
+                assert acc[n].dtype == torch.float32 and tuple(acc[n].shape) == tuple(w.shape) and acc[n].is_contiguous()
+            _check(self.lib, self.lib.moe_ep_expert_backward_accumulate(
+                self.h, _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(acc["dW_gate"]), _ptr(acc["dW_up"]), _ptr(acc["dW_down"]),
+                _ptr(self.own_ws), self.own_ws.numel(), self._stream()), "moe_ep_expert_backward_accumulate")
+            return acc
         out = {"dW_gate": torch.empty_like(W_gate), "dW_up": torch.empty_like(W_up), "dW_down": torch.empty_like(W_down)}
         _check(self.lib, self.lib.moe_ep_expert_backward(self.h, _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(out["dW_gate"]),
                                                          _ptr(out["dW_up"]), _ptr(out["dW_down"]), _ptr(self.own_ws),
@@ -220,11 +229,12 @@ class LocalGroup:
         ys = [rk.combine() for rk in R]
         return [dict(o, y=y) for o, y in zip(routed, ys)], all_counts
 
-    def backward(self, dys, d_aux: float, want_db: bool = False):
+    def backward(self, dys, d_aux: float, want_db: bool = False, acc=None):
+        """acc: one dict of fp32 main gradients per rank (see EPRank.expert_backward), or None."""
         R = self.ranks
         for rk, dy in zip(R, dys):
             rk.dispatch(dy, backward=True)
-        owner = [rk.expert_backward() for rk in R]
+        owner = [rk.expert_backward(None if acc is None else acc[r]) for r, rk in enumerate(R)]
         sender = [rk.router_backward(d_aux, want_db) for rk in R]
         return sender, owner
 
@@ -272,11 +282,11 @@ class DistGroup:
         out["y"] = rk.combine()
         return out
 
-    def backward(self, dy, d_aux: float, want_db: bool = False):
+    def backward(self, dy, d_aux: float, want_db: bool = False, acc=None):
         rk = self.rk
         self._barrier()  # every rank has finished reading the forward outputs it combines
         rk.dispatch(dy, backward=True)
         self._barrier()
-        owner = rk.expert_backward()
+        owner = rk.expert_backward(acc)
         self._barrier()
         return rk.router_backward(d_aux, want_db), owner

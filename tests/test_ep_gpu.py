@@ -125,3 +125,50 @@ def test_dist_group_with_one_rank():
         pytest.skip("symmetric memory is not available in this torch build: " + out.stderr[-300:])
     assert out.returncode == 0, out.stderr[-2000:]
     assert "DIST_GROUP_OK" in out.stdout, out.stdout[-500:] + out.stderr[-1500:]
+
+
+def test_ep_main_gradients_accumulate_over_micro_batches():
+    """moe_ep_expert_backward_accumulate: over a window of three micro-batches (uneven batches on two ranks) every rank's
+    fp32 main gradients of its own experts equal the oracle's gradients summed over the window; experts that saw no row
+    in the whole window keep the value the buffers started with."""
+    d, E, k, f, world = 128, 16, 2, 192, 2
+    e_loc = E // world
+    batches = [[90, 40], [10, 200], [128, 128]]
+    weights = synth.make_inputs(synth.MoEShape(8, d, E, k, f), 61)
+    # a bias that leaves the last two experts without tokens in every micro-batch
+    b_r = np.zeros(E, dtype=np.float32)
+    b_r[-2:] = -50.0
+    wdev = {n: to_dev_bf16(weights[n]) for n in ("W_r", "W_gate", "W_up", "W_down")}
+    b_dev = torch.from_numpy(b_r).cuda()
+    cap = ep.rows_cap_bound([max(b[r] for b in batches) for r in range(world)], k, E, world)
+    grp = ep.LocalGroup(d, E, f, k, world, cap)
+    acc = [{n: torch.zeros((e_loc,) + tuple(wdev[w].shape[1:]), dtype=torch.float32, device="cuda")
+            for n, w in (("dW_gate", "W_gate"), ("dW_up", "W_up"), ("dW_down", "W_down"))} for _ in range(world)]
+    sentinel = 0.25  # a recognisable start value in the slabs of the two experts that never get a row
+    for t in acc[world - 1].values():
+        t[-2:] = sentinel
+    ref = {n: np.zeros(weights[w].shape, dtype=np.float64) for n, w in (("dW_gate", "W_gate"), ("dW_up", "W_up"), ("dW_down", "W_down"))}
+    for step, tokens in enumerate(batches):
+        T = sum(tokens)
+        tok = synth.make_tokens(synth.MoEShape(T, d, E, k, f), 700 + step, weights["W_r"], b_r)
+        inp = dict(weights, x=tok["x"], dy=tok["dy"], b_r=b_r)
+        ofw, obw = oracle_run(inp, k, 0.0)
+        assert ofw["counts"][-2:].sum() == 0
+        for n in ref:
+            ref[n] += obw[n]
+        x, dy = to_dev_bf16(tok["x"]), to_dev_bf16(tok["dy"])
+        bounds = np.concatenate([[0], np.cumsum(tokens)])
+        xs = [x[bounds[r]:bounds[r + 1]].contiguous() for r in range(world)]
+        dys = [dy[bounds[r]:bounds[r + 1]].contiguous() for r in range(world)]
+        grp.forward(xs, wdev["W_r"], wdev["W_gate"], wdev["W_up"], wdev["W_down"], b_r=b_dev)
+        grp.backward(dys, 0.0, acc=acc)
+        grp.poll()
+    for r in range(world):
+        own = slice(r * e_loc, (r + 1) * e_loc)
+        for n in ref:
+            got = acc[r][n].cpu().numpy().astype(np.float64)
+            if r == world - 1:
+                assert np.all(got[-2:] == sentinel), n  # untouched
+                assert rel_fro(got[:-2], ref[n][own][:-2]) <= TOL, (r, n)
+            else:
+                assert rel_fro(got, ref[n][own]) <= TOL, (r, n)
