@@ -322,6 +322,21 @@ MOE_API moe_status moe_ep_router_backward(moe_ctx* ctx, int64_t T, float d_aux, 
                                           void* const* peer_own_ws /* host */, void* send_ws, size_t send_ws_bytes,
                                           uint16_t* dx, float* dW_r, float* db_r, void* cuda_stream);
 
+/* Listwise training loss on grouped reranker scores (paper, paragraph "Contrastive and distillation losses").
+ * scores [n,G] fp32 DEVICE, one row per query (G passages per query).
+ *   MOE_LISTWISE_CONTRASTIVE: the positive passage sits at position 0 of every row;
+ *       loss = (1/n) sum_g ( logsumexp(s_g) - s_g[0] );  teacher and the temperatures are ignored.
+ *   MOE_LISTWISE_DISTILL: teacher [n,G] fp32 DEVICE holds stored teacher scores;
+ *       loss = (s_temp^2 / n) sum_g KL( softmax(t_g / t_temp) || softmax(s_g / s_temp) );  s_temp, t_temp > 0.
+ * loss [1] fp32 DEVICE is overwritten; dscores [n,G] fp32 DEVICE (or NULL) receives dloss/dscores.  n = 0 gives loss 0.
+ * One small kernel on cuda_stream, no workspace, no host synchronisation; the sum over the rows runs in a fixed order
+ * (same bits on every run).  Invalid arguments (unknown kind, G < 1, a non-positive temperature, a missing pointer)
+ * return MOE_ERR_INVALID_ARG before anything is launched. */
+#define MOE_LISTWISE_CONTRASTIVE 0
+#define MOE_LISTWISE_DISTILL 1
+MOE_API moe_status moe_listwise_loss(int32_t kind, int64_t n, int32_t G, const float* scores, const float* teacher,
+                                     float s_temp, float t_temp, float* loss, float* dscores, void* cuda_stream);
+
 /* Host-buffer convenience used for end-to-end timing: every tensor argument is a HOST pointer (pinned
  * memory recommended); the call copies inputs to the device buffers of `dev` (a device scratch of
  * moe_e2e_device_bytes(ctx, T) bytes owned by the caller), runs forward and backward, copies y, dx, aux and

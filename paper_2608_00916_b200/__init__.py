@@ -5,7 +5,7 @@ library in-tree.  Importing the package loads nothing heavy."""
 
 
 def __getattr__(name):
-    if name in ("MoELayer", "load_library", "MoEError"):
+    if name in ("MoELayer", "load_library", "MoEError", "listwise_loss"):
         from . import binding
         return getattr(binding, name)
     raise AttributeError(name)

@@ -27,7 +27,7 @@ EXPORTS = ["moe_create", "moe_destroy", "moe_workspace_bytes", "moe_workspace_fi
            "moe_e2e_workspace_offset", "moe_ep_create", "moe_ep_send_workspace_bytes", "moe_ep_own_workspace_bytes",
            "moe_ep_workspace_find", "moe_ep_route", "moe_ep_plan", "moe_ep_dispatch", "moe_ep_expert_forward",
            "moe_ep_combine", "moe_ep_expert_backward", "moe_ep_expert_backward_accumulate", "moe_ep_router_backward",
-           "moe_backward_accumulate_grouped"]
+           "moe_backward_accumulate_grouped", "moe_listwise_loss"]
 EP_MAX_RANKS = 16  # MOE_EP_MAX_RANKS of include/moe.h
 STATIC_MAX_DE = 262144  # MOE_STATIC_MAX_DE of include/moe.h
 
@@ -124,6 +124,8 @@ def load_library() -> C.CDLL:
     lib.moe_ep_expert_backward_accumulate.restype = C.c_int
     lib.moe_ep_router_backward.argtypes = [vp, i64, C.c_float, vp, vp, C.POINTER(vp), vp, sz, vp, vp, vp, vp]
     lib.moe_ep_router_backward.restype = C.c_int
+    lib.moe_listwise_loss.argtypes = [C.c_int32, i64, C.c_int32, vp, vp, C.c_float, C.c_float, vp, vp, vp]
+    lib.moe_listwise_loss.restype = C.c_int
     lib.moe_selftest_timeout.argtypes = [vp, vp, vp]
     lib.moe_selftest_timeout.restype = C.c_int
     lib.moe_router_wgrad_static.argtypes = [i64, C.c_int32, C.c_int32, vp, vp, vp, vp]
@@ -144,6 +146,26 @@ def kernel_launches() -> int:
 
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def listwise_loss(scores, teacher=None, s_temp: float = 1.0, t_temp: float = 1.0, want_grad: bool = True):
+    """moe_listwise_loss on CUDA tensors: scores [n, G] fp32 (one row per query).  Without `teacher`: listwise
+    cross-entropy with the positive at position 0; with teacher [n, G] fp32: temperature-scaled KL to the teacher's
+    distribution.  Returns (loss [1] fp32, dloss/dscores [n, G] fp32 or None)."""
+    import torch
+    lib = load_library()
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.dim() == 2 and scores.is_contiguous()
+    n, G = scores.shape
+    kind = 0
+    if teacher is not None:
+        assert teacher.is_cuda and teacher.dtype == torch.float32 and tuple(teacher.shape) == (n, G) and teacher.is_contiguous()
+        kind = 1
+    loss = torch.empty(1, dtype=torch.float32, device=scores.device)
+    grad = torch.empty_like(scores) if want_grad else None
+    _check(lib, lib.moe_listwise_loss(kind, n, G, _ptr(scores), _ptr(teacher), C.c_float(s_temp), C.c_float(t_temp),
+                                      _ptr(loss), _ptr(grad), C.c_void_p(torch.cuda.current_stream().cuda_stream)),
+           "moe_listwise_loss")
+    return loss, grad
 
 
 def router_wgrad_static(x, dl, dW_r=None):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoe_b200.so")
-SOURCES = ["api.cu", "route.cu", "combine.cu", "gemm.cu", "gemm2.cu", "noalloc.cu", "ep.cu"]
+SOURCES = ["api.cu", "route.cu", "combine.cu", "gemm.cu", "gemm2.cu", "noalloc.cu", "ep.cu", "listwise.cu"]
 HEADERS = ["common.cuh", "ptx.cuh", "gemm_common.cuh", "tables.cuh", os.path.join("..", "..", "include", "moe.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
