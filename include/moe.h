@@ -89,7 +89,7 @@ typedef enum {
   MOE_ERR_WORKSPACE = -3,   /* workspace_bytes smaller than moe_workspace_bytes(ctx, T) */
   MOE_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                       */
   MOE_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait ran out                     */
-  MOE_ERR_DEVICE_BOUNDS = -6   /* a device-side bounds check failed (MOE_FLAG_DEBUG_CHECKS) */
+  MOE_ERR_DEVICE_BOUNDS = -6   /* a device-side bounds check failed (MOE_FLAG_DEBUG_CHECKS; moe_ep_plan: rows beyond rows_cap) */
 } moe_status;
 
 /* Number of per-stage timers filled by moe_stage_times (see below). */
@@ -276,7 +276,11 @@ MOE_API moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, floa
  * Workspaces (caller-allocated): the SENDER workspace (moe_ep_send_workspace_bytes(ctx, T): routing state of the
  * rank's tokens) and the OWNER workspace (moe_ep_own_workspace_bytes(ctx): tables and row buffers of the owned
  * experts, sized for rows_cap received rows - the caller's bound on sum over ranks of rows routed to this rank, at
- * most sum_r T_r * min(top_k, E/world); it is the owner workspace that peers map). */
+ * most sum_r T_r * min(top_k, E/world); it is the owner workspace that peers map).  rows_cap must be the same on every
+ * rank of the group.  A step whose rows do not fit (the rows of the experts of ANY rank, each expert padded to 128,
+ * exceed the owner buffers) is refused by moe_ep_plan on every rank alike - every rank sees the same counts: nothing
+ * is dispatched, no owner buffer is written, y, dx and the weight gradients of the step come out as zeros, and
+ * moe_poll_status on the sender workspace returns MOE_ERR_DEVICE_BOUNDS (once; the context stays usable). */
 #define MOE_EP_MAX_RANKS 16
 MOE_API moe_status moe_ep_create(const moe_config* cfg /* host */, int32_t world, int32_t rank, int64_t rows_cap,
                                  moe_ctx** out /* host */);

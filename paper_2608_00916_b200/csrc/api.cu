@@ -247,7 +247,7 @@ const char* moe_status_string(moe_status s) {
     case MOE_ERR_WORKSPACE: return "workspace too small";
     case MOE_ERR_CUDA: return "CUDA call failed";
     case MOE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
-    case MOE_ERR_DEVICE_BOUNDS: return "a device-side bounds check failed (debug checks)";
+    case MOE_ERR_DEVICE_BOUNDS: return "a device-side bounds check failed (debug checks, or expert-parallel rows beyond the owner buffers)";
   }
   return "unknown status";
 }

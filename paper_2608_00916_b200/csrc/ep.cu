@@ -38,11 +38,18 @@ struct EpPeers {
 
 // ---------------------------------------------------------------------------------------------- plan
 // One block.  all_counts[r * E + e]: rows rank r routes to expert e.
+// Every rank sees the same table, so every rank reaches the same verdict on whether the rows fit: if the padded rows
+// of ANY owner exceed the capacity of the owner buffers (own_rows_max rows, the same on every rank of the group), the
+// whole step is refused on every rank - all destinations become -1 (nothing is dispatched, combined outputs are zero),
+// the owned experts get empty tables, and the sender workspace's status word records DEV_BOUNDS.
 __global__ void __launch_bounds__(256) ep_plan_kernel(const int32_t* __restrict__ all_counts, int W, int rank, int E,
-                                                      int E_loc, int32_t* __restrict__ dest_base, const TableOut tabs) {
+                                                      int E_loc, int64_t own_rows_max, int32_t* __restrict__ dest_base,
+                                                      const TableOut tabs, int32_t* __restrict__ status) {
   __shared__ int s_tot[MAX_E], s_before[MAX_E], s_cnt[MAX_E];
   __shared__ TableScratch s_tab;
+  __shared__ int s_over;
   const int tid = threadIdx.x;
+  if (tid == 0) s_over = 0;
   for (int e = tid; e < E; e += blockDim.x) {
     int tot = 0, before = 0;
     for (int r = 0; r < W; ++r) {
@@ -54,13 +61,21 @@ __global__ void __launch_bounds__(256) ep_plan_kernel(const int32_t* __restrict_
     s_before[e] = before;
   }
   __syncthreads();
+  if (tid < W) {
+    int64_t rows = 0;
+    for (int q = tid * E_loc; q < (tid + 1) * E_loc; ++q) rows += (s_tot[q] + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
+    if (rows > own_rows_max) atomicExch(&s_over, 1);
+  }
+  __syncthreads();
+  const bool over = s_over != 0;
+  if (over && tid == 0) record_status(status, DEV_BOUNDS, 601);
   for (int e = tid; e < E; e += blockDim.x) {
     const int first = (e / E_loc) * E_loc;  // first expert of e's owner
     int pad = 0;
     for (int q = first; q < e; ++q) pad += (s_tot[q] + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
-    dest_base[e] = pad + s_before[e];
+    dest_base[e] = over ? -1 : pad + s_before[e];
   }
-  for (int el = tid; el < E_loc; el += blockDim.x) s_cnt[el] = s_tot[rank * E_loc + el];
+  for (int el = tid; el < E_loc; el += blockDim.x) s_cnt[el] = over ? 0 : s_tot[rank * E_loc + el];
   __syncthreads();
   build_expert_tables(E_loc, s_cnt, s_tab, tabs);
 }
@@ -98,6 +113,10 @@ __global__ void __launch_bounds__(TOK_TILE) ep_scatter_kernel(int64_t T, int E, 
   if (t >= T) return;
   for (int j = 0; j < k; ++j) {
     const int e = idx[t * k + j];
+    if (dest_base[e] < 0) {  // the plan refused the step (the rows do not fit the owner buffers)
+      inv[t * k + j] = -1;
+      continue;
+    }
     int rank = tile_base[static_cast<int64_t>(blockIdx.x) * E + e];
     for (int w = 0; w < warp; ++w) rank += __popc(ep_masks[w * E + e]);
     rank += __popc(ep_masks[warp * E + e] & ((1u << lane) - 1u));
@@ -125,6 +144,7 @@ __global__ void __launch_bounds__(256) ep_scatter_rows_kernel(int64_t T, int d, 
     for (int i = 0; i < 8; ++i)
       if (c0 + lane + 32 * i < n16) v[i] = __ldg(s4 + c0 + lane + 32 * i);
     for (int j = 0; j < k; ++j) {
+      if (inv[t * k + j] < 0) continue;  // refused step
       uint4* dst = reinterpret_cast<uint4*>(peers.ws[idx[t * k + j] / E_loc] + buf_off) +
                    static_cast<int64_t>(inv[t * k + j]) * n16;
 #pragma unroll
@@ -144,8 +164,10 @@ __global__ void __launch_bounds__(256) ep_gather_sum_kernel(int d, int k, int E_
   const int64_t t = blockIdx.x;
   __shared__ const uint16_t* srow[MAX_K];
   if (threadIdx.x < k)
-    srow[threadIdx.x] = reinterpret_cast<const uint16_t*>(peers.ws[idx[t * k + threadIdx.x] / E_loc] + buf_off) +
-                        static_cast<int64_t>(inv[t * k + threadIdx.x]) * d;
+    srow[threadIdx.x] = inv[t * k + threadIdx.x] < 0  // refused step: the row does not exist, it counts as zeros
+                            ? nullptr
+                            : reinterpret_cast<const uint16_t*>(peers.ws[idx[t * k + threadIdx.x] / E_loc] + buf_off) +
+                                  static_cast<int64_t>(inv[t * k + threadIdx.x]) * d;
   __syncthreads();
   for (int c = threadIdx.x * 8; c < d; c += 256 * 8) {
     float acc[8];
@@ -160,6 +182,7 @@ __global__ void __launch_bounds__(256) ep_gather_sum_kernel(int d, int k, int E_
     }
 #pragma unroll 8
     for (int j = 0; j < k; ++j) {
+      if (!srow[j]) continue;
       const uint4 v = *reinterpret_cast<const uint4*>(srow[j] + c);
       float a, b;
       unpack_bf16x2(v.x, a, b); acc[0] += a; acc[1] += b;
@@ -186,7 +209,8 @@ __global__ void __launch_bounds__(256) ep_gather_dg_kernel(int64_t n, int E_loc,
   const float* part = reinterpret_cast<const float*>(peers.ws[idx[i] / E_loc] + dg_part_off);
   const int r = inv[i];
   float s = 0.f;
-  for (int nt = 0; nt < dg_tiles; ++nt) s += part[nt * rows_max + r];
+  if (r >= 0)
+    for (int nt = 0; nt < dg_tiles; ++nt) s += part[nt * rows_max + r];
   dg[i] = s;
 }
 
@@ -329,9 +353,10 @@ moe_status moe_ep_plan(moe_ctx* ctx, int64_t T, const int32_t* all_counts, void*
   char* ows = static_cast<char*>(own_ws);
   launch_prepare(l.own, ows, st);  // row gates of the owner buffers start at zero; status block
   const int E_loc = c->own->s.E;
-  ep_plan_kernel<<<1, 256, 0, st>>>(all_counts, c->ep_world, c->ep_rank, c->s.E, E_loc,
+  ep_plan_kernel<<<1, 256, 0, st>>>(all_counts, c->ep_world, c->ep_rank, c->s.E, E_loc, l.own.rows_max,
                                     reinterpret_cast<int32_t*>(static_cast<char*>(send_ws) + l.send.ep_dest),
-                                    table_pointers(l.own, ows));
+                                    table_pointers(l.own, ows),
+                                    reinterpret_cast<int32_t*>(static_cast<char*>(send_ws) + l.send.status));
   note_launch();
   ep_zero_pad_kernel<<<E_loc, 256, 0, st>>>(c->s.d, reinterpret_cast<const int32_t*>(ows + l.own.counts),
                                             reinterpret_cast<const int32_t*>(ows + l.own.pad_offsets),

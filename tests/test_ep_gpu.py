@@ -172,3 +172,58 @@ def test_ep_main_gradients_accumulate_over_micro_batches():
                 assert rel_fro(got[:-2], ref[n][own][:-2]) <= TOL, (r, n)
             else:
                 assert rel_fro(got, ref[n][own]) <= TOL, (r, n)
+
+
+def test_rows_beyond_the_owner_buffers_are_refused_not_written():
+    """A rows_cap that the routing exceeds: the plan refuses the step on every rank (same counts everywhere), nothing is
+    written outside or inside the owner buffers' rows (canaries behind every owner workspace stay intact), y and dx are
+    zeros, the failure is reported once as MOE_ERR_DEVICE_BOUNDS, and the same contexts then run a step that fits."""
+    from paper_2608_00916_b200.binding import MoEError
+    from gpu_util import Run
+    d, E, k, f, world = 128, 16, 4, 128, 2
+    rows_cap = 1024
+    probe = ep.EPRank(d, E, f, k, world, 0, rows_cap)
+    own_bytes = probe.own_bytes
+    del probe
+    canary = 1 << 20
+    bufs = [torch.full((own_bytes + canary,), 0xA5, dtype=torch.uint8, device="cuda") for _ in range(world)]
+    ranks = [ep.EPRank(d, E, f, k, world, r, rows_cap, own_ws=bufs[r][:own_bytes]) for r in range(world)]
+    for rk in ranks:
+        rk.set_peers([b.data_ptr() for b in bufs])
+    grp = ep.LocalGroup.__new__(ep.LocalGroup)
+    grp.world, grp.ranks = world, ranks
+
+    def run(tokens, seed):
+        shape = synth.MoEShape(sum(tokens), d, E, k, f)
+        inp = synth.make_inputs(shape, seed, x_std=1.0)
+        dev = {n: to_dev_bf16(inp[n]) for n in ("x", "W_r", "W_gate", "W_up", "W_down", "dy")}
+        b = np.concatenate([[0], np.cumsum(tokens)])
+        xs = [dev["x"][b[r]:b[r + 1]].contiguous() for r in range(world)]
+        dys = [dev["dy"][b[r]:b[r + 1]].contiguous() for r in range(world)]
+        fw, _ = grp.forward(xs, dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
+        sender, owner = grp.backward(dys, 0.0)
+        torch.cuda.synchronize()
+        return inp, fw, sender, owner
+
+    # 2 x 700 tokens x 4 slots = 5600 rows for 2 owners of 1024 rows each: does not fit
+    _, fw, sender, owner = run([700, 700], 71)
+    for r in range(world):
+        with pytest.raises(MoEError, match="bounds"):
+            ranks[r].poll()
+        ranks[r].poll()  # reported once
+        assert not fw[r]["y"].float().abs().sum().item() and not sender[r]["dx"].float().abs().sum().item()
+        for n in ("dW_gate", "dW_up", "dW_down"):
+            assert not owner[r][n].float().abs().sum().item()
+        assert bool((bufs[r][own_bytes:] == 0xA5).all())
+        assert bool((ranks[r].buffer("inv", torch.int32, False) == -1).all())
+    # a step that fits, on the same contexts: the oracle's results
+    tokens = [100, 60]
+    inp, fw, sender, owner = run(tokens, 72)
+    ofw, obw = oracle_run(inp, k, 0.0)
+    b = np.concatenate([[0], np.cumsum(tokens)])
+    for r in range(world):
+        ranks[r].poll()
+        assert np.array_equal(fw[r]["idx"].cpu().numpy(), ofw["idx"][b[r]:b[r + 1]])
+        assert rel_fro(from_dev_bf16(fw[r]["y"]), ofw["y"][b[r]:b[r + 1]]) <= TOL
+        assert rel_fro(from_dev_bf16(sender[r]["dx"]), obw["dx"][b[r]:b[r + 1]]) <= TOL
+        assert bool((bufs[r][own_bytes:] == 0xA5).all())
