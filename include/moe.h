@@ -189,7 +189,12 @@ MOE_API moe_status moe_forward_inference(moe_ctx* ctx, int64_t T, const uint16_t
  *   x, W_r, W_gate, W_up, W_down: the forward inputs
  * Outputs (all OVERWRITTEN, not accumulated)
  *   dx [T,d] bf16;  dW_r [d,E] fp32;  db_r [E] fp32 or NULL;
- *   dW_gate, dW_up [E,d,f] bf16;  dW_down [E,f,d] bf16 (zero slabs for experts without tokens). */
+ *   dW_gate, dW_up [E,d,f] bf16;  dW_down [E,f,d] bf16 (zero slabs for experts without tokens).
+ * The workspace must be the one a training forward call (moe_forward; moe_lora_forward for moe_lora_backward) filled
+ * for the SAME T, untouched in between: its tables drive every index of the backward kernels.  The context remembers
+ * what its recent forward calls left in which workspace (the last eight workspaces) and returns MOE_ERR_INVALID_ARG,
+ * before any launch, when the workspace was last filled for another T, by moe_forward_inference, or by the other
+ * variant of the layer. */
 MOE_API moe_status moe_backward(moe_ctx* ctx, int64_t T, const uint16_t* dy, float d_aux, const uint16_t* x,
                         const uint16_t* W_r, const uint16_t* W_gate, const uint16_t* W_up,
                         const uint16_t* W_down, uint16_t* dx, float* dW_r, float* db_r, uint16_t* dW_gate,

@@ -352,6 +352,24 @@ moe_status moe_stage_times(moe_ctx* ctx, float* ms, int32_t* steps) {
   return MOE_OK;
 }
 
+// Host-side record of which forward call filled which workspace (see moe_ctx_impl::fwd).
+static void note_forward(moe_ctx_impl* c, const void* ws, int64_t T, int kind) {
+  for (auto& r : c->fwd)
+    if (r.ws == ws) {
+      r.T = T;
+      r.kind = kind;
+      return;
+    }
+  c->fwd[c->fwd_next] = {ws, T, kind};
+  c->fwd_next = (c->fwd_next + 1) % 8;
+}
+// false when `ws` was last filled, by this context, for another token count or another variant of the layer
+static bool forward_matches(const moe_ctx_impl* c, const void* ws, int64_t T, int kind) {
+  for (const auto& r : c->fwd)
+    if (r.ws == ws) return r.T == T && r.kind == kind;
+  return true;  // not on record (filled long ago or never): the caller's word stands
+}
+
 static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r,
                                const float* b_r, const float* logits_in, const uint16_t* W_gate,
                                const uint16_t* W_up, const uint16_t* W_down, uint16_t* y, int32_t* topk_idx,
@@ -434,7 +452,9 @@ static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uin
                      c->debug_checks ? reinterpret_cast<int32_t*>(ws + L.status) : nullptr, L.rows_max);
     }
   }
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  note_forward(c, workspace, T, lora ? FWD_LORA + lora->rank : (training ? FWD_TRAINING : FWD_INFERENCE));
+  return MOE_OK;
 }
 
 moe_status moe_forward(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r, const float* b_r,
@@ -484,6 +504,9 @@ static moe_status backward_impl(moe_ctx* ctx, int64_t T, const uint16_t* dy, flo
     return MOE_ERR_INVALID_ARG;
   const WsLayout L = make_layout(s, T);
   if (workspace_bytes < (lora ? L.lora_total : L.total)) return MOE_ERR_WORKSPACE;
+  // the tables in the workspace are the forward call's: another token count or a forward-only / other-variant pass
+  // would send the index-driven kernels out of range
+  if (!forward_matches(c, workspace, T, lora ? FWD_LORA + lora->rank : FWD_TRAINING)) return MOE_ERR_INVALID_ARG;
   moe_status rc = ensure_device(c);
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

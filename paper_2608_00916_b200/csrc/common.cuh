@@ -122,7 +122,16 @@ struct moe_ctx_impl {
   int ep_world, ep_rank;
   int64_t ep_rows_cap;
   moe_ctx_impl* own;
+  // what the most recent forward calls of this context left in which workspace (host-side bookkeeping): a backward call
+  // on a workspace found here must name the same token count and variant, else its tables would index out of range
+  struct FwdRecord {
+    const void* ws;
+    int64_t T;
+    int kind;  // FWD_TRAINING, FWD_INFERENCE, or FWD_LORA + rank
+  } fwd[8];
+  int fwd_next;
 };
+constexpr int FWD_TRAINING = 1, FWD_INFERENCE = 2, FWD_LORA = 16;
 
 // binds the context to the current device on first use (api.cu)
 moe_status ensure_device(moe_ctx_impl* c);

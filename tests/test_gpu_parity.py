@@ -10,7 +10,7 @@ import torch
 
 from paper_2608_00916_b200 import synth
 from gpu_util import ROW_TOL, Run, from_dev_bf16, oracle_run, rel_fro, rows_max_err
-from paper_2608_00916_b200.binding import MoELayer
+from paper_2608_00916_b200.binding import MoELayer, kernel_launches as binding_launches
 from oracle import moe_oracle as orc
 
 pytestmark = pytest.mark.gpu
@@ -303,6 +303,44 @@ def test_two_contexts_on_two_streams():
             assert torch.equal(outs[i][0][n], v), (i, n)
         for n, v in alone[i][1].items():
             assert torch.equal(outs[i][1][n], v), (i, n)
+
+
+def test_backward_refuses_a_workspace_filled_by_another_forward():
+    """The tables in the workspace belong to the forward call that filled it: a backward call (straight through the C
+    ABI) naming another token count, or following a forward-only pass, is refused before any launch (it would index out
+    of range); the matching call still works afterwards."""
+    import ctypes as C
+    inp = synth.make_inputs(synth.MoEShape(600, 128, 8, 2, 128), 81)
+    r = Run(inp, 2)
+    r.forward()
+    good = r.backward(0.0)
+    layer, dev = r.layer, r.dev
+    p = lambda t: C.c_void_p(t.data_ptr())
+    out = {n: torch.empty_like(v) for n, v in good.items() if v is not None}
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def c_backward(T):
+        return layer.lib.moe_backward(layer.h, T, p(dev["dy"]), C.c_float(0.0), p(dev["x"]), p(dev["W_r"]), p(dev["W_gate"]),
+                                      p(dev["W_up"]), p(dev["W_down"]), p(out["dx"]), p(out["dW_r"]), None, p(out["dW_gate"]),
+                                      p(out["dW_up"]), p(out["dW_down"]), p(layer.ws), layer.ws.numel(), stream)
+
+    layer.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
+    before = binding_launches()
+    assert c_backward(300) == -1      # forward was for 600 tokens
+    assert binding_launches() == before
+    assert c_backward(600) == 0
+    torch.cuda.synchronize()
+    for n in ("dx", "dW_r", "dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(out[n], good[n]), n
+    # a forward-only pass leaves no pre-activations: no backward on its workspace
+    layer.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"], inference=True)
+    assert c_backward(600) == -1
+    layer.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
+    out["dx"].zero_()
+    assert c_backward(600) == 0
+    torch.cuda.synchronize()
+    layer.poll()
+    assert torch.equal(out["dx"], good["dx"])
 
 
 @pytest.mark.parametrize("T,d,E,k,f,seed", [(1000, 512, 16, 4, 384, 14), (777, 256, 64, 8, 192, 27)])
