@@ -273,7 +273,8 @@ MOE_API moe_status moe_lora_backward(moe_ctx* ctx, int64_t T, int32_t rank, floa
  *              moe_ep_expert_forward | barrier | moe_ep_combine
  *   backward:  moe_ep_dispatch(dy, backward = 1) | barrier | moe_ep_expert_backward | barrier | moe_ep_router_backward
  *
- * Results are those of the one-GPU layer applied to the concatenation of the ranks' batches in rank order (same row
+ * Every phase that takes T must name the T of the moe_ep_route call that filled the sender workspace (the context
+ * checks this on the host and returns MOE_ERR_INVALID_ARG otherwise).  Results are those of the one-GPU layer applied to the concatenation of the ranks' batches in rank order (same row
  * order inside every expert), except that aux_loss, its gradient and dW_r / db_r are per rank, over the rank's own
  * tokens (each rank is also a data-parallel rank for the router weight; sum dW_r over the group as for any replicated
  * parameter).  Requirements: E a multiple of `world` and of 8, world <= MOE_EP_MAX_RANKS.

@@ -352,24 +352,6 @@ moe_status moe_stage_times(moe_ctx* ctx, float* ms, int32_t* steps) {
   return MOE_OK;
 }
 
-// Host-side record of which forward call filled which workspace (see moe_ctx_impl::fwd).
-static void note_forward(moe_ctx_impl* c, const void* ws, int64_t T, int kind) {
-  for (auto& r : c->fwd)
-    if (r.ws == ws) {
-      r.T = T;
-      r.kind = kind;
-      return;
-    }
-  c->fwd[c->fwd_next] = {ws, T, kind};
-  c->fwd_next = (c->fwd_next + 1) % 8;
-}
-// false when `ws` was last filled, by this context, for another token count or another variant of the layer
-static bool forward_matches(const moe_ctx_impl* c, const void* ws, int64_t T, int kind) {
-  for (const auto& r : c->fwd)
-    if (r.ws == ws) return r.T == T && r.kind == kind;
-  return true;  // not on record (filled long ago or never): the caller's word stands
-}
-
 static moe_status forward_impl(bool training, moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16_t* W_r,
                                const float* b_r, const float* logits_in, const uint16_t* W_gate,
                                const uint16_t* W_up, const uint16_t* W_down, uint16_t* y, int32_t* topk_idx,

@@ -131,7 +131,24 @@ struct moe_ctx_impl {
   } fwd[8];
   int fwd_next;
 };
-constexpr int FWD_TRAINING = 1, FWD_INFERENCE = 2, FWD_LORA = 16;
+constexpr int FWD_TRAINING = 1, FWD_INFERENCE = 2, FWD_EP = 3, FWD_LORA = 16;
+// Host-side record of which forward call (for the expert-parallel path: which moe_ep_route call) filled which workspace.
+inline void note_forward(moe_ctx_impl* c, const void* ws, int64_t T, int kind) {
+  for (auto& r : c->fwd)
+    if (r.ws == ws) {
+      r.T = T;
+      r.kind = kind;
+      return;
+    }
+  c->fwd[c->fwd_next] = {ws, T, kind};
+  c->fwd_next = (c->fwd_next + 1) % 8;
+}
+// false when `ws` was last filled, by this context, for another token count or another variant of the layer
+inline bool forward_matches(const moe_ctx_impl* c, const void* ws, int64_t T, int kind) {
+  for (const auto& r : c->fwd)
+    if (r.ws == ws) return r.T == T && r.kind == kind;
+  return true;  // not on record (filled long ago or never): the caller's word stands
+}
 
 // binds the context to the current device on first use (api.cu)
 moe_status ensure_device(moe_ctx_impl* c);

@@ -337,7 +337,9 @@ moe_status moe_ep_route(moe_ctx* ctx, int64_t T, const uint16_t* x, const uint16
   }
   launch_permute(s, T, L, ws, x, counts_local, nullptr, aux_loss, static_cast<int>(router_psum_rows(s, T, false)), st,
                  /*tables_only=*/true, /*histogram_done=*/T > 0 && router_writes_histogram(s));
-  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  note_forward(c, send_ws, T, FWD_EP);  // the later phases on this sender workspace must name the same T
+  return MOE_OK;
 }
 
 moe_status moe_ep_plan(moe_ctx* ctx, int64_t T, const int32_t* all_counts, void* send_ws, size_t send_ws_bytes,
@@ -346,6 +348,7 @@ moe_status moe_ep_plan(moe_ctx* ctx, int64_t T, const int32_t* all_counts, void*
   if (!c || !c->own || T < 0 || !all_counts || !send_ws || !own_ws || !aligned16(own_ws)) return MOE_ERR_INVALID_ARG;
   const EpLayouts l = ep_layouts(c, T);
   if (send_ws_bytes < l.send.total || own_ws_bytes < l.own.total) return MOE_ERR_WORKSPACE;
+  if (!forward_matches(c, send_ws, T, FWD_EP)) return MOE_ERR_INVALID_ARG;
   moe_status rc = ensure_device(c);
   if (rc == MOE_OK) rc = ensure_device(c->own);
   if (rc != MOE_OK) return rc;
@@ -372,6 +375,7 @@ moe_status moe_ep_dispatch(moe_ctx* ctx, int64_t T, const uint16_t* src, int bac
   if (T > 0 && (!src || !aligned16(src))) return MOE_ERR_INVALID_ARG;
   const EpLayouts l = ep_layouts(c, T);
   if (send_ws_bytes < l.send.total) return MOE_ERR_WORKSPACE;
+  if (!forward_matches(c, send_ws, T, FWD_EP)) return MOE_ERR_INVALID_ARG;
   if (T == 0) return MOE_OK;
   const moe_status rc = ensure_device(c);
   if (rc != MOE_OK) return rc;
@@ -421,6 +425,7 @@ moe_status moe_ep_combine(moe_ctx* ctx, int64_t T, void* const* peer_own_ws, con
   if (T > 0 && (!y || !aligned16(y))) return MOE_ERR_INVALID_ARG;
   const EpLayouts l = ep_layouts(c, T);
   if (send_ws_bytes < l.send.total) return MOE_ERR_WORKSPACE;
+  if (!forward_matches(c, send_ws, T, FWD_EP)) return MOE_ERR_INVALID_ARG;
   if (T == 0) return MOE_OK;
   const char* ws = static_cast<const char*>(send_ws);
   ep_gather_sum_kernel<<<static_cast<unsigned>(T), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
@@ -485,6 +490,7 @@ moe_status moe_ep_router_backward(moe_ctx* ctx, int64_t T, float d_aux, const ui
   if (!aligned16(x) || !aligned16(W_r) || !aligned16(dx) || !aligned16(send_ws)) return MOE_ERR_INVALID_ARG;
   const EpLayouts l = ep_layouts(c, T);
   if (send_ws_bytes < l.send.total) return MOE_ERR_WORKSPACE;
+  if (!forward_matches(c, send_ws, T, FWD_EP)) return MOE_ERR_INVALID_ARG;
   moe_status rc = ensure_device(c);
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -227,3 +227,24 @@ def test_rows_beyond_the_owner_buffers_are_refused_not_written():
         assert rel_fro(from_dev_bf16(fw[r]["y"]), ofw["y"][b[r]:b[r + 1]]) <= TOL
         assert rel_fro(from_dev_bf16(sender[r]["dx"]), obw["dx"][b[r]:b[r + 1]]) <= TOL
         assert bool((bufs[r][own_bytes:] == 0xA5).all())
+
+
+def test_phases_must_name_the_routed_token_count():
+    """The sender workspace holds the routing of moe_ep_route's T tokens: a later phase that names another T is refused
+    on the host before any launch."""
+    import ctypes as C
+    d, E, k, f = 128, 8, 2, 128
+    inp = synth.make_inputs(synth.MoEShape(200, d, E, k, f), 91)
+    x, W_r = to_dev_bf16(inp["x"]), to_dev_bf16(inp["W_r"])
+    rk = ep.EPRank(d, E, f, k, 1, 0, 200 * k)
+    rk.set_peers([rk.own_ws.data_ptr()])
+    out = rk.route(x, W_r)
+    rk.plan(out["counts_local"].view(1, E).contiguous())
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    p = lambda t: C.c_void_p(t.data_ptr())
+    assert rk.lib.moe_ep_dispatch(rk.h, 100, p(x), 0, rk.peers, p(rk.send_ws), rk.send_ws.numel(), stream) == -1
+    y = torch.empty(200, d, dtype=torch.bfloat16, device="cuda")
+    assert rk.lib.moe_ep_combine(rk.h, 199, rk.peers, p(rk.send_ws), rk.send_ws.numel(), p(y), stream) == -1
+    assert rk.lib.moe_ep_dispatch(rk.h, 200, p(x), 0, rk.peers, p(rk.send_ws), rk.send_ws.numel(), stream) == 0
+    torch.cuda.synchronize()
+    rk.poll()
