@@ -287,6 +287,7 @@ def main():
                          "buffers zeroed once per window)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay of the step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -580,6 +581,41 @@ def main():
     ms_step = pdist.max_over_ranks(ev0.elapsed_time(ev1)) / args.steps
     value = pdist.job_throughput(T, ms_step)  # tokens of all ranks over the slowest rank's time
 
+    # ---- the same step replayed from a CUDA graph (informative: what a training loop that captures its step gets; the
+    # library's calls are legal inside a stream capture, second stream included).  Only the plain training step.
+    graph = None
+    if args.mode == "train" and acc is None and not args.no_graph:
+        cap = torch.cuda.Stream()
+        cap.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(cap):
+            step()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=cap):
+                step()
+        torch.cuda.synchronize()
+        for _ in range(max(3, args.warmup)):
+            g.replay()
+        t_c = time.perf_counter()  # the capture paused the GPU: settle the power state again, as for the headline
+        while time.perf_counter() - t_c < args.condition_seconds:
+            for _ in range(10):
+                g.replay()
+            torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pdist.barrier()
+        torch.cuda.synchronize()
+        g0.record()
+        for _ in range(args.steps):
+            g.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        layer.poll()
+        gms = pdist.max_over_ranks(g0.elapsed_time(g1)) / args.steps
+        graph = {"ms_per_step": gms, "tokens_per_s": world * T / (gms / 1e3), "steps": args.steps,
+                 "note": "the timed step captured once and replayed after the same conditioning (no per-stage events, "
+                         "one launch per step); informative, the headline is the eager step"}
+        del g
+
     # ---- end to end through the host-buffer entry point (weights resident, activations cross PCIe each step)
     e2e = None
     if not args.no_e2e:
@@ -716,7 +752,8 @@ def main():
             "grouped_gemm_frac_of_sustained_bf16": gemm_tflops / peaks["bf16_tflops_sustained"],
             "grouped_gemm_frac_of_burst_bf16": gemm_tflops / peaks["bf16_tflops"],
             "grouped_gemm_frac_of_regime_peak": gemm_tflops / tensor_peak, "regime": regime,
-            "roofline": roof, "stages": stages, "burst": burst, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+            "roofline": roof, "stages": stages, "burst": burst, "graph_replay": graph, "cpu_baseline": cpu, "e2e": e2e,
+            "clocks": clocks,
             "gpu_launches": launches}
     print(json.dumps(line))
     pdist.finish()

@@ -35,6 +35,7 @@ def test_gpu_arm_prints_the_contract_line():
     assert e2e["value"] > 0 and e2e["h2d_bytes_per_step"] == 2 * 256 * 256 * 2 and e2e["d2h_bytes_per_step"] > 0
     assert e2e["value"] != d["value"]
     assert "sm_mhz" in d["clocks"] and "reasons" in d["clocks"]
+    assert d["graph_replay"]["ms_per_step"] > 0 and d["graph_replay"]["steps"] == 5
     rt = d["routing"]
     assert rt["rows_per_expert"]["mean"] == 256 * 2 / 8 and rt["empty_experts"] == 0 and len(rt["largest_five"]) == 5
     assert d["gpu_launches"] >= 5 * 10  # kernels of this library inside the timed region (5 steps)
