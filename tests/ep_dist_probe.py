@@ -28,6 +28,7 @@ def main():
     bw = layer.backward(dev["dy"], 0.03)
     layer.poll()
     grp = ep.DistGroup(shape.d, shape.E, shape.f, shape.k, shape.T * shape.k)
+    print("DIST_GROUP_READY", flush=True)  # the process group and the symmetric-memory rendezvous exist
     out = grp.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
     sender, owner = grp.backward(dev["dy"], 0.03)
     torch.cuda.synchronize()
