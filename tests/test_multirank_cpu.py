@@ -35,7 +35,8 @@ def _worker(rank, world, port, q):
 def test_two_gloo_ranks():
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 29650 + os.getpid() % 200
+    from paper_2608_00916_b200.dist import free_port
+    port = free_port()
     procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
     for p in procs:
         p.start()
@@ -79,7 +80,8 @@ def test_gradient_all_reduce_over_two_gloo_ranks():
     the sum of both ranks' weight gradients (bucketed along the expert axis, asynchronous)."""
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 29850 + os.getpid() % 100
+    from paper_2608_00916_b200.dist import free_port
+    port = free_port()
     procs = [ctx.Process(target=_reduce_worker, args=(r, 2, port, q)) for r in range(2)]
     for p in procs:
         p.start()
@@ -235,7 +237,8 @@ def test_expert_parallel_exchange_over_gloo_ranks(world):
     oracle's on the concatenated batch (routing bit-exact, values to rounding)."""
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 29950 + os.getpid() % 40 + 3 * world
+    from paper_2608_00916_b200.dist import free_port
+    port = free_port()
     procs = [ctx.Process(target=_ep_worker, args=(r, world, port, q)) for r in range(world)]
     for p in procs:
         p.start()
