@@ -245,11 +245,14 @@ class LocalGroup:
 
 class DistGroup:
     """One rank per process and GPU (torch.distributed initialised with the NCCL backend).  The owner workspace lives in
-    symmetric memory so that every rank can map its peers' copies; the per-rank expert counts travel by all_gather; a
-    group barrier (stream synchronise + dist.barrier) separates the phases.  The tests run it on a one-rank group (they
-    have one GPU; LocalGroup runs the same kernels for more ranks there)."""
+    symmetric memory so that every rank can map its peers' copies; the per-rank expert counts travel by all_gather.
+    The group barrier between phases is, by default, the symmetric-memory handle's device-side barrier (a small kernel
+    on the current stream in which the ranks signal one another through their signal pads, release / acquire at system
+    scope, with the library's own time-out): the stream never drains and the host never waits.  device_barrier=False
+    falls back to a host barrier (stream synchronise + dist.barrier).  The tests run both on a one-rank group (they have
+    one GPU; LocalGroup runs the same kernels for more ranks there)."""
 
-    def __init__(self, d, E, f, top_k, rows_cap, flags: int = 0, group=None):
+    def __init__(self, d, E, f, top_k, rows_cap, flags: int = 0, group=None, device_barrier: bool = True):
         import torch
         import torch.distributed as dist
         import torch.distributed._symmetric_memory as symm
@@ -260,10 +263,15 @@ class DistGroup:
         hdl = symm.rendezvous(buf, group if group is not None else dist.group.WORLD)
         self.rk = EPRank(d, E, f, top_k, self.world, self.rank, rows_cap, flags, own_ws=buf)
         self.rk.set_peers(list(hdl.buffer_ptrs))
+        self.hdl = hdl
+        self.device_barrier = bool(device_barrier) and hasattr(hdl, "barrier")
         del probe
 
     def _barrier(self):
         import torch
+        if self.device_barrier:
+            self.hdl.barrier()  # enqueued on the current stream
+            return
         torch.cuda.current_stream().synchronize()
         self.dist.barrier(self.group)
 

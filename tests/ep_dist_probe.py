@@ -27,14 +27,20 @@ def main():
     fw = layer.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
     bw = layer.backward(dev["dy"], 0.03)
     layer.poll()
-    grp = ep.DistGroup(shape.d, shape.E, shape.f, shape.k, shape.T * shape.k)
-    print("DIST_GROUP_READY", flush=True)  # the process group and the symmetric-memory rendezvous exist
-    out = grp.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
-    sender, owner = grp.backward(dev["dy"], 0.03)
-    torch.cuda.synchronize()
-    grp.rk.poll()
-    same = (torch.equal(out["y"], fw["y"]) and torch.equal(out["idx"], fw["idx"]) and torch.equal(sender["dx"], bw["dx"])
-            and torch.equal(sender["dW_r"], bw["dW_r"]) and all(torch.equal(owner[n], bw[n]) for n in ("dW_gate", "dW_up", "dW_down")))
+    same = True
+    for device_barrier in (True, False):
+        grp = ep.DistGroup(shape.d, shape.E, shape.f, shape.k, shape.T * shape.k, device_barrier=device_barrier)
+        if device_barrier:
+            print("DIST_GROUP_READY", flush=True)  # the process group and the symmetric-memory rendezvous exist
+            print("DEVICE_BARRIER", grp.device_barrier, flush=True)
+        out = grp.forward(dev["x"], dev["W_r"], dev["W_gate"], dev["W_up"], dev["W_down"])
+        sender, owner = grp.backward(dev["dy"], 0.03)
+        torch.cuda.synchronize()
+        grp.rk.poll()
+        same = same and (torch.equal(out["y"], fw["y"]) and torch.equal(out["idx"], fw["idx"])
+                         and torch.equal(sender["dx"], bw["dx"]) and torch.equal(sender["dW_r"], bw["dW_r"])
+                         and all(torch.equal(owner[n], bw[n]) for n in ("dW_gate", "dW_up", "dW_down")))
+        del grp
     dist.destroy_process_group()
     print("DIST_GROUP_OK" if same else "DIST_GROUP_MISMATCH")
 
