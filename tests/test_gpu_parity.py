@@ -699,6 +699,23 @@ def test_grouped_weight_gradients_signal_ranges_of_experts():
     assert touched == [(5, f, d)] * 4 + [(4, f, d)] + [(5, d, f)] * 8 + [(4, d, f)] * 2 + [(d, E)]
 
 
+def test_grouped_reduction_through_nccl_on_a_one_rank_group():
+    """The data-parallel gradient path with the real collective (NCCL all_reduce per range of experts on the reducer's
+    stream, as the grouped backward signals the ranges) in a child process on a one-rank group, where summing over the
+    ranks changes nothing: bitwise the plain accumulation window.  More ranks need more GPUs than a test run has."""
+    import os
+    import subprocess
+    import sys
+    from paper_2608_00916_b200.dist import free_port
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "tests", "dp_reduce_probe.py"), str(free_port())],
+                         capture_output=True, text=True, timeout=600, cwd=root)
+    if "GROUP_READY" not in out.stdout:
+        pytest.skip("this box cannot host a NCCL group: " + out.stderr[-300:])
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "REDUCE_OK" in out.stdout, out.stdout[-500:] + out.stderr[-1500:]
+
+
 def test_fp32_router_weight():
     """MOE_FLAG_ROUTER_FP32: W_r arrives as genuine fp32 values (not representable in bf16); the library splits it into
     three exact bf16 terms, so logits, routing and gradients follow the oracle evaluated with the fp32 weight."""
