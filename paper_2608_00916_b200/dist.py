@@ -67,7 +67,11 @@ def launch_ranks(n: int, script: str, argv, port: int | None = None, python: str
 def barrier() -> None:
     if _state["world"] > 1:
         import torch.distributed as dist
-        dist.barrier()
+        if _state["backend"] == "nccl":
+            import torch
+            dist.barrier(device_ids=[torch.cuda.current_device()])  # the rank's own GPU, not a guess from the rank number
+        else:
+            dist.barrier()
 
 
 def max_over_ranks(value: float) -> float:
