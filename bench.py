@@ -735,7 +735,7 @@ def main():
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:  # the oracle is timed beside the one-GPU run only
         sample_T = min(T, 16384)
         v, dt = oracle_sample_tokens_per_s(inp, shape, sample_T)
         cpu = {"value": v, "unit": "tokens/s", "cores": host_cores(), "kind": "oracle", "seconds": dt,
