@@ -38,7 +38,7 @@ struct EpPeers {
 
 // ---------------------------------------------------------------------------------------------- plan
 // One block.  all_counts[r * E + e]: rows rank r routes to expert e.
-// Every rank sees the same table, so every rank reaches the same verdict on whether the rows fit: if the padded rows
+// Every rank sees the same table, so every rank reaches the same decision on whether the rows fit: if the padded rows
 // of ANY owner exceed the capacity of the owner buffers (own_rows_max rows, the same on every rank of the group), the
 // whole step is refused on every rank - all destinations become -1 (nothing is dispatched, combined outputs are zero),
 // the owned experts get empty tables, and the sender workspace's status word records DEV_BOUNDS.
